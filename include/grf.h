@@ -1,0 +1,146 @@
+/*
+ * grf.h — C ABI of the GRF-masked linear-attention library (CUDA, sm_100a).
+ *
+ * The library evaluates linear attention under the topological mask M_alpha = sum_k alpha_k W^k
+ * (Eq. 4), replaced by its sparse Monte-Carlo factorisation Mhat = Phi Psi^T built from halting
+ * random walks (graph random features, Eq. 10), following Alg. 1.
+ *
+ * Conventions for every call
+ *   - returns 0 (GRF_OK) or a negative GRF_ERR_* code; nothing is thrown or printed;
+ *   - "DEVICE" pointers are plain CUDA device addresses on the context's device, "HOST" pointers
+ *     are ordinary host memory; the library never takes ownership of a caller's buffer;
+ *   - all device work is enqueued on the context's stream; unless a call says otherwise it
+ *     returns without waiting for that work;
+ *   - a context is not thread-safe: one host thread at a time per context;
+ *   - matrices are CSR with int32 row pointers/column indices (ascending inside a row) and fp32 values.
+ */
+#ifndef GRF_H
+#define GRF_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define GRF_OK              0
+#define GRF_ERR_INVALID    (-1)  /* NULL pointer, non-positive size, p_halt outside [0,1), unsupported m/d/dtype */
+#define GRF_ERR_TOO_LARGE  (-2)  /* a size exceeds a documented limit                                            */
+#define GRF_ERR_WORKSPACE  (-3)  /* caller's workspace too small                                                 */
+#define GRF_ERR_CUDA       (-4)  /* a CUDA runtime call failed                                                   */
+#define GRF_ERR_NOMEM      (-5)  /* device or host allocation failed                                             */
+#define GRF_ERR_BADGRAPH   (-6)  /* CSR input inconsistent (host-side checks of host-resident graphs only)       */
+
+#define GRF_DTYPE_F32  0
+#define GRF_DTYPE_BF16 1
+
+#define GRF_MAX_WALK_LEN 255     /* largest max_len accepted by the sampler */
+
+typedef struct grf_ctx grf_ctx;            /* device id, stream, reusable scratch                         */
+typedef struct grf_features grf_features;  /* device-resident Phi (N x R), Psi (N x R), Psi^T (R x N)     */
+
+/* Context bound to `device` and to the CUDA stream `cuda_stream` (a cudaStream_t passed as void*;
+ * NULL = the default stream).  Scratch buffers grow on demand and live until destroy. */
+int grf_ctx_create(grf_ctx** out, int device, void* cuda_stream);
+int grf_ctx_destroy(grf_ctx* ctx);   /* waits for the stream, frees scratch; features are freed separately */
+
+/* Remark 3.1: f with sum_{p=0..k} f_p f_{k-p} = alpha_k, k < len (fp64 recurrence on the host).
+ * HOST pointers.  GRF_ERR_INVALID unless alpha[0] > 0. */
+int grf_deconvolve(const double* alpha, int32_t len, double* f_out);
+
+/*
+ * Alg. 1 steps 1-2 (Sec. 3.3, Eqs. 9-10): simulate n_walks halting random walks out of every node for
+ * each of two independent ensembles and assemble the sparse feature matrices Phi (ensemble 0, modulation
+ * f_phi) and Psi (ensemble 1, modulation f_psi), plus Psi^T grouped by visited node.
+ *
+ *   N, rowptr[N+1], col[E], w[E]   DEVICE  CSR of the weighted adjacency matrix W
+ *   seed                                   64-bit key of the counter-based generator
+ *   n_walks >= 1, 0 <= p_halt < 1, 0 <= max_len <= GRF_MAX_WALK_LEN
+ *   f_phi[max_len+1], f_psi[max_len+1]  HOST  modulation coefficients; f_psi == NULL means f_phi
+ *   *inout   NULL: a new feature object is created; otherwise that object's buffers are reused
+ *            (regrown if needed) and its previous contents are overwritten.
+ *
+ * Walk rule: the walk from node i deposits f_t * load_t / n_walks at the node reached after t hops
+ * (nothing when f_t == 0), load_0 = 1 and load_{t+1} = load_t * W_uv * deg(u) / (1 - p_halt) for the hop
+ * u -> v; before every hop it halts with probability p_halt; it also stops after max_len hops or at a
+ * node without neighbours.  Random words come from Philox4x32-10 keyed by `seed` with counter
+ * (node, walk, t/2, ensemble): the result depends only on these, never on launch geometry.
+ * Deposits of a row that hit the same column are added in ascending (walk, t) order.
+ *
+ * Limits: n_walks*(max_len+1) <= 16384 and N * 2^ceil(log2(n_walks*(max_len+1))) <= 2^32, else
+ * GRF_ERR_TOO_LARGE.  The call waits once for the device (it reads back the two nonzero counts).
+ */
+int grf_sample(grf_ctx* ctx, int32_t N, const int32_t* rowptr, const int32_t* col, const float* w,
+               uint64_t seed, int32_t n_walks, float p_halt, int32_t max_len,
+               const float* f_phi, const float* f_psi, grf_features** inout);
+
+/* The walks themselves, for checking (Sec. 3.3): traj and load are DEVICE arrays
+ * [2][N][n_walks][max_len+1]; traj holds the node at step t or -1 after the walk ended, load the
+ * importance weight of that prefix (0 after the end).  Same arguments and limits as grf_sample. */
+int grf_debug_walks(grf_ctx* ctx, int32_t N, const int32_t* rowptr, const int32_t* col, const float* w,
+                    uint64_t seed, int32_t n_walks, float p_halt, int32_t max_len,
+                    int32_t* traj, float* load);
+
+/* Feature object from caller-made matrices (DEVICE CSR, N x R each); copies them and builds Psi^T.
+ * Used for the special case Psi = I (asymmetric features, App. "Asymmetric graph random features")
+ * and for tests.  nnz are read from the row pointers: waits for the device once. */
+int grf_features_from_csr(grf_ctx* ctx, int32_t N, int32_t R,
+                          const int32_t* phi_rowptr, const int32_t* phi_col, const float* phi_val,
+                          const int32_t* psi_rowptr, const int32_t* psi_col, const float* psi_val,
+                          grf_features** out);
+
+/* Borrowed DEVICE pointers into a feature object: which = 0 Phi, 1 Psi, 2 Psi^T.  Valid until the
+ * object is freed or resampled.  rows/cols/nnz are returned through HOST pointers (any may be NULL). */
+int grf_features_view(const grf_features* feat, int which, int32_t* rows, int32_t* cols, int64_t* nnz,
+                      const int32_t** rowptr, const int32_t** col, const float** val);
+int grf_features_free(grf_features* feat);
+
+/* Regroups a DEVICE CSR matrix (rows x cols, nnz = rowptr[rows] passed by the caller) by column:
+ * t_rowptr[cols+1], t_col[nnz], t_val[nnz] DEVICE outputs; inside an output row the source rows ascend
+ * (Psi -> Psi^T, which turns Phi_K^T V of Alg. 1 step 5 into a segmented reduction).  Asynchronous. */
+int grf_csr_transpose(grf_ctx* ctx, int32_t rows, int32_t cols, int64_t nnz,
+                      const int32_t* rowptr, const int32_t* col, const float* val,
+                      int32_t* t_rowptr, int32_t* t_col, float* t_val);
+
+/* Bytes of DEVICE workspace with which grf_masked_linear_attn processes all G problems in one pass
+ * (states S [G][R][m][d] in the storage type and z [G][R][m] in fp32).  A smaller workspace is accepted
+ * as long as it holds one problem; the call then works through G in chunks.  0 on invalid arguments. */
+size_t grf_attn_workspace_bytes(int32_t G, int32_t R, int32_t m, int32_t d, int dtype);
+
+/*
+ * Alg. 1 step 5 / Eq. 12 for G independent problems (batch x heads) sharing one feature object:
+ *   S_l = sum_j Psi_jl phi(k_j) v_j^T,  z_l = sum_j Psi_jl phi(k_j)              (per problem, per node l)
+ *   out_i = sum_l Phi_il phi(q_i)^T S_l / sum_l Phi_il phi(q_i)^T z_l
+ * phiQ, phiK [G][N][m], V [G][N][d], out [G][N][d]: DEVICE, row-major, 16-byte aligned, dtype
+ * GRF_DTYPE_F32 or _BF16 (bf16: S is stored in bf16, sums are carried in fp32).  den_out: optional
+ * DEVICE fp32 [G][N] receiving the denominators.  A row whose denominator is exactly 0 yields out = 0.
+ * m, d in {8, 16, 32, 64, 128}.  workspace: DEVICE, 256-byte aligned.  Summation order is fixed, so
+ * results are run-to-run identical.  Asynchronous.
+ */
+int grf_masked_linear_attn(grf_ctx* ctx, const grf_features* feat, int32_t G, int32_t N, int32_t m, int32_t d,
+                           int dtype, const void* phiQ, const void* phiK, const void* V,
+                           void* out, float* den_out, void* workspace, size_t workspace_bytes);
+
+/*
+ * The whole path of Alg. 1 from HOST buffers, for callers that keep nothing on the device:
+ * copies the graph and phi(Q), phi(K), V to the device, samples features, evaluates the attention and
+ * copies `out` ([G][N][d], dtype) back; returns after the result is in `out`.  Device buffers and the
+ * feature object are owned by the context and reused by later calls.  Graph consistency (monotone
+ * rowptr, indices in range) is checked on the host: GRF_ERR_BADGRAPH.
+ */
+int grf_step_host(grf_ctx* ctx, int32_t N, const int32_t* rowptr, const int32_t* col, const float* w,
+                  uint64_t seed, int32_t n_walks, float p_halt, int32_t max_len,
+                  const float* f_phi, const float* f_psi,
+                  int32_t G, int32_t m, int32_t d, int dtype,
+                  const void* phiQ, const void* phiK, const void* V, void* out);
+
+/* Number of kernels the context has launched since it was created (for accounting in benchmarks). */
+int64_t grf_ctx_launch_count(const grf_ctx* ctx);
+
+const char* grf_strerror(int code);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* GRF_H */

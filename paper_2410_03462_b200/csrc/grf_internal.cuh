@@ -1,0 +1,88 @@
+// Internal declarations shared by the library's translation units (not part of the C ABI).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "grf.h"
+
+#define GRF_CUDA_TRY(expr)                                  \
+    do {                                                    \
+        cudaError_t _e = (expr);                            \
+        if (_e != cudaSuccess) return GRF_ERR_CUDA;         \
+    } while (0)
+
+#define GRF_TRY(expr)                                       \
+    do {                                                    \
+        int _rc = (expr);                                   \
+        if (_rc != GRF_OK) return _rc;                      \
+    } while (0)
+
+// A device buffer that only ever grows; owned by a context or a feature object.
+struct grf_buf {
+    void* ptr = nullptr;
+    size_t bytes = 0;
+};
+
+struct grf_ctx {
+    int device = 0;
+    cudaStream_t stream = nullptr;
+    int sm_count = 0;
+    int64_t launches = 0;
+    // sampler scratch
+    grf_buf stage_col, stage_val;   // merged rows at a fixed stride, before compaction
+    grf_buf counts;                 // per-row nonzero counts (both matrices)
+    grf_buf rowptr2;                // scanned counts, [2][N+1]
+    grf_buf scan_blocks;            // block totals of the two-level scan
+    // transpose scratch
+    grf_buf t_cursor, t_tmp_col, t_tmp_val;
+    // host-buffer path
+    grf_buf h_rowptr, h_col, h_w, h_q, h_k, h_v, h_out, h_ws;
+    grf_features* h_feat = nullptr;
+    int32_t* pinned = nullptr;      // small pinned host block for read-backs
+};
+
+struct grf_csr_dev {
+    int32_t rows = 0, cols = 0;
+    int64_t nnz = 0;
+    grf_buf rowptr, col, val;
+};
+
+struct grf_features {
+    int device = 0;
+    grf_csr_dev phi, psi, psit;
+};
+
+int grf_buf_reserve(grf_buf* b, size_t bytes);          // grows (contents not preserved)
+void grf_buf_release(grf_buf* b);
+int grf_csr_reserve(grf_csr_dev* m, int32_t rows, int32_t cols, int64_t nnz_cap);
+
+// sample.cu
+struct grf_walk_params {
+    int32_t N, n_walks, max_len;
+    uint32_t key0, key1, halt_threshold;
+    float inv_keep, inv_n;
+    int32_t cap;        // n_walks * (max_len + 1)
+    int32_t seq_bits;   // ceil(log2(cap)), at least 1
+    float f[2][GRF_MAX_WALK_LEN + 1];
+};
+int grf_walk_params_init(grf_walk_params* p, int32_t N, uint64_t seed, int32_t n_walks, float p_halt,
+                         int32_t max_len, const float* f_phi, const float* f_psi);
+
+// scan.cu: exclusive scan of `segments` independent int32 arrays of length n each (in[s*n + i]) into
+// out[s*(n+1) + i], with out[s*(n+1) + n] = total.
+int grf_exclusive_scan(grf_ctx* ctx, const int32_t* in, int32_t* out, int32_t n, int32_t segments);
+
+// transpose.cu
+int grf_transpose_launch(grf_ctx* ctx, int32_t rows, int32_t cols, int64_t nnz,
+                         const int32_t* rowptr, const int32_t* col, const float* val,
+                         int32_t* t_rowptr, int32_t* t_col, float* t_val);
+
+// attn_state.cu / attn_gather.cu
+int grf_build_states(grf_ctx* ctx, const grf_csr_dev& psit, int32_t G, int32_t N, int32_t m, int32_t d, int dtype,
+                     const void* phiK, const void* V, void* S, float* z);
+int grf_gather_contract(grf_ctx* ctx, const grf_csr_dev& phi, int32_t G, int32_t N, int32_t m, int32_t d, int dtype,
+                        const void* phiQ, const void* S, const float* z, void* out, float* den_out);
+
+static inline int grf_ceil_div(int64_t a, int64_t b) { return (int)((a + b - 1) / b); }

@@ -1,0 +1,112 @@
+// Psi -> Psi^T: regroup a CSR matrix by column (Alg. 1 step 5 needs, for every node l, the list of
+// keys j with Psi_jl != 0, so that Phi_K^T V becomes a segmented reduction with a fixed order).
+//
+// Bucket sort keyed on the full column index: count per column (integer atomics, order-free), scan,
+// scatter into the buckets in arrival order, then order every bucket by source row.  Source rows
+// inside a bucket are distinct, so the result is unique whatever the arrival order was.
+#include "grf_internal.cuh"
+
+namespace {
+
+__global__ void __launch_bounds__(256)
+column_histogram_kernel(int64_t nnz, const int32_t* __restrict__ col, int32_t* __restrict__ counts)
+{
+    for (int64_t p = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; p < nnz; p += (int64_t)gridDim.x * blockDim.x)
+        atomicAdd(counts + col[p], 1);
+}
+
+__global__ void __launch_bounds__(256)
+bucket_scatter_kernel(int32_t rows, const int32_t* __restrict__ rowptr, const int32_t* __restrict__ col,
+                      const float* __restrict__ val, int32_t* __restrict__ cursor,
+                      int32_t* __restrict__ tmp_row, float* __restrict__ tmp_val)
+{
+    const int lane = threadIdx.x & 31;
+    const int32_t r = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    if (r >= rows) return;
+    for (int32_t p = rowptr[r] + lane; p < rowptr[r + 1]; p += 32) {
+        const int32_t dst = atomicAdd(cursor + col[p], 1);
+        tmp_row[dst] = r;
+        tmp_val[dst] = val[p];
+    }
+}
+
+constexpr int BUCKET_SMEM = 1024;  // entries of one bucket staged per warp
+
+// One warp per bucket: each element's final position is the number of bucket entries with a smaller
+// source row (rows are distinct).  Buckets longer than the staging area are ranked from global memory.
+__global__ void __launch_bounds__(128)
+bucket_order_kernel(int32_t cols, const int32_t* __restrict__ t_rowptr,
+                    const int32_t* __restrict__ tmp_row, const float* __restrict__ tmp_val,
+                    int32_t* __restrict__ t_col, float* __restrict__ t_val)
+{
+    __shared__ int32_t staged[4][BUCKET_SMEM];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int32_t c = blockIdx.x * 4 + warp;
+    if (c >= cols) return;
+    const int32_t beg = t_rowptr[c], len = t_rowptr[c + 1] - beg;
+    const bool in_smem = len <= BUCKET_SMEM;
+    if (in_smem)
+        for (int32_t x = lane; x < len; x += 32) staged[warp][x] = tmp_row[beg + x];
+    __syncwarp();
+    for (int32_t x = lane; x < len; x += 32) {
+        const int32_t mine = in_smem ? staged[warp][x] : tmp_row[beg + x];
+        int32_t rank = 0;
+        if (in_smem) {
+            for (int32_t y = 0; y < len; ++y) rank += staged[warp][y] < mine;
+        } else {
+            for (int32_t y = 0; y < len; ++y) rank += tmp_row[beg + y] < mine;
+        }
+        t_col[beg + rank] = mine;
+        t_val[beg + rank] = tmp_val[beg + x];
+    }
+}
+
+__global__ void copy_i32_kernel(const int32_t* __restrict__ src, int32_t* __restrict__ dst, int32_t n)
+{
+    const int32_t i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < n) dst[i] = src[i];
+}
+
+}  // namespace
+
+int grf_transpose_launch(grf_ctx* ctx, int32_t rows, int32_t cols, int64_t nnz,
+                         const int32_t* rowptr, const int32_t* col, const float* val,
+                         int32_t* t_rowptr, int32_t* t_col, float* t_val)
+{
+    if (rows <= 0 || cols <= 0 || nnz < 0) return GRF_ERR_INVALID;
+    if (nnz >= (1ll << 31)) return GRF_ERR_TOO_LARGE;
+    // scratch: per-column counts, later the scatter cursors; and the unordered buckets
+    GRF_TRY(grf_buf_reserve(&ctx->t_cursor, sizeof(int32_t) * ((size_t)cols + 1)));
+    GRF_TRY(grf_buf_reserve(&ctx->t_tmp_col, sizeof(int32_t) * (size_t)(nnz > 0 ? nnz : 1)));
+    GRF_TRY(grf_buf_reserve(&ctx->t_tmp_val, sizeof(float) * (size_t)(nnz > 0 ? nnz : 1)));
+    int32_t* cursor = (int32_t*)ctx->t_cursor.ptr;
+    GRF_CUDA_TRY(cudaMemsetAsync(cursor, 0, sizeof(int32_t) * ((size_t)cols + 1), ctx->stream));
+    if (nnz > 0) {
+        int blocks = grf_ceil_div(nnz, 256);
+        if (blocks > 148 * 16) blocks = 148 * 16;
+        column_histogram_kernel<<<blocks, 256, 0, ctx->stream>>>(nnz, col, cursor);
+        ctx->launches++;
+    }
+    GRF_TRY(grf_exclusive_scan(ctx, cursor, t_rowptr, cols, 1));
+    copy_i32_kernel<<<grf_ceil_div(cols, 256), 256, 0, ctx->stream>>>(t_rowptr, cursor, cols);
+    ctx->launches++;
+    if (nnz > 0) {
+        bucket_scatter_kernel<<<grf_ceil_div(rows, 8), 256, 0, ctx->stream>>>(
+            rows, rowptr, col, val, cursor, (int32_t*)ctx->t_tmp_col.ptr, (float*)ctx->t_tmp_val.ptr);
+        bucket_order_kernel<<<grf_ceil_div(cols, 4), 128, 0, ctx->stream>>>(
+            cols, t_rowptr, (const int32_t*)ctx->t_tmp_col.ptr, (const float*)ctx->t_tmp_val.ptr, t_col, t_val);
+        ctx->launches += 2;
+    }
+    GRF_CUDA_TRY(cudaGetLastError());
+    return GRF_OK;
+}
+
+extern "C" int grf_csr_transpose(grf_ctx* ctx, int32_t rows, int32_t cols, int64_t nnz,
+                                 const int32_t* rowptr, const int32_t* col, const float* val,
+                                 int32_t* t_rowptr, int32_t* t_col, float* t_val)
+{
+    if (!ctx || !rowptr || !t_rowptr) return GRF_ERR_INVALID;
+    if (nnz > 0 && (!col || !val || !t_col || !t_val)) return GRF_ERR_INVALID;
+    GRF_CUDA_TRY(cudaSetDevice(ctx->device));
+    return grf_transpose_launch(ctx, rows, cols, nnz, rowptr, col, val, t_rowptr, t_col, t_val);
+}
