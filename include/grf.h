@@ -94,6 +94,9 @@ int grf_features_from_csr(grf_ctx* ctx, int32_t N, int32_t R,
  * object is freed or resampled.  rows/cols/nnz are returned through HOST pointers (any may be NULL). */
 int grf_features_view(const grf_features* feat, int which, int32_t* rows, int32_t* cols, int64_t* nnz,
                       const int32_t** rowptr, const int32_t** col, const float** val);
+/* Copies one matrix of a feature object into caller DEVICE arrays rowptr[rows+1], col[nnz], val[nnz]
+ * (sizes as reported by grf_features_view).  Asynchronous. */
+int grf_features_copy(grf_ctx* ctx, const grf_features* feat, int which, int32_t* rowptr, int32_t* col, float* val);
 int grf_features_free(grf_features* feat);
 
 /* Regroups a DEVICE CSR matrix (rows x cols, nnz = rowptr[rows] passed by the caller) by column:

@@ -1,0 +1,285 @@
+// C-ABI entry points that are not kernels themselves: contexts, buffers, feature objects, the
+// attention driver (Alg. 1 step 5 in chunks of problems) and the host-buffer path.
+#include <cstring>
+#include <new>
+
+#include "grf_internal.cuh"
+
+int grf_buf_reserve(grf_buf* b, size_t bytes)
+{
+    if (bytes == 0) bytes = 1;
+    if (b->bytes >= bytes) return GRF_OK;
+    if (b->ptr) { cudaFree(b->ptr); b->ptr = nullptr; b->bytes = 0; }
+    void* p = nullptr;
+    const cudaError_t e = cudaMalloc(&p, bytes);
+    if (e != cudaSuccess) { cudaGetLastError(); return GRF_ERR_NOMEM; }
+    b->ptr = p; b->bytes = bytes;
+    return GRF_OK;
+}
+
+void grf_buf_release(grf_buf* b)
+{
+    if (b->ptr) cudaFree(b->ptr);
+    b->ptr = nullptr; b->bytes = 0;
+}
+
+int grf_csr_reserve(grf_csr_dev* m, int32_t rows, int32_t cols, int64_t nnz_cap)
+{
+    m->rows = rows; m->cols = cols;
+    GRF_TRY(grf_buf_reserve(&m->rowptr, sizeof(int32_t) * ((size_t)rows + 1)));
+    GRF_TRY(grf_buf_reserve(&m->col, sizeof(int32_t) * (size_t)(nnz_cap > 0 ? nnz_cap : 1)));
+    GRF_TRY(grf_buf_reserve(&m->val, sizeof(float) * (size_t)(nnz_cap > 0 ? nnz_cap : 1)));
+    return GRF_OK;
+}
+
+extern "C" int grf_ctx_create(grf_ctx** out, int device, void* cuda_stream)
+{
+    if (!out || device < 0) return GRF_ERR_INVALID;
+    int count = 0;
+    if (cudaGetDeviceCount(&count) != cudaSuccess || device >= count) { cudaGetLastError(); return GRF_ERR_CUDA; }
+    GRF_CUDA_TRY(cudaSetDevice(device));
+    grf_ctx* c = new (std::nothrow) grf_ctx();
+    if (!c) return GRF_ERR_NOMEM;
+    c->device = device;
+    c->stream = (cudaStream_t)cuda_stream;
+    if (cudaDeviceGetAttribute(&c->sm_count, cudaDevAttrMultiProcessorCount, device) != cudaSuccess ||
+        cudaMallocHost((void**)&c->pinned, 64) != cudaSuccess) {
+        cudaGetLastError();
+        delete c;
+        return GRF_ERR_CUDA;
+    }
+    *out = c;
+    return GRF_OK;
+}
+
+extern "C" int grf_ctx_destroy(grf_ctx* ctx)
+{
+    if (!ctx) return GRF_ERR_INVALID;
+    cudaSetDevice(ctx->device);
+    cudaStreamSynchronize(ctx->stream);
+    grf_buf* bufs[] = {&ctx->stage_col, &ctx->stage_val, &ctx->counts, &ctx->rowptr2, &ctx->scan_blocks,
+                       &ctx->t_cursor, &ctx->t_tmp_col, &ctx->t_tmp_val, &ctx->h_rowptr, &ctx->h_col, &ctx->h_w,
+                       &ctx->h_q, &ctx->h_k, &ctx->h_v, &ctx->h_out, &ctx->h_ws};
+    for (grf_buf* b : bufs) grf_buf_release(b);
+    if (ctx->h_feat) grf_features_free(ctx->h_feat);
+    if (ctx->pinned) cudaFreeHost(ctx->pinned);
+    delete ctx;
+    return GRF_OK;
+}
+
+extern "C" int64_t grf_ctx_launch_count(const grf_ctx* ctx) { return ctx ? ctx->launches : -1; }
+
+extern "C" int grf_deconvolve(const double* alpha, int32_t len, double* f_out)
+{
+    if (!alpha || !f_out || len < 1 || !(alpha[0] > 0.0)) return GRF_ERR_INVALID;
+    // sum_{p=0..k} f_p f_{k-p} = alpha_k  =>  f_0 = sqrt(alpha_0), then solve for f_k (Remark 3.1)
+    f_out[0] = sqrt(alpha[0]);
+    for (int32_t k = 1; k < len; ++k) {
+        double cross = 0.0;
+        for (int32_t p = 1; p < k; ++p) cross += f_out[p] * f_out[k - p];
+        f_out[k] = (alpha[k] - cross) / (2.0 * f_out[0]);
+    }
+    return GRF_OK;
+}
+
+static void csr_release(grf_csr_dev* m)
+{
+    grf_buf_release(&m->rowptr); grf_buf_release(&m->col); grf_buf_release(&m->val);
+}
+
+extern "C" int grf_features_free(grf_features* feat)
+{
+    if (!feat) return GRF_ERR_INVALID;
+    cudaSetDevice(feat->device);
+    csr_release(&feat->phi); csr_release(&feat->psi); csr_release(&feat->psit);
+    delete feat;
+    return GRF_OK;
+}
+
+extern "C" int grf_features_view(const grf_features* feat, int which, int32_t* rows, int32_t* cols, int64_t* nnz,
+                                 const int32_t** rowptr, const int32_t** col, const float** val)
+{
+    if (!feat || which < 0 || which > 2) return GRF_ERR_INVALID;
+    const grf_csr_dev& m = which == 0 ? feat->phi : (which == 1 ? feat->psi : feat->psit);
+    if (rows) *rows = m.rows;
+    if (cols) *cols = m.cols;
+    if (nnz) *nnz = m.nnz;
+    if (rowptr) *rowptr = (const int32_t*)m.rowptr.ptr;
+    if (col) *col = (const int32_t*)m.col.ptr;
+    if (val) *val = (const float*)m.val.ptr;
+    return GRF_OK;
+}
+
+extern "C" int grf_features_copy(grf_ctx* ctx, const grf_features* feat, int which, int32_t* rowptr, int32_t* col,
+                                 float* val)
+{
+    if (!ctx || !feat || which < 0 || which > 2 || !rowptr) return GRF_ERR_INVALID;
+    const grf_csr_dev& m = which == 0 ? feat->phi : (which == 1 ? feat->psi : feat->psit);
+    if (m.nnz > 0 && (!col || !val)) return GRF_ERR_INVALID;
+    GRF_CUDA_TRY(cudaSetDevice(ctx->device));
+    GRF_CUDA_TRY(cudaMemcpyAsync(rowptr, m.rowptr.ptr, sizeof(int32_t) * ((size_t)m.rows + 1), cudaMemcpyDeviceToDevice,
+                                 ctx->stream));
+    if (m.nnz > 0) {
+        GRF_CUDA_TRY(cudaMemcpyAsync(col, m.col.ptr, sizeof(int32_t) * (size_t)m.nnz, cudaMemcpyDeviceToDevice, ctx->stream));
+        GRF_CUDA_TRY(cudaMemcpyAsync(val, m.val.ptr, sizeof(float) * (size_t)m.nnz, cudaMemcpyDeviceToDevice, ctx->stream));
+    }
+    return GRF_OK;
+}
+
+extern "C" int grf_features_from_csr(grf_ctx* ctx, int32_t N, int32_t R,
+                                     const int32_t* phi_rowptr, const int32_t* phi_col, const float* phi_val,
+                                     const int32_t* psi_rowptr, const int32_t* psi_col, const float* psi_val,
+                                     grf_features** out)
+{
+    if (!ctx || !out || N <= 0 || R <= 0 || !phi_rowptr || !psi_rowptr) return GRF_ERR_INVALID;
+    GRF_CUDA_TRY(cudaSetDevice(ctx->device));
+    GRF_CUDA_TRY(cudaMemcpyAsync(ctx->pinned + 0, phi_rowptr + N, sizeof(int32_t), cudaMemcpyDeviceToHost, ctx->stream));
+    GRF_CUDA_TRY(cudaMemcpyAsync(ctx->pinned + 1, psi_rowptr + N, sizeof(int32_t), cudaMemcpyDeviceToHost, ctx->stream));
+    GRF_CUDA_TRY(cudaStreamSynchronize(ctx->stream));
+    const int64_t nnz_phi = ctx->pinned[0], nnz_psi = ctx->pinned[1];
+    if (nnz_phi < 0 || nnz_psi < 0) return GRF_ERR_INVALID;
+    if ((nnz_phi > 0 && (!phi_col || !phi_val)) || (nnz_psi > 0 && (!psi_col || !psi_val))) return GRF_ERR_INVALID;
+    grf_features* f = new (std::nothrow) grf_features();
+    if (!f) return GRF_ERR_NOMEM;
+    f->device = ctx->device;
+    int rc = grf_csr_reserve(&f->phi, N, R, nnz_phi);
+    if (rc == GRF_OK) rc = grf_csr_reserve(&f->psi, N, R, nnz_psi);
+    if (rc == GRF_OK) rc = grf_csr_reserve(&f->psit, R, N, nnz_psi);
+    if (rc != GRF_OK) { grf_features_free(f); return rc; }
+    f->phi.nnz = nnz_phi; f->psi.nnz = nnz_psi; f->psit.nnz = nnz_psi;
+    auto copy = [&](grf_csr_dev& m, const int32_t* rp, const int32_t* c, const float* v, int64_t nnz) {
+        cudaMemcpyAsync(m.rowptr.ptr, rp, sizeof(int32_t) * ((size_t)N + 1), cudaMemcpyDeviceToDevice, ctx->stream);
+        if (nnz > 0) {
+            cudaMemcpyAsync(m.col.ptr, c, sizeof(int32_t) * (size_t)nnz, cudaMemcpyDeviceToDevice, ctx->stream);
+            cudaMemcpyAsync(m.val.ptr, v, sizeof(float) * (size_t)nnz, cudaMemcpyDeviceToDevice, ctx->stream);
+        }
+    };
+    copy(f->phi, phi_rowptr, phi_col, phi_val, nnz_phi);
+    copy(f->psi, psi_rowptr, psi_col, psi_val, nnz_psi);
+    rc = grf_transpose_launch(ctx, N, R, nnz_psi, (const int32_t*)f->psi.rowptr.ptr, (const int32_t*)f->psi.col.ptr,
+                              (const float*)f->psi.val.ptr, (int32_t*)f->psit.rowptr.ptr,
+                              (int32_t*)f->psit.col.ptr, (float*)f->psit.val.ptr);
+    if (rc == GRF_OK && cudaGetLastError() != cudaSuccess) rc = GRF_ERR_CUDA;
+    if (rc != GRF_OK) { grf_features_free(f); return rc; }
+    *out = f;
+    return GRF_OK;
+}
+
+static bool dim_ok(int32_t x) { return x == 8 || x == 16 || x == 32 || x == 64 || x == 128; }
+static size_t elem_size(int dtype) { return dtype == GRF_DTYPE_F32 ? 4 : 2; }
+static size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
+
+// per-problem workspace: S [R][m][d] in the storage type, then z [R][m] fp32, each 256-byte aligned
+static size_t ws_per_problem(int32_t R, int32_t m, int32_t d, int dtype)
+{
+    return align256((size_t)R * m * d * elem_size(dtype)) + align256((size_t)R * m * sizeof(float));
+}
+
+extern "C" size_t grf_attn_workspace_bytes(int32_t G, int32_t R, int32_t m, int32_t d, int dtype)
+{
+    if (G <= 0 || R <= 0 || !dim_ok(m) || !dim_ok(d) || (dtype != GRF_DTYPE_F32 && dtype != GRF_DTYPE_BF16)) return 0;
+    return ws_per_problem(R, m, d, dtype) * (size_t)G;
+}
+
+extern "C" int grf_masked_linear_attn(grf_ctx* ctx, const grf_features* feat, int32_t G, int32_t N, int32_t m,
+                                      int32_t d, int dtype, const void* phiQ, const void* phiK, const void* V,
+                                      void* out, float* den_out, void* workspace, size_t workspace_bytes)
+{
+    if (!ctx || !feat || !phiQ || !phiK || !V || !out || !workspace) return GRF_ERR_INVALID;
+    if (G <= 0 || N <= 0 || !dim_ok(m) || !dim_ok(d)) return GRF_ERR_INVALID;
+    if (dtype != GRF_DTYPE_F32 && dtype != GRF_DTYPE_BF16) return GRF_ERR_INVALID;
+    if (feat->phi.rows != N || feat->psit.cols != N || feat->phi.cols != feat->psit.rows) return GRF_ERR_INVALID;
+    if (((uintptr_t)workspace & 255) != 0) return GRF_ERR_INVALID;
+    const int32_t R = feat->phi.cols;
+    const size_t per = ws_per_problem(R, m, d, dtype);
+    if (workspace_bytes < per) return GRF_ERR_WORKSPACE;
+    GRF_CUDA_TRY(cudaSetDevice(ctx->device));
+    int64_t chunk = (int64_t)(workspace_bytes / per);
+    if (chunk > G) chunk = G;
+    if (chunk > 65535) chunk = 65535;
+    const size_t es = elem_size(dtype);
+    const size_t s_bytes = align256((size_t)R * m * d * es);
+    for (int64_t g0 = 0; g0 < G; g0 += chunk) {
+        const int32_t gc = (int32_t)((G - g0) < chunk ? (G - g0) : chunk);
+        // chunk layout: S for gc problems (contiguous, [gc][R][m][d]) then z ([gc][R][m])
+        char* Sbuf = (char*)workspace;
+        float* zbuf = (float*)((char*)workspace + align256((size_t)gc * R * m * d * es));
+        (void)s_bytes;
+        const char* k_ptr = (const char*)phiK + (size_t)g0 * N * m * es;
+        const char* v_ptr = (const char*)V + (size_t)g0 * N * d * es;
+        const char* q_ptr = (const char*)phiQ + (size_t)g0 * N * m * es;
+        char* o_ptr = (char*)out + (size_t)g0 * N * d * es;
+        float* den_ptr = den_out ? den_out + (size_t)g0 * N : nullptr;
+        GRF_TRY(grf_build_states(ctx, feat->psit, gc, N, m, d, dtype, k_ptr, v_ptr, Sbuf, zbuf));
+        GRF_TRY(grf_gather_contract(ctx, feat->phi, gc, N, m, d, dtype, q_ptr, Sbuf, zbuf, o_ptr, den_ptr));
+    }
+    return GRF_OK;
+}
+
+static int check_graph_host(int32_t N, const int32_t* rowptr, const int32_t* col)
+{
+    if (rowptr[0] != 0) return GRF_ERR_BADGRAPH;
+    for (int32_t i = 0; i < N; ++i)
+        if (rowptr[i + 1] < rowptr[i]) return GRF_ERR_BADGRAPH;
+    const int64_t E = rowptr[N];
+    for (int64_t p = 0; p < E; ++p)
+        if (col[p] < 0 || col[p] >= N) return GRF_ERR_BADGRAPH;
+    return GRF_OK;
+}
+
+extern "C" int grf_step_host(grf_ctx* ctx, int32_t N, const int32_t* rowptr, const int32_t* col, const float* w,
+                             uint64_t seed, int32_t n_walks, float p_halt, int32_t max_len,
+                             const float* f_phi, const float* f_psi,
+                             int32_t G, int32_t m, int32_t d, int dtype,
+                             const void* phiQ, const void* phiK, const void* V, void* out)
+{
+    if (!ctx || !rowptr || !col || !w || !phiQ || !phiK || !V || !out || N <= 0 || G <= 0) return GRF_ERR_INVALID;
+    if (!dim_ok(m) || !dim_ok(d) || (dtype != GRF_DTYPE_F32 && dtype != GRF_DTYPE_BF16)) return GRF_ERR_INVALID;
+    GRF_TRY(check_graph_host(N, rowptr, col));
+    GRF_CUDA_TRY(cudaSetDevice(ctx->device));
+    const size_t E = (size_t)rowptr[N], es = elem_size(dtype);
+    const size_t qk_bytes = (size_t)G * N * m * es, v_bytes = (size_t)G * N * d * es;
+    GRF_TRY(grf_buf_reserve(&ctx->h_rowptr, ((size_t)N + 1) * 4));
+    GRF_TRY(grf_buf_reserve(&ctx->h_col, E * 4));
+    GRF_TRY(grf_buf_reserve(&ctx->h_w, E * 4));
+    GRF_TRY(grf_buf_reserve(&ctx->h_q, qk_bytes));
+    GRF_TRY(grf_buf_reserve(&ctx->h_k, qk_bytes));
+    GRF_TRY(grf_buf_reserve(&ctx->h_v, v_bytes));
+    GRF_TRY(grf_buf_reserve(&ctx->h_out, v_bytes));
+    cudaStream_t s = ctx->stream;
+    GRF_CUDA_TRY(cudaMemcpyAsync(ctx->h_rowptr.ptr, rowptr, ((size_t)N + 1) * 4, cudaMemcpyHostToDevice, s));
+    if (E > 0) {
+        GRF_CUDA_TRY(cudaMemcpyAsync(ctx->h_col.ptr, col, E * 4, cudaMemcpyHostToDevice, s));
+        GRF_CUDA_TRY(cudaMemcpyAsync(ctx->h_w.ptr, w, E * 4, cudaMemcpyHostToDevice, s));
+    }
+    GRF_CUDA_TRY(cudaMemcpyAsync(ctx->h_q.ptr, phiQ, qk_bytes, cudaMemcpyHostToDevice, s));
+    GRF_CUDA_TRY(cudaMemcpyAsync(ctx->h_k.ptr, phiK, qk_bytes, cudaMemcpyHostToDevice, s));
+    GRF_CUDA_TRY(cudaMemcpyAsync(ctx->h_v.ptr, V, v_bytes, cudaMemcpyHostToDevice, s));
+    GRF_TRY(grf_sample(ctx, N, (const int32_t*)ctx->h_rowptr.ptr, (const int32_t*)ctx->h_col.ptr,
+                       (const float*)ctx->h_w.ptr, seed, n_walks, p_halt, max_len, f_phi, f_psi, &ctx->h_feat));
+    // workspace: everything if it is modest, else chunks of about 1 GiB
+    const size_t per = ws_per_problem(N, m, d, dtype);
+    size_t want = per * (size_t)G;
+    const size_t cap = (size_t)1 << 31;
+    if (want > cap) want = per * (cap / per > 0 ? cap / per : 1);
+    GRF_TRY(grf_buf_reserve(&ctx->h_ws, want));
+    GRF_TRY(grf_masked_linear_attn(ctx, ctx->h_feat, G, N, m, d, dtype, ctx->h_q.ptr, ctx->h_k.ptr, ctx->h_v.ptr,
+                                   ctx->h_out.ptr, nullptr, ctx->h_ws.ptr, ctx->h_ws.bytes));
+    GRF_CUDA_TRY(cudaMemcpyAsync(out, ctx->h_out.ptr, v_bytes, cudaMemcpyDeviceToHost, s));
+    GRF_CUDA_TRY(cudaStreamSynchronize(s));
+    return GRF_OK;
+}
+
+extern "C" const char* grf_strerror(int code)
+{
+    switch (code) {
+        case GRF_OK: return "ok";
+        case GRF_ERR_INVALID: return "invalid argument";
+        case GRF_ERR_TOO_LARGE: return "size exceeds a documented limit";
+        case GRF_ERR_WORKSPACE: return "workspace too small";
+        case GRF_ERR_CUDA: return "CUDA runtime error";
+        case GRF_ERR_NOMEM: return "out of memory";
+        case GRF_ERR_BADGRAPH: return "inconsistent graph CSR";
+        default: return "unknown error";
+    }
+}

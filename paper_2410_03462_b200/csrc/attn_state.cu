@@ -1,0 +1,145 @@
+// Per-node states of Alg. 1 step 5 (Eq. 12):  S_l = sum_j Psi_jl phi(k_j) v_j^T  (m x d),
+// z_l = sum_j Psi_jl phi(k_j)  (m), for every problem g and node l — the rows of Phi_K^T V and
+// Phi_K^T 1 of Corollary 3.4.  A segmented reduction over the column-grouped Psi^T with a fixed
+// summation order (ascending j), fp32 accumulation, no atomics.
+#include "grf_internal.cuh"
+
+namespace {
+
+template <typename T> __device__ __forceinline__ float to_f32(T x);
+template <> __device__ __forceinline__ float to_f32<float>(float x) { return x; }
+template <> __device__ __forceinline__ float to_f32<__nv_bfloat16>(__nv_bfloat16 x) { return __bfloat162float(x); }
+
+__device__ __forceinline__ void store4(float* dst, const float (&v)[4])
+{
+    *reinterpret_cast<float4*>(dst) = make_float4(v[0], v[1], v[2], v[3]);
+}
+__device__ __forceinline__ void store4(__nv_bfloat16* dst, const float (&v)[4])
+{
+    __nv_bfloat162 lo = __floats2bfloat162_rn(v[0], v[1]);
+    __nv_bfloat162 hi = __floats2bfloat162_rn(v[2], v[3]);
+    uint2 u;
+    u.x = *reinterpret_cast<uint32_t*>(&lo);
+    u.y = *reinterpret_cast<uint32_t*>(&hi);
+    *reinterpret_cast<uint2*>(dst) = u;
+}
+
+template <int M, int D>
+struct StateTiling {
+    static constexpr int TX = D / 4;                              // threads across a row of the tile
+    static constexpr int THREADS = (TX * M < 128) ? TX * M : 128;
+    static constexpr int TY = THREADS / TX;
+    static constexpr int TA = M / TY;                             // tile rows per thread
+    static constexpr int JC = 8;                                  // source rows staged per step
+};
+
+// One CTA per (node l, problem g).  Each thread keeps a TA x 4 block of the m x d tile in registers.
+template <typename T, int M, int D>
+__global__ void __launch_bounds__(StateTiling<M, D>::THREADS)
+build_states_kernel(int32_t R, int32_t N, const int32_t* __restrict__ t_rowptr, const int32_t* __restrict__ t_col,
+                    const float* __restrict__ t_val, const T* __restrict__ phiK, const T* __restrict__ V,
+                    T* __restrict__ S, float* __restrict__ z)
+{
+    using Tl = StateTiling<M, D>;
+    constexpr int TX = Tl::TX, TY = Tl::TY, TA = Tl::TA, JC = Tl::JC, THREADS = Tl::THREADS;
+    __shared__ __align__(16) float ks[JC][M];
+    __shared__ __align__(16) float vs[JC][D];
+
+    const int32_t l = blockIdx.x, g = blockIdx.y;
+    const int tid = threadIdx.x, tx = tid % TX, ty = tid / TX;
+    const T* Kg = phiK + (size_t)g * N * M;
+    const T* Vg = V + (size_t)g * N * D;
+
+    float acc[TA][4];
+    float zacc[TA];
+#pragma unroll
+    for (int r = 0; r < TA; ++r) {
+        zacc[r] = 0.0f;
+#pragma unroll
+        for (int c = 0; c < 4; ++c) acc[r][c] = 0.0f;
+    }
+
+    const int32_t beg = t_rowptr[l], end = t_rowptr[l + 1];
+    for (int32_t p0 = beg; p0 < end; p0 += JC) {
+        const int32_t nj = min(JC, end - p0);
+        for (int idx = tid; idx < JC * M; idx += THREADS) {
+            const int jj = idx / M, a = idx % M;
+            float x = 0.0f;
+            if (jj < nj) x = t_val[p0 + jj] * to_f32(Kg[(size_t)t_col[p0 + jj] * M + a]);
+            ks[jj][a] = x;
+        }
+        for (int idx = tid; idx < JC * D; idx += THREADS) {
+            const int jj = idx / D, b = idx % D;
+            vs[jj][b] = jj < nj ? to_f32(Vg[(size_t)t_col[p0 + jj] * D + b]) : 0.0f;
+        }
+        __syncthreads();
+#pragma unroll
+        for (int jj = 0; jj < JC; ++jj) {
+            const float4 v4 = *reinterpret_cast<const float4*>(&vs[jj][tx * 4]);
+#pragma unroll
+            for (int r = 0; r < TA; ++r) {
+                const float kr = ks[jj][ty + r * TY];
+                acc[r][0] = fmaf(kr, v4.x, acc[r][0]);
+                acc[r][1] = fmaf(kr, v4.y, acc[r][1]);
+                acc[r][2] = fmaf(kr, v4.z, acc[r][2]);
+                acc[r][3] = fmaf(kr, v4.w, acc[r][3]);
+                zacc[r] += kr;
+            }
+        }
+        __syncthreads();
+    }
+
+    T* Sl = S + ((size_t)g * R + l) * M * D;
+#pragma unroll
+    for (int r = 0; r < TA; ++r) store4(Sl + (size_t)(ty + r * TY) * D + tx * 4, acc[r]);
+    if (tx == 0) {
+        float* zl = z + ((size_t)g * R + l) * M;
+#pragma unroll
+        for (int r = 0; r < TA; ++r) zl[ty + r * TY] = zacc[r];
+    }
+}
+
+template <typename T, int M>
+int launch_m(grf_ctx* ctx, const grf_csr_dev& psit, int32_t G, int32_t N, int32_t d,
+             const void* phiK, const void* V, void* S, float* z)
+{
+    const dim3 grid(psit.rows, G);
+#define GRF_STATE_CASE(DD)                                                                                  \
+    case DD:                                                                                                \
+        build_states_kernel<T, M, DD><<<grid, StateTiling<M, DD>::THREADS, 0, ctx->stream>>>(               \
+            psit.rows, N, (const int32_t*)psit.rowptr.ptr, (const int32_t*)psit.col.ptr,                    \
+            (const float*)psit.val.ptr, (const T*)phiK, (const T*)V, (T*)S, z);                            \
+        break;
+    switch (d) {
+        GRF_STATE_CASE(8) GRF_STATE_CASE(16) GRF_STATE_CASE(32) GRF_STATE_CASE(64) GRF_STATE_CASE(128)
+        default: return GRF_ERR_INVALID;
+    }
+#undef GRF_STATE_CASE
+    ctx->launches++;
+    return cudaGetLastError() == cudaSuccess ? GRF_OK : GRF_ERR_CUDA;
+}
+
+template <typename T>
+int launch_t(grf_ctx* ctx, const grf_csr_dev& psit, int32_t G, int32_t N, int32_t m, int32_t d,
+             const void* phiK, const void* V, void* S, float* z)
+{
+    switch (m) {
+        case 8: return launch_m<T, 8>(ctx, psit, G, N, d, phiK, V, S, z);
+        case 16: return launch_m<T, 16>(ctx, psit, G, N, d, phiK, V, S, z);
+        case 32: return launch_m<T, 32>(ctx, psit, G, N, d, phiK, V, S, z);
+        case 64: return launch_m<T, 64>(ctx, psit, G, N, d, phiK, V, S, z);
+        case 128: return launch_m<T, 128>(ctx, psit, G, N, d, phiK, V, S, z);
+        default: return GRF_ERR_INVALID;
+    }
+}
+
+}  // namespace
+
+int grf_build_states(grf_ctx* ctx, const grf_csr_dev& psit, int32_t G, int32_t N, int32_t m, int32_t d, int dtype,
+                     const void* phiK, const void* V, void* S, float* z)
+{
+    if (G > 65535) return GRF_ERR_TOO_LARGE;
+    if (dtype == GRF_DTYPE_F32) return launch_t<float>(ctx, psit, G, N, m, d, phiK, V, S, z);
+    if (dtype == GRF_DTYPE_BF16) return launch_t<__nv_bfloat16>(ctx, psit, G, N, m, d, phiK, V, S, z);
+    return GRF_ERR_INVALID;
+}
