@@ -141,6 +141,15 @@ int grf_step_host(grf_ctx* ctx, int32_t N, const int32_t* rowptr, const int32_t*
 /* Number of kernels the context has launched since it was created (for accounting in benchmarks). */
 int64_t grf_ctx_launch_count(const grf_ctx* ctx);
 
+/* Per-kernel device timing for benchmarks.  While enabled, every kernel launch of the context is
+ * bracketed by two CUDA events on the context's stream.  grf_ctx_kernel_times waits for the stream, adds
+ * the elapsed times since the previous read to ms[GRF_KERNEL_CLASSES] / launches[GRF_KERNEL_CLASSES]
+ * (HOST arrays, overwritten) and clears the record.  Classes: 0 walk+merge, 1 prefix scans, 2 row
+ * compaction, 3 column regrouping (histogram, scatter, ordering), 4 state build (S, z), 5 gather-contract. */
+#define GRF_KERNEL_CLASSES 6
+int grf_ctx_enable_timing(grf_ctx* ctx, int enable);
+int grf_ctx_kernel_times(grf_ctx* ctx, float* ms, int64_t* launches);
+
 const char* grf_strerror(int code);
 
 #ifdef __cplusplus

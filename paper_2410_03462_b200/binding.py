@@ -41,6 +41,8 @@ _SIGNATURES = {
     "grf_step_host": (_int, [_vp, _i32, _vp, _vp, _vp, _u64, _i32, _f32, _i32, _vp, _vp,
                              _i32, _i32, _i32, _int, _vp, _vp, _vp, _vp]),
     "grf_ctx_launch_count": (_i64, [_vp]),
+    "grf_ctx_enable_timing": (_int, [_vp, _int]),
+    "grf_ctx_kernel_times": (_int, [_vp, _vp, _vp]),
     "grf_strerror": (ctypes.c_char_p, [_int]),
 }
 for _name, (_res, _args) in _SIGNATURES.items():
@@ -101,6 +103,21 @@ def grf_ctx_destroy(ctx: int):
 
 def grf_ctx_launch_count(ctx: int) -> int:
     return int(lib.grf_ctx_launch_count(ctx))
+
+
+KERNEL_CLASSES = ("walk_merge", "scan", "compact", "regroup", "build_states", "gather_contract")
+
+
+def grf_ctx_enable_timing(ctx: int, enable: bool):
+    _check(lib.grf_ctx_enable_timing(ctx, int(enable)), "grf_ctx_enable_timing")
+
+
+def grf_ctx_kernel_times(ctx: int):
+    """{class name: (milliseconds, timed launch groups)} since the previous read."""
+    ms = np.zeros(len(KERNEL_CLASSES), dtype=np.float32)
+    n = np.zeros(len(KERNEL_CLASSES), dtype=np.int64)
+    _check(lib.grf_ctx_kernel_times(ctx, ms.ctypes.data, n.ctypes.data), "grf_ctx_kernel_times")
+    return {k: (float(ms[i]), int(n[i])) for i, k in enumerate(KERNEL_CLASSES)}
 
 
 def grf_deconvolve(alpha) -> np.ndarray:

@@ -63,7 +63,56 @@ extern "C" int grf_ctx_destroy(grf_ctx* ctx)
     for (grf_buf* b : bufs) grf_buf_release(b);
     if (ctx->h_feat) grf_features_free(ctx->h_feat);
     if (ctx->pinned) cudaFreeHost(ctx->pinned);
+    for (auto& t : ctx->timed) { cudaEventDestroy(t.beg); cudaEventDestroy(t.end); }
+    for (cudaEvent_t e : ctx->free_events) cudaEventDestroy(e);
     delete ctx;
+    return GRF_OK;
+}
+
+static cudaEvent_t take_event(grf_ctx* c)
+{
+    if (!c->free_events.empty()) { cudaEvent_t e = c->free_events.back(); c->free_events.pop_back(); return e; }
+    cudaEvent_t e = nullptr;
+    if (cudaEventCreate(&e) != cudaSuccess) { cudaGetLastError(); return nullptr; }
+    return e;
+}
+
+grf_launch_scope::grf_launch_scope(grf_ctx* c, int cls_, int n_launches) : ctx(c), cls(cls_), n(n_launches)
+{
+    if (!ctx->timing) return;
+    beg = take_event(ctx); end = take_event(ctx);
+    if (beg && end) cudaEventRecord(beg, ctx->stream);
+}
+
+grf_launch_scope::~grf_launch_scope()
+{
+    ctx->launches += n;
+    if (!ctx->timing || !beg || !end) return;
+    cudaEventRecord(end, ctx->stream);
+    ctx->timed.push_back({cls, beg, end});
+}
+
+extern "C" int grf_ctx_enable_timing(grf_ctx* ctx, int enable)
+{
+    if (!ctx) return GRF_ERR_INVALID;
+    ctx->timing = enable != 0;
+    return GRF_OK;
+}
+
+extern "C" int grf_ctx_kernel_times(grf_ctx* ctx, float* ms, int64_t* launches)
+{
+    if (!ctx || !ms || !launches) return GRF_ERR_INVALID;
+    GRF_CUDA_TRY(cudaSetDevice(ctx->device));
+    GRF_CUDA_TRY(cudaStreamSynchronize(ctx->stream));
+    for (int k = 0; k < GRF_KERNEL_CLASSES; ++k) { ms[k] = 0.0f; launches[k] = 0; }
+    for (auto& t : ctx->timed) {
+        float x = 0.0f;
+        if (cudaEventElapsedTime(&x, t.beg, t.end) == cudaSuccess) { ms[t.cls] += x; launches[t.cls] += 1; }
+        ctx->free_events.push_back(t.beg);
+        ctx->free_events.push_back(t.end);
+    }
+    ctx->timed.clear();
+    cudaGetLastError();
     return GRF_OK;
 }
 

@@ -131,12 +131,14 @@ int launch_m(grf_ctx* ctx, const grf_csr_dev& phi, int32_t G, int32_t N, int32_t
             N, phi.cols, (const int32_t*)phi.rowptr.ptr, (const int32_t*)phi.col.ptr,                        \
             (const float*)phi.val.ptr, (const T*)phiQ, (const T*)S, z, (T*)out, den_out);                   \
         break;
+    {
+    grf_launch_scope scope(ctx, 5);
     switch (d) {
         GRF_GATHER_CASE(8) GRF_GATHER_CASE(16) GRF_GATHER_CASE(32) GRF_GATHER_CASE(64) GRF_GATHER_CASE(128)
         default: return GRF_ERR_INVALID;
     }
+    }
 #undef GRF_GATHER_CASE
-    ctx->launches++;
     return cudaGetLastError() == cudaSuccess ? GRF_OK : GRF_ERR_CUDA;
 }
 

@@ -110,12 +110,14 @@ int launch_m(grf_ctx* ctx, const grf_csr_dev& psit, int32_t G, int32_t N, int32_
             psit.rows, N, (const int32_t*)psit.rowptr.ptr, (const int32_t*)psit.col.ptr,                    \
             (const float*)psit.val.ptr, (const T*)phiK, (const T*)V, (T*)S, z);                            \
         break;
+    {
+    grf_launch_scope scope(ctx, 4);
     switch (d) {
         GRF_STATE_CASE(8) GRF_STATE_CASE(16) GRF_STATE_CASE(32) GRF_STATE_CASE(64) GRF_STATE_CASE(128)
         default: return GRF_ERR_INVALID;
     }
+    }
 #undef GRF_STATE_CASE
-    ctx->launches++;
     return cudaGetLastError() == cudaSuccess ? GRF_OK : GRF_ERR_CUDA;
 }
 

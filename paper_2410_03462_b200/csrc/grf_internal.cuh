@@ -5,6 +5,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <vector>
+
 #include "grf.h"
 
 #define GRF_CUDA_TRY(expr)                                  \
@@ -41,6 +43,21 @@ struct grf_ctx {
     grf_buf h_rowptr, h_col, h_w, h_q, h_k, h_v, h_out, h_ws;
     grf_features* h_feat = nullptr;
     int32_t* pinned = nullptr;      // small pinned host block for read-backs
+    // optional per-launch timing
+    bool timing = false;
+    struct timed_launch { int cls; cudaEvent_t beg, end; };
+    std::vector<timed_launch> timed;
+    std::vector<cudaEvent_t> free_events;
+};
+
+// Brackets one kernel launch (or a short run of launches of one class) with events when timing is on.
+struct grf_launch_scope {
+    grf_ctx* ctx;
+    int cls;
+    int n;
+    cudaEvent_t beg = nullptr, end = nullptr;
+    grf_launch_scope(grf_ctx* c, int cls_, int n_launches = 1);
+    ~grf_launch_scope();
 };
 
 struct grf_csr_dev {

@@ -251,10 +251,12 @@ static int sample_into(grf_ctx* ctx, grf_features* feat, const grf_walk_params& 
     const size_t smem = per_warp * warps;
     static_assert(sizeof(grf_walk_params) <= 4096, "kernel parameter block too large");
     GRF_CUDA_TRY(cudaFuncSetAttribute(walk_merge_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    walk_merge_kernel<<<grf_ceil_div(rows2, warps), warps * 32, smem, ctx->stream>>>(
-        P, rowptr, col, w, stride, (int32_t*)ctx->stage_col.ptr, (float*)ctx->stage_val.ptr,
-        (int32_t*)ctx->counts.ptr);
-    ctx->launches++;
+    {
+        grf_launch_scope scope(ctx, 0);
+        walk_merge_kernel<<<grf_ceil_div(rows2, warps), warps * 32, smem, ctx->stream>>>(
+            P, rowptr, col, w, stride, (int32_t*)ctx->stage_col.ptr, (float*)ctx->stage_val.ptr,
+            (int32_t*)ctx->counts.ptr);
+    }
     GRF_CUDA_TRY(cudaGetLastError());
 
     // counts -> row pointers of Phi (segment 0) and Psi (segment 1)
@@ -279,12 +281,14 @@ static int sample_into(grf_ctx* ctx, grf_features* feat, const grf_walk_params& 
     feat->phi.nnz = nnz_phi; feat->psi.nnz = nnz_psi; feat->psit.nnz = nnz_psi;
     feat->psit.rows = N; feat->psit.cols = N;
 
-    compact_rows_kernel<<<grf_ceil_div(rows2, 8), 256, 0, ctx->stream>>>(
-        N, stride, (const int32_t*)ctx->stage_col.ptr, (const float*)ctx->stage_val.ptr,
-        (const int32_t*)feat->phi.rowptr.ptr, (const int32_t*)feat->psi.rowptr.ptr,
-        (int32_t*)feat->phi.col.ptr, (float*)feat->phi.val.ptr,
-        (int32_t*)feat->psi.col.ptr, (float*)feat->psi.val.ptr);
-    ctx->launches++;
+    {
+        grf_launch_scope scope(ctx, 2);
+        compact_rows_kernel<<<grf_ceil_div(rows2, 8), 256, 0, ctx->stream>>>(
+            N, stride, (const int32_t*)ctx->stage_col.ptr, (const float*)ctx->stage_val.ptr,
+            (const int32_t*)feat->phi.rowptr.ptr, (const int32_t*)feat->psi.rowptr.ptr,
+            (int32_t*)feat->phi.col.ptr, (float*)feat->phi.val.ptr,
+            (int32_t*)feat->psi.col.ptr, (float*)feat->psi.val.ptr);
+    }
     GRF_CUDA_TRY(cudaGetLastError());
 
     return grf_transpose_launch(ctx, N, N, nnz_psi, (const int32_t*)feat->psi.rowptr.ptr,
@@ -326,8 +330,10 @@ extern "C" int grf_debug_walks(grf_ctx* ctx, int32_t N, const int32_t* rowptr, c
     GRF_TRY(grf_walk_params_init(&P, N, seed, n_walks, p_halt, max_len, ones, ones));
     GRF_CUDA_TRY(cudaSetDevice(ctx->device));
     const int64_t total = 2ll * N * n_walks;
-    debug_walks_kernel<<<grf_ceil_div(total, 256), 256, 0, ctx->stream>>>(P, rowptr, col, w, traj, load);
-    ctx->launches++;
+    {
+        grf_launch_scope scope(ctx, 0);
+        debug_walks_kernel<<<grf_ceil_div(total, 256), 256, 0, ctx->stream>>>(P, rowptr, col, w, traj, load);
+    }
     GRF_CUDA_TRY(cudaGetLastError());
     return GRF_OK;
 }

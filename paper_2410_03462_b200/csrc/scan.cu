@@ -102,10 +102,12 @@ int grf_exclusive_scan(grf_ctx* ctx, const int32_t* in, int32_t* out, int32_t n,
     GRF_TRY(grf_buf_reserve(&ctx->scan_blocks, sizeof(int32_t) * (size_t)nblocks * segments));
     int32_t* totals = (int32_t*)ctx->scan_blocks.ptr;
     const dim3 grid(nblocks, segments);
-    scan_block_totals_kernel<<<grid, SCAN_THREADS, 0, ctx->stream>>>(in, n, totals);
-    scan_totals_kernel<<<segments, SCAN_THREADS, 0, ctx->stream>>>(totals, nblocks);
-    scan_write_kernel<<<grid, SCAN_THREADS, 0, ctx->stream>>>(in, n, totals, out);
-    ctx->launches += 3;
+    {
+        grf_launch_scope scope(ctx, 1, 3);
+        scan_block_totals_kernel<<<grid, SCAN_THREADS, 0, ctx->stream>>>(in, n, totals);
+        scan_totals_kernel<<<segments, SCAN_THREADS, 0, ctx->stream>>>(totals, nblocks);
+        scan_write_kernel<<<grid, SCAN_THREADS, 0, ctx->stream>>>(in, n, totals, out);
+    }
     GRF_CUDA_TRY(cudaGetLastError());
     return GRF_OK;
 }

@@ -84,18 +84,20 @@ int grf_transpose_launch(grf_ctx* ctx, int32_t rows, int32_t cols, int64_t nnz,
     if (nnz > 0) {
         int blocks = grf_ceil_div(nnz, 256);
         if (blocks > 148 * 16) blocks = 148 * 16;
+        grf_launch_scope scope(ctx, 3);
         column_histogram_kernel<<<blocks, 256, 0, ctx->stream>>>(nnz, col, cursor);
-        ctx->launches++;
     }
     GRF_TRY(grf_exclusive_scan(ctx, cursor, t_rowptr, cols, 1));
-    copy_i32_kernel<<<grf_ceil_div(cols, 256), 256, 0, ctx->stream>>>(t_rowptr, cursor, cols);
-    ctx->launches++;
+    {
+        grf_launch_scope scope(ctx, 3);
+        copy_i32_kernel<<<grf_ceil_div(cols, 256), 256, 0, ctx->stream>>>(t_rowptr, cursor, cols);
+    }
     if (nnz > 0) {
+        grf_launch_scope scope(ctx, 3, 2);
         bucket_scatter_kernel<<<grf_ceil_div(rows, 8), 256, 0, ctx->stream>>>(
             rows, rowptr, col, val, cursor, (int32_t*)ctx->t_tmp_col.ptr, (float*)ctx->t_tmp_val.ptr);
         bucket_order_kernel<<<grf_ceil_div(cols, 4), 128, 0, ctx->stream>>>(
             cols, t_rowptr, (const int32_t*)ctx->t_tmp_col.ptr, (const float*)ctx->t_tmp_val.ptr, t_col, t_val);
-        ctx->launches += 2;
     }
     GRF_CUDA_TRY(cudaGetLastError());
     return GRF_OK;

@@ -1,0 +1,55 @@
+"""Shared test helpers: oracle-side preparation of a workload and the comparison rules.
+
+Tolerance rule for attention outputs (stated by the workloads' accuracy target: 1e-5 for fp32, 2e-2 for
+bf16 storage, "relative"): with out = num/den, num and den sums of signed terms, an implementation whose
+sums are each accurate to tol relative to the sum of the ABSOLUTE values of its terms satisfies
+    |out' - out| <= tol * (num_abs + |out| * den_abs) / |den|
+to first order.  For same-sign terms this is the plain relative error of den and the error of num on the
+scale of its terms.  Rows whose denominator cancels almost completely (|den| < 1e-3 den_abs) are excluded
+from the out comparison and checked through den alone."""
+from __future__ import annotations
+
+import numpy as np
+
+import oracle
+from workloads import tensors
+
+TOL = {"fp32": 1e-5, "bf16": 2e-2}
+
+
+def oracle_features(w, g, seed, f_phi=None, f_psi=None):
+    if f_phi is None:
+        f_phi = oracle.deconvolve(w.alpha).astype(np.float32)
+    return oracle.sample(g.rowptr, g.col, g.w, seed, w.n_walks, w.p_halt, w.max_len, f_phi, f_psi)
+
+
+def assert_csr_equal(got, want: oracle.CSR, what: str, val_rtol=1e-5):
+    rp, c, v = got
+    assert np.array_equal(rp, want.rowptr), f"{what}: row pointers differ"
+    assert np.array_equal(c, want.col), f"{what}: column indices differ"
+    scale = np.maximum(np.abs(want.val), 1e-30)
+    assert (np.abs(v - want.val) <= val_rtol * scale).all(), f"{what}: values differ"
+
+
+def assert_attn_close(out_gpu: np.ndarray, ref: dict, tol: float, den_gpu: np.ndarray | None = None, what=""):
+    out_gpu = np.asarray(out_gpu, dtype=np.float64)
+    den, den_abs, num_abs, out = ref["den"], ref["den_abs"], ref["num_abs"], ref["out"]
+    ok_rows = np.abs(den) >= 1e-3 * den_abs
+    ok_rows &= den_abs > 0
+    assert ok_rows.mean() > 0.9, f"{what}: too many ill-conditioned rows"
+    bound = tol * (num_abs + np.abs(out) * den_abs[..., None]) / np.maximum(np.abs(den), 1e-300)[..., None]
+    err = np.abs(out_gpu - out)
+    bad = (err > bound + 1e-30) & ok_rows[..., None]
+    assert not bad.any(), f"{what}: {bad.sum()} outputs beyond tolerance, worst ratio {np.max(err[ok_rows] / (bound[ok_rows] + 1e-300)):.3g}"
+    if den_gpu is not None:
+        derr = np.abs(np.asarray(den_gpu, dtype=np.float64) - den)
+        assert (derr <= tol * den_abs + 1e-30).all(), f"{what}: denominators beyond tolerance"
+    # rows with no features at all must come out as zeros
+    empty = den_abs == 0
+    if empty.any():
+        assert (out_gpu[empty] == 0).all()
+
+
+def qkv_for(w, N, G=None, seed=None):
+    from workloads import configs
+    return tensors.qkv(G or w.G, N, w.m, w.d, w.dtype, configs.QKV_SEED if seed is None else seed)
