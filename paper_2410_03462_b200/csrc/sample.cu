@@ -74,7 +74,7 @@ walk_merge_kernel(const __grid_constant__ grf_walk_params P,
     const int32_t e = row >= P.N ? 1 : 0;
     const int32_t i = row - e * P.N;
 
-    const int32_t key_slots = 1 << P.seq_bits;
+    const int32_t key_slots = max(32, 1 << P.seq_bits);   // the sort pads a row to at least one key per lane
     uint32_t* keys = reinterpret_cast<uint32_t*>(smem_raw) + (size_t)warp * (key_slots + P.cap);
     float* vals = reinterpret_cast<float*>(keys + key_slots);
     const uint32_t lt_mask = (1u << lane) - 1u;
@@ -200,7 +200,11 @@ debug_walks_kernel(const __grid_constant__ grf_walk_params P,
     for (++t; t < Lp1; ++t) { tr[t] = -1; ld[t] = 0.0f; }
 }
 
-size_t walk_smem_per_warp(const grf_walk_params& P) { return ((size_t)(1 << P.seq_bits) + (size_t)P.cap) * 4; }
+size_t walk_smem_per_warp(const grf_walk_params& P)
+{
+    const size_t key_slots = (1 << P.seq_bits) < 32 ? 32 : (size_t)(1 << P.seq_bits);
+    return (key_slots + (size_t)P.cap) * 4;
+}
 
 }  // namespace
 
