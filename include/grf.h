@@ -106,6 +106,33 @@ int grf_csr_transpose(grf_ctx* ctx, int32_t rows, int32_t cols, int64_t nnz,
                       const int32_t* rowptr, const int32_t* col, const float* val,
                       int32_t* t_rowptr, int32_t* t_col, float* t_val);
 
+/*
+ * grf_csr_transpose without any allocation.  (The paper has no counterpart: this entry point exists for
+ * the sake of callers, not of the method.)
+ *
+ * Who needs it: a process whose device memory is already handed out in full to its own pool or to a
+ * framework's caching allocator, where a cudaMalloc inside a library call can fail or fragment that budget;
+ * and code that must not stall its other streams, since cudaMalloc and cudaFree wait for the whole device.
+ * grf_csr_transpose grows scratch buffers through its context when a larger matrix arrives; this variant
+ * never does.  It takes no context: its scratch (column counters, unordered buckets, scan totals, about
+ * 4.5 MB) is a fixed array inside the library image, so every GPU that loads libgrf.so holds that much
+ * until the process ends, whether or not this function is ever called.
+ *
+ * Same inputs, outputs and result as grf_csr_transpose, all DEVICE pointers on `device`; work is
+ * enqueued on `cuda_stream` (a cudaStream_t as void*, NULL = default stream) and not waited for.
+ * Limits: cols <= GRF_NOALLOC_MAX_COLS and nnz <= GRF_NOALLOC_MAX_NNZ, otherwise GRF_ERR_TOO_LARGE and
+ * nothing is launched.  The function calls no cudaMalloc/cudaFree and no allocating library routine.
+ * The first call on a device looks up the array's device address (once per device); make that first
+ * call before any stream capture begins.  All calls on one GPU share the array and it keeps the previous
+ * call's contents (the function clears what has to start at zero): two calls whose device work overlaps in
+ * time, on different streams or from different threads, race on it and give wrong results — order them.
+ */
+#define GRF_NOALLOC_MAX_COLS 65536
+#define GRF_NOALLOC_MAX_NNZ  524288
+int grf_csr_transpose_noalloc(int device, void* cuda_stream, int32_t rows, int32_t cols, int64_t nnz,
+                              const int32_t* rowptr, const int32_t* col, const float* val,
+                              int32_t* t_rowptr, int32_t* t_col, float* t_val);
+
 /* Bytes of DEVICE workspace with which grf_masked_linear_attn processes all G problems in one pass
  * (states S [G][R][m][d] in the storage type and z [G][R][m] in fp32).  A smaller workspace is accepted
  * as long as it holds one problem; the call then works through G in chunks.  0 on invalid arguments. */

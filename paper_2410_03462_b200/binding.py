@@ -36,6 +36,7 @@ _SIGNATURES = {
     "grf_features_copy": (_int, [_vp, _vp, _int, _vp, _vp, _vp]),
     "grf_features_free": (_int, [_vp]),
     "grf_csr_transpose": (_int, [_vp, _i32, _i32, _i64, _vp, _vp, _vp, _vp, _vp, _vp]),
+    "grf_csr_transpose_noalloc": (_int, [_int, _vp, _i32, _i32, _i64, _vp, _vp, _vp, _vp, _vp, _vp]),
     "grf_attn_workspace_bytes": (_sz, [_i32, _i32, _i32, _i32, _int]),
     "grf_masked_linear_attn": (_int, [_vp, _vp, _i32, _i32, _i32, _i32, _int, _vp, _vp, _vp, _vp, _vp, _vp, _sz]),
     "grf_step_host": (_int, [_vp, _i32, _vp, _vp, _vp, _u64, _i32, _f32, _i32, _vp, _vp,
@@ -172,6 +173,12 @@ def grf_features_free(features: int):
 def grf_csr_transpose(ctx, rows, cols, nnz, rowptr, col, val, t_rowptr, t_col, t_val):
     _check(lib.grf_csr_transpose(ctx, rows, cols, nnz, _dev(rowptr), _dev(col), _dev(val),
                                  _dev(t_rowptr), _dev(t_col), _dev(t_val)), "grf_csr_transpose")
+
+
+def grf_csr_transpose_noalloc(device, stream, rows, cols, nnz, rowptr, col, val, t_rowptr, t_col, t_val):
+    """Allocation-free variant of grf_csr_transpose (fixed in-library scratch; see grf.h for its limits)."""
+    _check(lib.grf_csr_transpose_noalloc(device, stream, rows, cols, nnz, _dev(rowptr), _dev(col), _dev(val),
+                                         _dev(t_rowptr), _dev(t_col), _dev(t_val)), "grf_csr_transpose_noalloc")
 
 
 def grf_attn_workspace_bytes(G, R, m, d, dtype) -> int:

@@ -91,6 +91,9 @@ int grf_walk_params_init(grf_walk_params* p, int32_t N, uint64_t seed, int32_t n
 // out[s*(n+1) + i], with out[s*(n+1) + n] = total.
 int grf_exclusive_scan(grf_ctx* ctx, const int32_t* in, int32_t* out, int32_t n, int32_t segments);
 
+int grf_exclusive_scan_scratch(cudaStream_t stream, const int32_t* in, int32_t* out, int32_t n, int32_t segments,
+                               int32_t* totals);
+
 // transpose.cu
 int grf_transpose_launch(grf_ctx* ctx, int32_t rows, int32_t cols, int64_t nnz,
                          const int32_t* rowptr, const int32_t* col, const float* val,

@@ -111,3 +111,18 @@ int grf_exclusive_scan(grf_ctx* ctx, const int32_t* in, int32_t* out, int32_t n,
     GRF_CUDA_TRY(cudaGetLastError());
     return GRF_OK;
 }
+
+// Same three launches with the block-total scratch supplied by the caller (needs ceil(n / 4096) * segments
+// int32 entries) and no context: used where nothing may be allocated.
+int grf_exclusive_scan_scratch(cudaStream_t stream, const int32_t* in, int32_t* out, int32_t n, int32_t segments,
+                               int32_t* totals)
+{
+    if (n <= 0 || segments <= 0 || !totals) return GRF_ERR_INVALID;
+    const int nblocks = grf_ceil_div(n, SCAN_TILE);
+    const dim3 grid(nblocks, segments);
+    scan_block_totals_kernel<<<grid, SCAN_THREADS, 0, stream>>>(in, n, totals);
+    scan_totals_kernel<<<segments, SCAN_THREADS, 0, stream>>>(totals, nblocks);
+    scan_write_kernel<<<grid, SCAN_THREADS, 0, stream>>>(in, n, totals, out);
+    GRF_CUDA_TRY(cudaGetLastError());
+    return GRF_OK;
+}

@@ -112,3 +112,61 @@ extern "C" int grf_csr_transpose(grf_ctx* ctx, int32_t rows, int32_t cols, int64
     GRF_CUDA_TRY(cudaSetDevice(ctx->device));
     return grf_transpose_launch(ctx, rows, cols, nnz, rowptr, col, val, t_rowptr, t_col, t_val);
 }
+
+// ---------------------------------------------------------------------------------------------------
+// Variant that allocates nothing: its scratch is a fixed array that is part of the loaded module.
+
+namespace {
+
+constexpr int32_t NOALLOC_MAX_COLS = GRF_NOALLOC_MAX_COLS;
+constexpr int64_t NOALLOC_MAX_NNZ = GRF_NOALLOC_MAX_NNZ;
+constexpr size_t NOALLOC_CURSOR_WORDS = (size_t)NOALLOC_MAX_COLS + 64;          // counts / cursors, padded
+constexpr size_t NOALLOC_TOTALS_WORDS = 64;                                     // scan block totals (<= 17 used)
+constexpr size_t NOALLOC_WORDS = NOALLOC_CURSOR_WORDS + NOALLOC_TOTALS_WORDS + 2 * (size_t)NOALLOC_MAX_NNZ;
+
+// Every GPU that loads this library holds one copy of this array until the process exits.
+static __device__ __align__(256) uint32_t g_noalloc_scratch[NOALLOC_WORDS];
+
+constexpr int NOALLOC_MAX_DEVICES = 64;
+uint32_t* g_noalloc_ptr[NOALLOC_MAX_DEVICES] = {};   // device address of the array, per device, once resolved
+
+}  // namespace
+
+extern "C" int grf_csr_transpose_noalloc(int device, void* cuda_stream, int32_t rows, int32_t cols, int64_t nnz,
+                                         const int32_t* rowptr, const int32_t* col, const float* val,
+                                         int32_t* t_rowptr, int32_t* t_col, float* t_val)
+{
+    if (device < 0 || device >= NOALLOC_MAX_DEVICES || rows <= 0 || cols <= 0 || nnz < 0 || !rowptr || !t_rowptr)
+        return GRF_ERR_INVALID;
+    if (nnz > 0 && (!col || !val || !t_col || !t_val)) return GRF_ERR_INVALID;
+    if (cols > NOALLOC_MAX_COLS || nnz > NOALLOC_MAX_NNZ) return GRF_ERR_TOO_LARGE;
+    GRF_CUDA_TRY(cudaSetDevice(device));
+    if (!g_noalloc_ptr[device]) {
+        // In host code the array's name only stands for the symbol; the address kernels can use has to be
+        // asked for, with the owning device current.
+        uint32_t* p = nullptr;
+        GRF_CUDA_TRY(cudaGetSymbolAddress((void**)&p, g_noalloc_scratch));
+        if (!p) return GRF_ERR_CUDA;
+        g_noalloc_ptr[device] = p;
+    }
+    cudaStream_t stream = (cudaStream_t)cuda_stream;
+    int32_t* cursor = (int32_t*)g_noalloc_ptr[device];
+    int32_t* totals = cursor + NOALLOC_CURSOR_WORDS;
+    int32_t* tmp_row = totals + NOALLOC_TOTALS_WORDS;
+    float* tmp_val = (float*)(tmp_row + NOALLOC_MAX_NNZ);
+    // the array keeps whatever the previous call left: the per-column counts must start from zero
+    GRF_CUDA_TRY(cudaMemsetAsync(cursor, 0, sizeof(int32_t) * ((size_t)cols + 1), stream));
+    if (nnz > 0) {
+        int blocks = grf_ceil_div(nnz, 256);
+        if (blocks > 148 * 16) blocks = 148 * 16;
+        column_histogram_kernel<<<blocks, 256, 0, stream>>>(nnz, col, cursor);
+    }
+    GRF_TRY(grf_exclusive_scan_scratch(stream, cursor, t_rowptr, cols, 1, totals));
+    copy_i32_kernel<<<grf_ceil_div(cols, 256), 256, 0, stream>>>(t_rowptr, cursor, cols);
+    if (nnz > 0) {
+        bucket_scatter_kernel<<<grf_ceil_div(rows, 8), 256, 0, stream>>>(rows, rowptr, col, val, cursor, tmp_row, tmp_val);
+        bucket_order_kernel<<<grf_ceil_div(cols, 4), 128, 0, stream>>>(cols, t_rowptr, tmp_row, tmp_val, t_col, t_val);
+    }
+    GRF_CUDA_TRY(cudaGetLastError());
+    return GRF_OK;
+}
