@@ -31,6 +31,7 @@ extern "C" {
 #define GRF_ERR_CUDA       (-4)  /* a CUDA runtime call failed                                                   */
 #define GRF_ERR_NOMEM      (-5)  /* device or host allocation failed                                             */
 #define GRF_ERR_BADGRAPH   (-6)  /* CSR input inconsistent (host-side checks of host-resident graphs only)       */
+#define GRF_ERR_TIMEOUT    (-7)  /* a kernel gave up a bounded wait; its outputs are not valid                   */
 
 #define GRF_DTYPE_F32  0
 #define GRF_DTYPE_BF16 1
@@ -164,6 +165,14 @@ int grf_step_host(grf_ctx* ctx, int32_t N, const int32_t* rowptr, const int32_t*
                   const float* f_phi, const float* f_psi,
                   int32_t G, int32_t m, int32_t d, int dtype,
                   const void* phiQ, const void* phiK, const void* V, void* out);
+
+/* Waits for the context's stream and reports whether any kernel since the previous check gave up one of its
+ * bounded waits (GRF_ERR_TIMEOUT; the affected outputs are invalid), else GRF_OK. */
+int grf_ctx_check(grf_ctx* ctx);
+
+/* Chooses the gather-contract kernel for bf16 problems: 1 (default) = tensor-core kernel where a block plan
+ * exists and m, d are multiples of 16; 0 = plain-ALU kernel always.  Results agree within the stated tolerance. */
+int grf_ctx_use_tensor_cores(grf_ctx* ctx, int enable);
 
 /* Number of kernels the context has launched since it was created (for accounting in benchmarks). */
 int64_t grf_ctx_launch_count(const grf_ctx* ctx);

@@ -14,6 +14,7 @@ from . import build as _build
 
 GRF_OK = 0
 GRF_ERR_INVALID, GRF_ERR_TOO_LARGE, GRF_ERR_WORKSPACE, GRF_ERR_CUDA, GRF_ERR_NOMEM, GRF_ERR_BADGRAPH = -1, -2, -3, -4, -5, -6
+GRF_ERR_TIMEOUT = -7
 GRF_DTYPE_F32, GRF_DTYPE_BF16 = 0, 1
 
 _LIB_PATH = _build.LIB
@@ -42,6 +43,8 @@ _SIGNATURES = {
     "grf_step_host": (_int, [_vp, _i32, _vp, _vp, _vp, _u64, _i32, _f32, _i32, _vp, _vp,
                              _i32, _i32, _i32, _int, _vp, _vp, _vp, _vp]),
     "grf_ctx_launch_count": (_i64, [_vp]),
+    "grf_ctx_check": (_int, [_vp]),
+    "grf_ctx_use_tensor_cores": (_int, [_vp, _int]),
     "grf_ctx_enable_timing": (_int, [_vp, _int]),
     "grf_ctx_kernel_times": (_int, [_vp, _vp, _vp]),
     "grf_strerror": (ctypes.c_char_p, [_int]),
@@ -104,6 +107,14 @@ def grf_ctx_destroy(ctx: int):
 
 def grf_ctx_launch_count(ctx: int) -> int:
     return int(lib.grf_ctx_launch_count(ctx))
+
+
+def grf_ctx_check(ctx: int):
+    _check(lib.grf_ctx_check(ctx), "grf_ctx_check")
+
+
+def grf_ctx_use_tensor_cores(ctx: int, enable: bool):
+    _check(lib.grf_ctx_use_tensor_cores(ctx, int(enable)), "grf_ctx_use_tensor_cores")
 
 
 KERNEL_CLASSES = ("walk_merge", "scan", "compact", "regroup", "build_states", "gather_contract")

@@ -43,7 +43,9 @@ extern "C" int grf_ctx_create(grf_ctx** out, int device, void* cuda_stream)
     c->device = device;
     c->stream = (cudaStream_t)cuda_stream;
     if (cudaDeviceGetAttribute(&c->sm_count, cudaDevAttrMultiProcessorCount, device) != cudaSuccess ||
-        cudaMallocHost((void**)&c->pinned, 64) != cudaSuccess) {
+        cudaMallocHost((void**)&c->pinned, 64) != cudaSuccess ||
+        cudaMalloc((void**)&c->error_word, sizeof(int)) != cudaSuccess ||
+        cudaMemset(c->error_word, 0, sizeof(int)) != cudaSuccess) {
         cudaGetLastError();
         delete c;
         return GRF_ERR_CUDA;
@@ -63,6 +65,7 @@ extern "C" int grf_ctx_destroy(grf_ctx* ctx)
     for (grf_buf* b : bufs) grf_buf_release(b);
     if (ctx->h_feat) grf_features_free(ctx->h_feat);
     if (ctx->pinned) cudaFreeHost(ctx->pinned);
+    if (ctx->error_word) cudaFree(ctx->error_word);
     for (auto& t : ctx->timed) { cudaEventDestroy(t.beg); cudaEventDestroy(t.end); }
     for (cudaEvent_t e : ctx->free_events) cudaEventDestroy(e);
     delete ctx;
@@ -90,6 +93,26 @@ grf_launch_scope::~grf_launch_scope()
     if (!ctx->timing || !beg || !end) return;
     cudaEventRecord(end, ctx->stream);
     ctx->timed.push_back({cls, beg, end});
+}
+
+extern "C" int grf_ctx_use_tensor_cores(grf_ctx* ctx, int enable)
+{
+    if (!ctx) return GRF_ERR_INVALID;
+    ctx->use_tensor_cores = enable != 0;
+    return GRF_OK;
+}
+
+extern "C" int grf_ctx_check(grf_ctx* ctx)
+{
+    if (!ctx) return GRF_ERR_INVALID;
+    GRF_CUDA_TRY(cudaSetDevice(ctx->device));
+    GRF_CUDA_TRY(cudaMemcpyAsync(ctx->pinned + 8, ctx->error_word, sizeof(int), cudaMemcpyDeviceToHost, ctx->stream));
+    GRF_CUDA_TRY(cudaStreamSynchronize(ctx->stream));
+    if (ctx->pinned[8] != 0) {
+        cudaMemsetAsync(ctx->error_word, 0, sizeof(int), ctx->stream);
+        return GRF_ERR_TIMEOUT;
+    }
+    return GRF_OK;
 }
 
 extern "C" int grf_ctx_enable_timing(grf_ctx* ctx, int enable)
@@ -141,6 +164,8 @@ extern "C" int grf_features_free(grf_features* feat)
     if (!feat) return GRF_ERR_INVALID;
     cudaSetDevice(feat->device);
     csr_release(&feat->phi); csr_release(&feat->psi); csr_release(&feat->psit);
+    grf_buf_release(&feat->plan_off); grf_buf_release(&feat->plan_cnt);
+    grf_buf_release(&feat->plan_col); grf_buf_release(&feat->plan_total);
     delete feat;
     return GRF_OK;
 }
@@ -208,6 +233,7 @@ extern "C" int grf_features_from_csr(grf_ctx* ctx, int32_t N, int32_t R,
     rc = grf_transpose_launch(ctx, N, R, nnz_psi, (const int32_t*)f->psi.rowptr.ptr, (const int32_t*)f->psi.col.ptr,
                               (const float*)f->psi.val.ptr, (int32_t*)f->psit.rowptr.ptr,
                               (int32_t*)f->psit.col.ptr, (float*)f->psit.val.ptr);
+    if (rc == GRF_OK) rc = grf_build_block_plan(ctx, f);
     if (rc == GRF_OK && cudaGetLastError() != cudaSuccess) rc = GRF_ERR_CUDA;
     if (rc != GRF_OK) { grf_features_free(f); return rc; }
     *out = f;
@@ -260,7 +286,11 @@ extern "C" int grf_masked_linear_attn(grf_ctx* ctx, const grf_features* feat, in
         char* o_ptr = (char*)out + (size_t)g0 * N * d * es;
         float* den_ptr = den_out ? den_out + (size_t)g0 * N : nullptr;
         GRF_TRY(grf_build_states(ctx, feat->psit, gc, N, m, d, dtype, k_ptr, v_ptr, Sbuf, zbuf));
-        GRF_TRY(grf_gather_contract(ctx, feat->phi, gc, N, m, d, dtype, q_ptr, Sbuf, zbuf, o_ptr, den_ptr));
+        int rc = 1;
+        if (dtype == GRF_DTYPE_BF16 && ctx->use_tensor_cores)
+            rc = grf_gather_contract_tc(ctx, feat, gc, N, m, d, q_ptr, Sbuf, zbuf, o_ptr, den_ptr);
+        if (rc > 0) rc = grf_gather_contract_alu(ctx, feat->phi, gc, N, m, d, dtype, q_ptr, Sbuf, zbuf, o_ptr, den_ptr);
+        GRF_TRY(rc);
     }
     return GRF_OK;
 }
@@ -315,8 +345,7 @@ extern "C" int grf_step_host(grf_ctx* ctx, int32_t N, const int32_t* rowptr, con
     GRF_TRY(grf_masked_linear_attn(ctx, ctx->h_feat, G, N, m, d, dtype, ctx->h_q.ptr, ctx->h_k.ptr, ctx->h_v.ptr,
                                    ctx->h_out.ptr, nullptr, ctx->h_ws.ptr, ctx->h_ws.bytes));
     GRF_CUDA_TRY(cudaMemcpyAsync(out, ctx->h_out.ptr, v_bytes, cudaMemcpyDeviceToHost, s));
-    GRF_CUDA_TRY(cudaStreamSynchronize(s));
-    return GRF_OK;
+    return grf_ctx_check(ctx);
 }
 
 extern "C" const char* grf_strerror(int code)
@@ -329,6 +358,7 @@ extern "C" const char* grf_strerror(int code)
         case GRF_ERR_CUDA: return "CUDA runtime error";
         case GRF_ERR_NOMEM: return "out of memory";
         case GRF_ERR_BADGRAPH: return "inconsistent graph CSR";
+        case GRF_ERR_TIMEOUT: return "a kernel gave up a bounded wait";
         default: return "unknown error";
     }
 }

@@ -1,26 +1,23 @@
 // Gather-and-contract with normalisation (Alg. 1 step 5, Eq. 12):
 //   num_i = sum_l Phi_il phi(q_i)^T S_l,  den_i = sum_l Phi_il phi(q_i)^T z_l,  out_i = num_i / den_i.
-// One warp per (problem g, query i).  Every S_l tile is read with 16-byte loads, a group of lanes
-// per tile row; sums are carried in fp32 in a fixed order.
+//
+// Plain-ALU kernel (any supported m, d; fp32 or bf16 storage): one warp per (problem g, query i).  A tile
+// is read as consecutive 16-byte chunks (512 contiguous bytes per warp-wide load); sums are carried in
+// fp32 in a fixed order.
 #include "grf_internal.cuh"
 
 namespace {
 
-template <typename T> struct Vec16;
-template <> struct Vec16<float> {
-    static constexpr int N = 4;
+template <typename T> struct Chunk;
+template <> struct Chunk<float> {
     __device__ static __forceinline__ void load(const float* p, float (&v)[4])
     {
         const float4 x = __ldg(reinterpret_cast<const float4*>(p));
         v[0] = x.x; v[1] = x.y; v[2] = x.z; v[3] = x.w;
     }
-    __device__ static __forceinline__ void store(float* p, const float (&v)[4])
-    {
-        *reinterpret_cast<float4*>(p) = make_float4(v[0], v[1], v[2], v[3]);
-    }
+    __device__ static __forceinline__ void store1(float* p, float x) { *p = x; }
 };
-template <> struct Vec16<__nv_bfloat16> {
-    static constexpr int N = 8;
+template <> struct Chunk<__nv_bfloat16> {
     __device__ static __forceinline__ void load(const __nv_bfloat16* p, float (&v)[8])
     {
         const uint4 x = __ldg(reinterpret_cast<const uint4*>(p));
@@ -31,16 +28,7 @@ template <> struct Vec16<__nv_bfloat16> {
             v[2 * q + 1] = __uint_as_float(w[q] & 0xffff0000u);
         }
     }
-    __device__ static __forceinline__ void store(__nv_bfloat16* p, const float (&v)[8])
-    {
-        uint32_t w[4];
-#pragma unroll
-        for (int q = 0; q < 4; ++q) {
-            __nv_bfloat162 h = __floats2bfloat162_rn(v[2 * q], v[2 * q + 1]);
-            w[q] = *reinterpret_cast<uint32_t*>(&h);
-        }
-        *reinterpret_cast<uint4*>(p) = make_uint4(w[0], w[1], w[2], w[3]);
-    }
+    __device__ static __forceinline__ void store1(__nv_bfloat16* p, float x) { *p = __float2bfloat16_rn(x); }
 };
 
 template <typename T> __device__ __forceinline__ float to_f32(T x);
@@ -49,23 +37,15 @@ template <> __device__ __forceinline__ float to_f32<__nv_bfloat16>(__nv_bfloat16
 
 constexpr int GATHER_WARPS = 4;
 
-template <typename T, int D> struct GatherShape {
-    static constexpr int VEC = (Vec16<T>::N < D) ? Vec16<T>::N : D;   // elements per lane per tile row
-    static constexpr int LPR = D / VEC;                               // lanes that share one tile row
-    static constexpr int RPI = 32 / LPR;                              // tile rows per warp-wide load
-};
-
 template <typename T, int M, int D>
 __global__ void __launch_bounds__(GATHER_WARPS * 32)
 gather_contract_kernel(int32_t N, int32_t R, const int32_t* __restrict__ rowptr, const int32_t* __restrict__ col,
                        const float* __restrict__ val, const T* __restrict__ phiQ, const T* __restrict__ S,
                        const float* __restrict__ z, T* __restrict__ out, float* __restrict__ den_out)
 {
-    constexpr int VEC = Vec16<T>::N;
-    static_assert(D % VEC == 0, "head dimension must fill whole 16-byte vectors");
-    constexpr int LPR = D / VEC;
-    constexpr int RPI = 32 / LPR;
-    static_assert(LPR >= 1 && LPR <= 32, "unsupported head dimension");
+    constexpr int CH = grf_tile_chunk<T>();
+    constexpr int NCHUNK = (M / CH) * D;            // 16-byte chunks per tile, chunk x = (a / CH) * D + b
+    constexpr int NACC = D >= 32 ? D / 32 : 1;      // output columns per lane
     __shared__ float qs[GATHER_WARPS][M];
 
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -76,11 +56,9 @@ gather_contract_kernel(int32_t N, int32_t R, const int32_t* __restrict__ rowptr,
     for (int a = lane; a < M; a += 32) qs[warp][a] = to_f32(qrow[a]);
     __syncwarp();
 
-    const int sub = lane / LPR;         // which of the RPI rows this lane reads
-    const int cg = lane % LPR;          // which 16-byte column group
-    float acc[VEC];
+    float acc[NACC];
 #pragma unroll
-    for (int v = 0; v < VEC; ++v) acc[v] = 0.0f;
+    for (int j = 0; j < NACC; ++j) acc[j] = 0.0f;
     float den = 0.0f;
 
     const T* Sg = S + (size_t)g * R * M * D;
@@ -91,31 +69,35 @@ gather_contract_kernel(int32_t N, int32_t R, const int32_t* __restrict__ rowptr,
         const T* tile = Sg + (size_t)l * M * D;
         const float* zl = zg + (size_t)l * M;
 #pragma unroll
-        for (int a0 = 0; a0 < M; a0 += RPI) {
-            const int a = a0 + sub;
-            if (RPI <= M || a < M) {
-                const float c = phi * qs[warp][a];
-                float s[VEC];
-                Vec16<T>::load(tile + (size_t)a * D + cg * VEC, s);
+        for (int x0 = 0; x0 < NCHUNK; x0 += 32) {
+            const int x = x0 + lane;
+            if (NCHUNK % 32 == 0 || x < NCHUNK) {
+                const int kc = D >= 32 ? x0 / D : x / D;
+                float s[CH];
+                Chunk<T>::load(tile + (size_t)x * CH, s);
+                float dot = 0.0f;
 #pragma unroll
-                for (int v = 0; v < VEC; ++v) acc[v] = fmaf(c, s[v], acc[v]);
-                if (cg == 0) den = fmaf(c, __ldg(zl + a), den);
+                for (int c = 0; c < CH; ++c) dot = fmaf(qs[warp][kc * CH + c], s[c], dot);
+                acc[D >= 32 ? (x0 % D) / 32 : 0] = fmaf(phi, dot, acc[D >= 32 ? (x0 % D) / 32 : 0]);
             }
         }
+        for (int a = lane; a < M; a += 32) den = fmaf(phi * qs[warp][a], __ldg(zl + a), den);
     }
+    if (D < 32) {
+        // lanes with the same column b = lane % D hold partial sums over different row chunks
 #pragma unroll
-    for (int off = LPR; off < 32; off <<= 1)
-#pragma unroll
-        for (int v = 0; v < VEC; ++v) acc[v] += __shfl_xor_sync(0xffffffffu, acc[v], off);
+        for (int off = D; off < 32; off <<= 1) acc[0] += __shfl_xor_sync(0xffffffffu, acc[0], off);
+    }
 #pragma unroll
     for (int off = 1; off < 32; off <<= 1) den += __shfl_xor_sync(0xffffffffu, den, off);
 
-    if (lane < LPR) {
-        const float inv = den != 0.0f ? 1.0f / den : 0.0f;
-        float o[VEC];
+    const float inv = den != 0.0f ? 1.0f / den : 0.0f;
+    T* orow = out + ((size_t)g * N + i) * D;
+    if (D >= 32) {
 #pragma unroll
-        for (int v = 0; v < VEC; ++v) o[v] = acc[v] * inv;
-        Vec16<T>::store(out + ((size_t)g * N + i) * D + cg * VEC, o);
+        for (int j = 0; j < NACC; ++j) Chunk<T>::store1(orow + j * 32 + lane, acc[j] * inv);
+    } else if (lane < D) {
+        Chunk<T>::store1(orow + lane, acc[0] * inv);
     }
     if (lane == 0 && den_out) den_out[(size_t)g * N + i] = den;
 }
@@ -132,11 +114,11 @@ int launch_m(grf_ctx* ctx, const grf_csr_dev& phi, int32_t G, int32_t N, int32_t
             (const float*)phi.val.ptr, (const T*)phiQ, (const T*)S, z, (T*)out, den_out);                   \
         break;
     {
-    grf_launch_scope scope(ctx, 5);
-    switch (d) {
-        GRF_GATHER_CASE(8) GRF_GATHER_CASE(16) GRF_GATHER_CASE(32) GRF_GATHER_CASE(64) GRF_GATHER_CASE(128)
-        default: return GRF_ERR_INVALID;
-    }
+        grf_launch_scope scope(ctx, 5);
+        switch (d) {
+            GRF_GATHER_CASE(8) GRF_GATHER_CASE(16) GRF_GATHER_CASE(32) GRF_GATHER_CASE(64) GRF_GATHER_CASE(128)
+            default: return GRF_ERR_INVALID;
+        }
     }
 #undef GRF_GATHER_CASE
     return cudaGetLastError() == cudaSuccess ? GRF_OK : GRF_ERR_CUDA;
@@ -158,8 +140,8 @@ int launch_t(grf_ctx* ctx, const grf_csr_dev& phi, int32_t G, int32_t N, int32_t
 
 }  // namespace
 
-int grf_gather_contract(grf_ctx* ctx, const grf_csr_dev& phi, int32_t G, int32_t N, int32_t m, int32_t d, int dtype,
-                        const void* phiQ, const void* S, const float* z, void* out, float* den_out)
+int grf_gather_contract_alu(grf_ctx* ctx, const grf_csr_dev& phi, int32_t G, int32_t N, int32_t m, int32_t d,
+                            int dtype, const void* phiQ, const void* S, const float* z, void* out, float* den_out)
 {
     if (G > 65535) return GRF_ERR_TOO_LARGE;
     if (dtype == GRF_DTYPE_F32) return launch_t<float>(ctx, phi, G, N, m, d, phiQ, S, z, out, den_out);

@@ -2,6 +2,8 @@
 // z_l = sum_j Psi_jl phi(k_j)  (m), for every problem g and node l — the rows of Phi_K^T V and
 // Phi_K^T 1 of Corollary 3.4.  A segmented reduction over the column-grouped Psi^T with a fixed
 // summation order (ascending j), fp32 accumulation, no atomics.
+//
+// This file holds the plain-ALU kernel (any supported m, d; fp32 or bf16 storage).
 #include "grf_internal.cuh"
 
 namespace {
@@ -10,53 +12,57 @@ template <typename T> __device__ __forceinline__ float to_f32(T x);
 template <> __device__ __forceinline__ float to_f32<float>(float x) { return x; }
 template <> __device__ __forceinline__ float to_f32<__nv_bfloat16>(__nv_bfloat16 x) { return __bfloat162float(x); }
 
-__device__ __forceinline__ void store4(float* dst, const float (&v)[4])
+// one 16-byte chunk of the tile: CH consecutive feature rows a of one column b
+__device__ __forceinline__ void store_chunk(float* dst, const float (&v)[4])
 {
     *reinterpret_cast<float4*>(dst) = make_float4(v[0], v[1], v[2], v[3]);
 }
-__device__ __forceinline__ void store4(__nv_bfloat16* dst, const float (&v)[4])
+__device__ __forceinline__ void store_chunk(__nv_bfloat16* dst, const float (&v)[8])
 {
-    __nv_bfloat162 lo = __floats2bfloat162_rn(v[0], v[1]);
-    __nv_bfloat162 hi = __floats2bfloat162_rn(v[2], v[3]);
-    uint2 u;
-    u.x = *reinterpret_cast<uint32_t*>(&lo);
-    u.y = *reinterpret_cast<uint32_t*>(&hi);
-    *reinterpret_cast<uint2*>(dst) = u;
+    uint32_t w[4];
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+        __nv_bfloat162 h = __floats2bfloat162_rn(v[2 * q], v[2 * q + 1]);
+        w[q] = *reinterpret_cast<uint32_t*>(&h);
+    }
+    *reinterpret_cast<uint4*>(dst) = make_uint4(w[0], w[1], w[2], w[3]);
 }
 
-template <int M, int D>
+template <typename T, int M, int D>
 struct StateTiling {
-    static constexpr int TX = D / 4;                              // threads across a row of the tile
-    static constexpr int THREADS = (TX * M < 128) ? TX * M : 128;
-    static constexpr int TY = THREADS / TX;
-    static constexpr int TA = M / TY;                             // tile rows per thread
+    static constexpr int CH = grf_tile_chunk<T>();               // feature rows per 16-byte chunk
+    static constexpr int TXB = D < 32 ? D : 32;                   // threads across the columns b
+    static constexpr int TB = D / TXB;                            // columns per thread (b, b+TXB, ...)
+    static constexpr int KC = M / CH;                             // chunks along a
+    static constexpr int THREADS = KC * TXB;
     static constexpr int JC = 8;                                  // source rows staged per step
 };
 
-// One CTA per (node l, problem g).  Each thread keeps a TA x 4 block of the m x d tile in registers.
+// One CTA per (node l, problem g).  Thread (kc, bx) keeps the CH x TB block
+// {a in chunk kc} x {b = bx + TXB*t} of the tile in registers and writes it as TB 16-byte chunks.
 template <typename T, int M, int D>
-__global__ void __launch_bounds__(StateTiling<M, D>::THREADS)
+__global__ void __launch_bounds__(StateTiling<T, M, D>::THREADS)
 build_states_kernel(int32_t R, int32_t N, const int32_t* __restrict__ t_rowptr, const int32_t* __restrict__ t_col,
                     const float* __restrict__ t_val, const T* __restrict__ phiK, const T* __restrict__ V,
                     T* __restrict__ S, float* __restrict__ z)
 {
-    using Tl = StateTiling<M, D>;
-    constexpr int TX = Tl::TX, TY = Tl::TY, TA = Tl::TA, JC = Tl::JC, THREADS = Tl::THREADS;
+    using Tl = StateTiling<T, M, D>;
+    constexpr int CH = Tl::CH, TXB = Tl::TXB, TB = Tl::TB, JC = Tl::JC, THREADS = Tl::THREADS;
     __shared__ __align__(16) float ks[JC][M];
     __shared__ __align__(16) float vs[JC][D];
 
     const int32_t l = blockIdx.x, g = blockIdx.y;
-    const int tid = threadIdx.x, tx = tid % TX, ty = tid / TX;
+    const int tid = threadIdx.x, bx = tid % TXB, kc = tid / TXB;
     const T* Kg = phiK + (size_t)g * N * M;
     const T* Vg = V + (size_t)g * N * D;
 
-    float acc[TA][4];
-    float zacc[TA];
+    float acc[TB][CH];
+    float zacc[CH];
 #pragma unroll
-    for (int r = 0; r < TA; ++r) {
-        zacc[r] = 0.0f;
+    for (int c = 0; c < CH; ++c) {
+        zacc[c] = 0.0f;
 #pragma unroll
-        for (int c = 0; c < 4; ++c) acc[r][c] = 0.0f;
+        for (int t = 0; t < TB; ++t) acc[t][c] = 0.0f;
     }
 
     const int32_t beg = t_rowptr[l], end = t_rowptr[l + 1];
@@ -75,27 +81,28 @@ build_states_kernel(int32_t R, int32_t N, const int32_t* __restrict__ t_rowptr, 
         __syncthreads();
 #pragma unroll
         for (int jj = 0; jj < JC; ++jj) {
-            const float4 v4 = *reinterpret_cast<const float4*>(&vs[jj][tx * 4]);
+            float kr[CH];
 #pragma unroll
-            for (int r = 0; r < TA; ++r) {
-                const float kr = ks[jj][ty + r * TY];
-                acc[r][0] = fmaf(kr, v4.x, acc[r][0]);
-                acc[r][1] = fmaf(kr, v4.y, acc[r][1]);
-                acc[r][2] = fmaf(kr, v4.z, acc[r][2]);
-                acc[r][3] = fmaf(kr, v4.w, acc[r][3]);
-                zacc[r] += kr;
+            for (int c = 0; c < CH; ++c) kr[c] = ks[jj][kc * CH + c];
+#pragma unroll
+            for (int t = 0; t < TB; ++t) {
+                const float vb = vs[jj][bx + t * TXB];
+#pragma unroll
+                for (int c = 0; c < CH; ++c) acc[t][c] = fmaf(kr[c], vb, acc[t][c]);
             }
+#pragma unroll
+            for (int c = 0; c < CH; ++c) zacc[c] += kr[c];
         }
         __syncthreads();
     }
 
     T* Sl = S + ((size_t)g * R + l) * M * D;
 #pragma unroll
-    for (int r = 0; r < TA; ++r) store4(Sl + (size_t)(ty + r * TY) * D + tx * 4, acc[r]);
-    if (tx == 0) {
+    for (int t = 0; t < TB; ++t) store_chunk(Sl + grf_tile_index<T>(kc * CH, bx + t * TXB, D), acc[t]);
+    if (bx == 0) {
         float* zl = z + ((size_t)g * R + l) * M;
 #pragma unroll
-        for (int r = 0; r < TA; ++r) zl[ty + r * TY] = zacc[r];
+        for (int c = 0; c < CH; ++c) zl[kc * CH + c] = zacc[c];
     }
 }
 
@@ -106,16 +113,16 @@ int launch_m(grf_ctx* ctx, const grf_csr_dev& psit, int32_t G, int32_t N, int32_
     const dim3 grid(psit.rows, G);
 #define GRF_STATE_CASE(DD)                                                                                  \
     case DD:                                                                                                \
-        build_states_kernel<T, M, DD><<<grid, StateTiling<M, DD>::THREADS, 0, ctx->stream>>>(               \
+        build_states_kernel<T, M, DD><<<grid, StateTiling<T, M, DD>::THREADS, 0, ctx->stream>>>(            \
             psit.rows, N, (const int32_t*)psit.rowptr.ptr, (const int32_t*)psit.col.ptr,                    \
             (const float*)psit.val.ptr, (const T*)phiK, (const T*)V, (T*)S, z);                            \
         break;
     {
-    grf_launch_scope scope(ctx, 4);
-    switch (d) {
-        GRF_STATE_CASE(8) GRF_STATE_CASE(16) GRF_STATE_CASE(32) GRF_STATE_CASE(64) GRF_STATE_CASE(128)
-        default: return GRF_ERR_INVALID;
-    }
+        grf_launch_scope scope(ctx, 4);
+        switch (d) {
+            GRF_STATE_CASE(8) GRF_STATE_CASE(16) GRF_STATE_CASE(32) GRF_STATE_CASE(64) GRF_STATE_CASE(128)
+            default: return GRF_ERR_INVALID;
+        }
     }
 #undef GRF_STATE_CASE
     return cudaGetLastError() == cudaSuccess ? GRF_OK : GRF_ERR_CUDA;

@@ -43,6 +43,8 @@ struct grf_ctx {
     grf_buf h_rowptr, h_col, h_w, h_q, h_k, h_v, h_out, h_ws;
     grf_features* h_feat = nullptr;
     int32_t* pinned = nullptr;      // small pinned host block for read-backs
+    int* error_word = nullptr;      // device word set by a kernel that gave up a bounded wait
+    bool use_tensor_cores = true;
     // optional per-launch timing
     bool timing = false;
     struct timed_launch { int cls; cudaEvent_t beg, end; };
@@ -66,9 +68,15 @@ struct grf_csr_dev {
     grf_buf rowptr, col, val;
 };
 
+#define GRF_PLAN_BLOCK 128   // queries per block of the tensor-core gather kernel
+
 struct grf_features {
     int device = 0;
     grf_csr_dev phi, psi, psit;
+    // block plan of Phi: per block of GRF_PLAN_BLOCK rows, the sorted distinct columns
+    grf_buf plan_off, plan_cnt, plan_col, plan_total;
+    int32_t plan_blocks = 0;
+    bool plan_ready = false;
 };
 
 int grf_buf_reserve(grf_buf* b, size_t bytes);          // grows (contents not preserved)
@@ -102,7 +110,21 @@ int grf_transpose_launch(grf_ctx* ctx, int32_t rows, int32_t cols, int64_t nnz,
 // attn_state.cu / attn_gather.cu
 int grf_build_states(grf_ctx* ctx, const grf_csr_dev& psit, int32_t G, int32_t N, int32_t m, int32_t d, int dtype,
                      const void* phiK, const void* V, void* S, float* z);
-int grf_gather_contract(grf_ctx* ctx, const grf_csr_dev& phi, int32_t G, int32_t N, int32_t m, int32_t d, int dtype,
-                        const void* phiQ, const void* S, const float* z, void* out, float* den_out);
+int grf_gather_contract_alu(grf_ctx* ctx, const grf_csr_dev& phi, int32_t G, int32_t N, int32_t m, int32_t d,
+                            int dtype, const void* phiQ, const void* S, const float* z, void* out, float* den_out);
+// attn_gather_tc.cu
+int grf_build_block_plan(grf_ctx* ctx, grf_features* feat);
+int grf_gather_contract_tc(grf_ctx* ctx, const grf_features* feat, int32_t G, int32_t N, int32_t m, int32_t d,
+                           const void* phiQ, const void* S, const float* z, void* out, float* den_out);
+
+// Layout of one state tile S_l (m x d) inside the workspace: 16-byte chunks that hold CH consecutive feature
+// rows a of one column b, ordered [a / CH][b][a % CH].  With bf16 (CH = 8) this is the K-major, unswizzled
+// shared-memory operand layout of the tensor-core gather kernel (8-row core matrices of 128 contiguous
+// bytes), so a tile is brought in with one contiguous bulk copy; the ALU kernels read the same chunks.
+template <typename T> __host__ __device__ constexpr int grf_tile_chunk() { return 16 / (int)sizeof(T); }
+template <typename T> __host__ __device__ constexpr size_t grf_tile_index(int a, int b, int D)
+{
+    return ((size_t)(a / grf_tile_chunk<T>()) * D + b) * grf_tile_chunk<T>() + (a % grf_tile_chunk<T>());
+}
 
 static inline int grf_ceil_div(int64_t a, int64_t b) { return (int)((a + b - 1) / b); }

@@ -295,10 +295,11 @@ static int sample_into(grf_ctx* ctx, grf_features* feat, const grf_walk_params& 
     }
     GRF_CUDA_TRY(cudaGetLastError());
 
-    return grf_transpose_launch(ctx, N, N, nnz_psi, (const int32_t*)feat->psi.rowptr.ptr,
-                                (const int32_t*)feat->psi.col.ptr, (const float*)feat->psi.val.ptr,
-                                (int32_t*)feat->psit.rowptr.ptr, (int32_t*)feat->psit.col.ptr,
-                                (float*)feat->psit.val.ptr);
+    GRF_TRY(grf_transpose_launch(ctx, N, N, nnz_psi, (const int32_t*)feat->psi.rowptr.ptr,
+                                 (const int32_t*)feat->psi.col.ptr, (const float*)feat->psi.val.ptr,
+                                 (int32_t*)feat->psit.rowptr.ptr, (int32_t*)feat->psit.col.ptr,
+                                 (float*)feat->psit.val.ptr));
+    return grf_build_block_plan(ctx, feat);
 }
 
 extern "C" int grf_sample(grf_ctx* ctx, int32_t N, const int32_t* rowptr, const int32_t* col, const float* w,

@@ -70,13 +70,20 @@ def _attn_case(lib, w, g, G, f_phi=None, f_psi=None, ws_bytes=None):
         f_phi = oracle.deconvolve(w.alpha).astype(np.float32)
     feat = api.sample(ctx, api.DeviceGraph(g), configs.WALK_SEED, w.n_walks, w.p_halt, w.max_len, f_phi, f_psi)
     q, k, v = tensors.qkv(G, g.N, w.m, w.d, w.dtype, configs.QKV_SEED)
-    out, den = api.masked_linear_attn(ctx, feat, q.cuda(), k.cuda(), v.cuda(), want_den=True, workspace_bytes=ws_bytes)
-    torch.cuda.synchronize()
     Phi, Psi, PsiT, _, _ = helpers.oracle_features(w, g, configs.WALK_SEED, f_phi, f_psi)
     ref = oracle.attn_sparse(tensors.widen(q), tensors.widen(k), tensors.widen(v), Phi, PsiT)
-    helpers.assert_attn_close(out.float().cpu().numpy(), ref, helpers.TOL[w.dtype], den.cpu().numpy(), w.name)
+    outs = []
+    for tensor_cores in ((True, False) if w.dtype == "bf16" else (True,)):   # both gather kernels for bf16
+        B.grf_ctx_use_tensor_cores(ctx.handle, tensor_cores)
+        out, den = api.masked_linear_attn(ctx, feat, q.cuda(), k.cuda(), v.cuda(), want_den=True,
+                                          workspace_bytes=ws_bytes)
+        B.grf_ctx_check(ctx.handle)
+        helpers.assert_attn_close(out.float().cpu().numpy(), ref, helpers.TOL[w.dtype], den.cpu().numpy(),
+                                  f"{w.name} tensor_cores={tensor_cores}")
+        outs.append(out)
+    B.grf_ctx_use_tensor_cores(ctx.handle, True)
     feat.free()
-    return out
+    return outs[0]
 
 
 def test_attention_tiny_fp32(lib):
@@ -117,12 +124,12 @@ def test_attention_chunked_workspace_matches_single_pass(lib):
 
 
 @pytest.mark.parametrize("dtype", ["fp32", "bf16"])
-@pytest.mark.parametrize("m,d", [(8, 8), (16, 128), (128, 16), (64, 64), (32, 64), (128, 128)])
+@pytest.mark.parametrize("m,d", [(8, 8), (16, 128), (128, 16), (64, 64), (32, 64), (128, 128), (16, 16), (64, 32)])
 def test_attention_shapes_random_features(lib, m, d, dtype):
     """Rectangular (N x R), signed features: catches index or operand mix-ups for every tile shape."""
     api, B, ctx = lib
     rng = np.random.default_rng(m * 1000 + d)
-    N, R, G = 75, 41, 3
+    N, R, G = 331, 141, 3       # three query blocks of the tensor-core kernel, the last one ragged
 
     def rand_csr(rows, cols, per_row):
         rowptr = [0]; col = []; val = []
@@ -136,9 +143,14 @@ def test_attention_shapes_random_features(lib, m, d, dtype):
     PsiT = oracle.transpose(Psi)
     helpers.assert_csr_equal(feat.to_host(2), PsiT, "Psi^T", val_rtol=0)
     q, k, v = tensors.qkv(G, N, m, d, dtype, 5)
-    out, den = api.masked_linear_attn(ctx, feat, q.cuda(), k.cuda(), v.cuda(), want_den=True)
     ref = oracle.attn_sparse(tensors.widen(q), tensors.widen(k), tensors.widen(v), Phi, PsiT)
-    helpers.assert_attn_close(out.float().cpu().numpy(), ref, helpers.TOL[dtype], den.cpu().numpy(), f"m{m} d{d}", min_ok=0.5)
+    for tensor_cores in ((True, False) if dtype == "bf16" else (True,)):
+        B.grf_ctx_use_tensor_cores(ctx.handle, tensor_cores)
+        out, den = api.masked_linear_attn(ctx, feat, q.cuda(), k.cuda(), v.cuda(), want_den=True)
+        B.grf_ctx_check(ctx.handle)
+        helpers.assert_attn_close(out.float().cpu().numpy(), ref, helpers.TOL[dtype], den.cpu().numpy(),
+                                  f"m{m} d{d} tensor_cores={tensor_cores}", min_ok=0.5)
+    B.grf_ctx_use_tensor_cores(ctx.handle, True)
     feat.free()
 
 
