@@ -257,6 +257,8 @@ def run_ours(args):
                          "frac": achieved / peak_gbs, "peak_source": peak_kind, "traffic": None,
                          "ms_per_launch": dom_ms},
             "phases": {"sample_ms": statistics.mean(sample_ms), "attn_ms": statistics.mean(attn_ms),
+                       "sample_ms_min_med_max": [min(sample_ms), statistics.median(sample_ms), max(sample_ms)],
+                       "attn_ms_min_med_max": [min(attn_ms), statistics.median(attn_ms), max(attn_ms)],
                        "walks_per_s": 2 * N * w.n_walks / (statistics.mean(sample_ms) * 1e-3),
                        "attn_tokens_per_s": w.batch * N / (statistics.mean(attn_ms) * 1e-3),
                        "wall_s_timed_region": wall},

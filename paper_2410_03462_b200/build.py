@@ -13,7 +13,7 @@ SOURCES = ["api.cu", "sample.cu", "scan.cu", "transpose.cu", "attn_state.cu", "a
 
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-std=c++17", "-lineinfo",
-    "-Xcompiler", "-fPIC", "--fmad=true", "-I", INCLUDE, "-I", CSRC,
+    "-Xcompiler", "-fPIC", "--fmad=true", "-diag-suppress", "177", "-I", INCLUDE, "-I", CSRC,
 ]
 
 

@@ -60,7 +60,7 @@ extern "C" int grf_ctx_destroy(grf_ctx* ctx)
     cudaSetDevice(ctx->device);
     cudaStreamSynchronize(ctx->stream);
     grf_buf* bufs[] = {&ctx->stage_col, &ctx->stage_val, &ctx->counts, &ctx->rowptr2, &ctx->scan_blocks,
-                       &ctx->t_cursor, &ctx->t_tmp_col, &ctx->t_tmp_val, &ctx->h_rowptr, &ctx->h_col, &ctx->h_w,
+                       &ctx->t_cursor, &ctx->t_tmp_col, &ctx->t_tmp_val, &ctx->den_scratch, &ctx->h_rowptr, &ctx->h_col, &ctx->h_w,
                        &ctx->h_q, &ctx->h_k, &ctx->h_v, &ctx->h_out, &ctx->h_ws};
     for (grf_buf* b : bufs) grf_buf_release(b);
     if (ctx->h_feat) grf_features_free(ctx->h_feat);
@@ -244,10 +244,10 @@ static bool dim_ok(int32_t x) { return x == 8 || x == 16 || x == 32 || x == 64 |
 static size_t elem_size(int dtype) { return dtype == GRF_DTYPE_F32 ? 4 : 2; }
 static size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
 
-// per-problem workspace: S [R][m][d] in the storage type, then z [R][m] fp32, each 256-byte aligned
+// per-problem workspace: R records (state tile in the storage type, then z in fp32), 256-byte aligned
 static size_t ws_per_problem(int32_t R, int32_t m, int32_t d, int dtype)
 {
-    return align256((size_t)R * m * d * elem_size(dtype)) + align256((size_t)R * m * sizeof(float));
+    return align256((size_t)R * ((size_t)m * d * elem_size(dtype) + (size_t)m * sizeof(float)));
 }
 
 extern "C" size_t grf_attn_workspace_bytes(int32_t G, int32_t R, int32_t m, int32_t d, int dtype)
@@ -273,23 +273,19 @@ extern "C" int grf_masked_linear_attn(grf_ctx* ctx, const grf_features* feat, in
     if (chunk > G) chunk = G;
     if (chunk > 65535) chunk = 65535;
     const size_t es = elem_size(dtype);
-    const size_t s_bytes = align256((size_t)R * m * d * es);
     for (int64_t g0 = 0; g0 < G; g0 += chunk) {
         const int32_t gc = (int32_t)((G - g0) < chunk ? (G - g0) : chunk);
-        // chunk layout: S for gc problems (contiguous, [gc][R][m][d]) then z ([gc][R][m])
-        char* Sbuf = (char*)workspace;
-        float* zbuf = (float*)((char*)workspace + align256((size_t)gc * R * m * d * es));
-        (void)s_bytes;
+        // chunk layout: records [gc][R], contiguous
         const char* k_ptr = (const char*)phiK + (size_t)g0 * N * m * es;
         const char* v_ptr = (const char*)V + (size_t)g0 * N * d * es;
         const char* q_ptr = (const char*)phiQ + (size_t)g0 * N * m * es;
         char* o_ptr = (char*)out + (size_t)g0 * N * d * es;
         float* den_ptr = den_out ? den_out + (size_t)g0 * N : nullptr;
-        GRF_TRY(grf_build_states(ctx, feat->psit, gc, N, m, d, dtype, k_ptr, v_ptr, Sbuf, zbuf));
+        GRF_TRY(grf_build_states(ctx, feat->psit, gc, N, m, d, dtype, k_ptr, v_ptr, workspace));
         int rc = 1;
         if (dtype == GRF_DTYPE_BF16 && ctx->use_tensor_cores)
-            rc = grf_gather_contract_tc(ctx, feat, gc, N, m, d, q_ptr, Sbuf, zbuf, o_ptr, den_ptr);
-        if (rc > 0) rc = grf_gather_contract_alu(ctx, feat->phi, gc, N, m, d, dtype, q_ptr, Sbuf, zbuf, o_ptr, den_ptr);
+            rc = grf_gather_contract_tc(ctx, feat, gc, N, m, d, q_ptr, workspace, o_ptr, den_ptr);
+        if (rc > 0) rc = grf_gather_contract_alu(ctx, feat->phi, gc, N, m, d, dtype, q_ptr, workspace, o_ptr, den_ptr);
         GRF_TRY(rc);
     }
     return GRF_OK;

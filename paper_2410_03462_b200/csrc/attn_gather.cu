@@ -40,8 +40,8 @@ constexpr int GATHER_WARPS = 4;
 template <typename T, int M, int D>
 __global__ void __launch_bounds__(GATHER_WARPS * 32)
 gather_contract_kernel(int32_t N, int32_t R, const int32_t* __restrict__ rowptr, const int32_t* __restrict__ col,
-                       const float* __restrict__ val, const T* __restrict__ phiQ, const T* __restrict__ S,
-                       const float* __restrict__ z, T* __restrict__ out, float* __restrict__ den_out)
+                       const float* __restrict__ val, const T* __restrict__ phiQ,
+                       const unsigned char* __restrict__ records, T* __restrict__ out, float* __restrict__ den_out)
 {
     constexpr int CH = grf_tile_chunk<T>();
     constexpr int NCHUNK = (M / CH) * D;            // 16-byte chunks per tile, chunk x = (a / CH) * D + b
@@ -61,13 +61,13 @@ gather_contract_kernel(int32_t N, int32_t R, const int32_t* __restrict__ rowptr,
     for (int j = 0; j < NACC; ++j) acc[j] = 0.0f;
     float den = 0.0f;
 
-    const T* Sg = S + (size_t)g * R * M * D;
-    const float* zg = z + (size_t)g * R * M;
+    constexpr size_t REC = grf_record_bytes<T>(M, D);
+    const unsigned char* recs = records + (size_t)g * R * REC;
     for (int32_t p = rowptr[i]; p < rowptr[i + 1]; ++p) {
         const int32_t l = __ldg(col + p);
         const float phi = __ldg(val + p);
-        const T* tile = Sg + (size_t)l * M * D;
-        const float* zl = zg + (size_t)l * M;
+        const T* tile = reinterpret_cast<const T*>(recs + (size_t)l * REC);
+        const float* zl = reinterpret_cast<const float*>(recs + (size_t)l * REC + (size_t)M * D * sizeof(T));
 #pragma unroll
         for (int x0 = 0; x0 < NCHUNK; x0 += 32) {
             const int x = x0 + lane;
@@ -104,14 +104,14 @@ gather_contract_kernel(int32_t N, int32_t R, const int32_t* __restrict__ rowptr,
 
 template <typename T, int M>
 int launch_m(grf_ctx* ctx, const grf_csr_dev& phi, int32_t G, int32_t N, int32_t d,
-             const void* phiQ, const void* S, const float* z, void* out, float* den_out)
+             const void* phiQ, const void* records, void* out, float* den_out)
 {
     const dim3 grid(grf_ceil_div(N, GATHER_WARPS), G);
 #define GRF_GATHER_CASE(DD)                                                                                  \
     case DD:                                                                                                 \
         gather_contract_kernel<T, M, DD><<<grid, GATHER_WARPS * 32, 0, ctx->stream>>>(                       \
             N, phi.cols, (const int32_t*)phi.rowptr.ptr, (const int32_t*)phi.col.ptr,                        \
-            (const float*)phi.val.ptr, (const T*)phiQ, (const T*)S, z, (T*)out, den_out);                   \
+            (const float*)phi.val.ptr, (const T*)phiQ, (const unsigned char*)records, (T*)out, den_out);                   \
         break;
     {
         grf_launch_scope scope(ctx, 5);
@@ -126,14 +126,14 @@ int launch_m(grf_ctx* ctx, const grf_csr_dev& phi, int32_t G, int32_t N, int32_t
 
 template <typename T>
 int launch_t(grf_ctx* ctx, const grf_csr_dev& phi, int32_t G, int32_t N, int32_t m, int32_t d,
-             const void* phiQ, const void* S, const float* z, void* out, float* den_out)
+             const void* phiQ, const void* records, void* out, float* den_out)
 {
     switch (m) {
-        case 8: return launch_m<T, 8>(ctx, phi, G, N, d, phiQ, S, z, out, den_out);
-        case 16: return launch_m<T, 16>(ctx, phi, G, N, d, phiQ, S, z, out, den_out);
-        case 32: return launch_m<T, 32>(ctx, phi, G, N, d, phiQ, S, z, out, den_out);
-        case 64: return launch_m<T, 64>(ctx, phi, G, N, d, phiQ, S, z, out, den_out);
-        case 128: return launch_m<T, 128>(ctx, phi, G, N, d, phiQ, S, z, out, den_out);
+        case 8: return launch_m<T, 8>(ctx, phi, G, N, d, phiQ, records, out, den_out);
+        case 16: return launch_m<T, 16>(ctx, phi, G, N, d, phiQ, records, out, den_out);
+        case 32: return launch_m<T, 32>(ctx, phi, G, N, d, phiQ, records, out, den_out);
+        case 64: return launch_m<T, 64>(ctx, phi, G, N, d, phiQ, records, out, den_out);
+        case 128: return launch_m<T, 128>(ctx, phi, G, N, d, phiQ, records, out, den_out);
         default: return GRF_ERR_INVALID;
     }
 }
@@ -141,10 +141,10 @@ int launch_t(grf_ctx* ctx, const grf_csr_dev& phi, int32_t G, int32_t N, int32_t
 }  // namespace
 
 int grf_gather_contract_alu(grf_ctx* ctx, const grf_csr_dev& phi, int32_t G, int32_t N, int32_t m, int32_t d,
-                            int dtype, const void* phiQ, const void* S, const float* z, void* out, float* den_out)
+                            int dtype, const void* phiQ, const void* records, void* out, float* den_out)
 {
     if (G > 65535) return GRF_ERR_TOO_LARGE;
-    if (dtype == GRF_DTYPE_F32) return launch_t<float>(ctx, phi, G, N, m, d, phiQ, S, z, out, den_out);
-    if (dtype == GRF_DTYPE_BF16) return launch_t<__nv_bfloat16>(ctx, phi, G, N, m, d, phiQ, S, z, out, den_out);
+    if (dtype == GRF_DTYPE_F32) return launch_t<float>(ctx, phi, G, N, m, d, phiQ, records, out, den_out);
+    if (dtype == GRF_DTYPE_BF16) return launch_t<__nv_bfloat16>(ctx, phi, G, N, m, d, phiQ, records, out, den_out);
     return GRF_ERR_INVALID;
 }

@@ -3,12 +3,19 @@
 // A CTA owns a block of 128 consecutive queries of one problem g.  The block's rows of Phi touch a
 // union U of nodes l (the "block plan", a sorted list built once per feature object).  For every l in U
 //     D[128 x d] += A_l[128 x m] * S_l[m x d],      A_l[i, a] = Phi_il * phi(q_i)_a   (0 where Phi_il = 0)
-// is one or more tcgen05.mma instructions (M = 128, N = d, K = 16 each) accumulating in tensor memory:
-// the sum over l of Eq. 12 becomes the K dimension of one long matrix product, evaluated in a fixed order.
-//   - S_l arrives by one contiguous bulk async copy (the workspace stores tiles in operand layout),
-//   - A_l is produced by the 128 "row" threads, one query each, walking their own CSR row of Phi in step
-//     with the union list,
-//   - one thread issues the MMAs; completion is tracked with mbarriers, every wait is bounded.
+// is m/16 tcgen05.mma instructions (M = 128, N = d, K = 16) accumulating in tensor memory: the sum over l
+// of Eq. 12 becomes the K dimension of one long matrix product, evaluated in a fixed order.
+//   - the record of node l (S_l in operand layout, then z_l) arrives by one contiguous bulk async copy into
+//     a ring of shared-memory slots; records further ahead are prefetched into L2;
+//   - A_l lives in tensor memory: each of the 128 "row" threads owns one query (= one TMEM lane), walks its
+//     own CSR row of Phi in step with the union list and stores its scaled phi(q) (or zeros) with tcgen05.st;
+//     so the MMA reads only S_l from shared memory;
+//   - two warps issue the MMAs for alternate groups of union entries into two accumulators (one issuing
+//     thread cannot keep the tensor pipe busy with N = d this small); one tcgen05.commit per group frees both
+//     the A slots and the record slots of that group; the epilogue adds the two accumulators, divides by the
+//     denominators (accumulated by the row threads from z_l) and writes the block's outputs;
+//   - every mbarrier wait is bounded: a wait that outlasts its limit raises an error word and the CTA drains
+//     its copies and MMAs, frees its tensor memory and exits.
 // Nodes that no query of the block touches are never loaded; a tile is loaded once per block, not once
 // per query, which is where the method's "constant multiplicative cost" is paid down.
 #include "grf_internal.cuh"
@@ -16,8 +23,7 @@
 namespace {
 
 constexpr int BQ = GRF_PLAN_BLOCK;  // queries per CTA = MMA M
-constexpr int TC_THREADS = 192;     // warps 0-3: row threads / epilogue, warp 4: tile loader, warp 5: MMA issuer
-constexpr unsigned long long WAIT_NS = 2000000000ull;   // a wait that lasts longer than this gives up
+constexpr long long WAIT_CYCLES = 4000000000ll;   // a wait that lasts longer than this (about 2 s) gives up
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
@@ -43,22 +49,19 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
         : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
     return ok != 0;
 }
-__device__ __forceinline__ unsigned long long global_ns()
-{
-    unsigned long long t;
-    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
-    return t;
-}
 // Bounded wait: false when another thread of the CTA has given up or when this wait lasted too long
 // (then it raises the CTA's abort flag itself).
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag)
 {
-    if (mbar_try_wait(bar, parity)) return true;
-    const unsigned long long t0 = global_ns();
-    for (uint32_t it = 1;; ++it) {
+    long long t0 = 0;
+    for (uint32_t it = 0;; ++it) {
         if (mbar_try_wait(bar, parity)) return true;
-        if (*abort_flag) return false;
-        if ((it & 255u) == 0u && global_ns() - t0 > WAIT_NS) { *abort_flag = 1; return false; }
+        if ((it & 63u) == 63u) {
+            if (*abort_flag) return false;
+            const long long now = clock64();
+            if (t0 == 0) t0 = now;
+            else if (now - t0 > WAIT_CYCLES) { *abort_flag = 1; return false; }
+        }
     }
 }
 
@@ -85,15 +88,6 @@ __host__ __device__ constexpr uint32_t instr_desc_bf16(int n)
     return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
 }
 
-__device__ __forceinline__ void mma_bf16_ss(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
-                                            uint32_t accumulate)
-{
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-        ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
-}
 __device__ __forceinline__ void mma_commit(uint32_t bar)
 {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
@@ -109,44 +103,84 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16])
     asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 }
 
+__device__ __forceinline__ void tmem_st8(uint32_t taddr, const uint32_t (&r)[8])
+{
+    asm volatile("tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
+                 ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7])
+                 : "memory");
+}
+
+__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&r)[16])
+{
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};"
+        ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),
+          "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
+        : "memory");
+}
+
+// A operand in tensor memory (row i of the block = lane i, two bf16 per 32-bit column), B in shared memory
+__device__ __forceinline__ void mma_bf16_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t bdesc, uint32_t idesc,
+                                            uint32_t accumulate)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_tmem), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+}
+
+constexpr int pow2_at_least(int x) { return x <= 32 ? 32 : (x <= 64 ? 64 : (x <= 128 ? 128 : (x <= 256 ? 256 : 512))); }
+
 template <int M, int D> struct TcShape {
-    static constexpr int KC = M / 8;                          // 16-byte K chunks of one A row
-    static constexpr int A_BYTES = KC * BQ * 16;              // [chunk][row][16 B]
-    static constexpr int B_BYTES = M * D * 2;                 // one state tile
-    static constexpr int STAGE = A_BYTES + B_BYTES;
-    static constexpr int STAGES = (160 * 1024 / STAGE) >= 4 ? 4 : ((160 * 1024 / STAGE) >= 3 ? 3 : 2);
-    static constexpr int TMEM_COLS = D < 32 ? 32 : D;
-    static constexpr size_t SMEM = (size_t)STAGES * STAGE + 1024; // + alignment slack
+    static constexpr int A_COLS = M / 2;                      // TMEM columns of one union entry's A operand
+    static constexpr int GU = M <= 32 ? 4 : (M == 64 ? 2 : 1); // union entries per group (one commit per group)
+    static constexpr int NA = 2;                              // A stages (groups in flight on the row-thread side)
+    static constexpr int TMEM_COLS = pow2_at_least(2 * D + NA * GU * A_COLS);   // two accumulators + A ring
+    static constexpr int TILE_BYTES = M * D * 2;
+    static constexpr int REC_BYTES = TILE_BYTES + M * 4;      // state tile followed by z
+    static constexpr int CHUNK_BYTES = GU * REC_BYTES;
+    static constexpr int SMEM_BUDGET = TMEM_COLS <= 256 ? 104 * 1024 : 200 * 1024;   // two CTAs per SM, or one
+    static constexpr int NBC_WANT = SMEM_BUDGET / CHUNK_BYTES;
+    static constexpr int NBC = NBC_WANT > 8 ? 8 : (NBC_WANT < 2 ? 2 : NBC_WANT);     // record chunks in flight
+    static constexpr size_t SMEM = (size_t)NBC * CHUNK_BYTES + 1024;                  // + alignment slack
 };
+
+// warps 0-3: row threads (A operand, denominators, epilogue); warp 4: record loader; warps 5, 6: MMA issuers
+constexpr int TC_THREADS = 224;
 
 template <int M, int D>
 __global__ void __launch_bounds__(TC_THREADS)
 gather_contract_tc_kernel(int32_t N, int32_t R, const int32_t* __restrict__ rowptr, const int32_t* __restrict__ col,
                           const float* __restrict__ val, const int32_t* __restrict__ plan_off,
                           const int32_t* __restrict__ plan_cnt, const int32_t* __restrict__ plan_col,
-                          const __nv_bfloat16* __restrict__ phiQ, const __nv_bfloat16* __restrict__ S,
-                          const float* __restrict__ z, __nv_bfloat16* __restrict__ out, float* __restrict__ den_out,
-                          int* __restrict__ error_word)
+                          const __nv_bfloat16* __restrict__ phiQ, const unsigned char* __restrict__ records,
+                          __nv_bfloat16* __restrict__ out, const float* __restrict__ den_in, int* __restrict__ error_word)
 {
     using Sh = TcShape<M, D>;
-    constexpr int NS = Sh::STAGES;
+    constexpr int NA = Sh::NA, NBC = Sh::NBC, GU = Sh::GU, NREC = NBC * GU;
     extern __shared__ unsigned char smem_dyn[];
-    __shared__ __align__(8) unsigned long long bars[3 * NS + 1];   // a_full, b_full, empty per stage; acc_done
+    // a_full per A stage; rec_full per record slot; done per record chunk (= per group); acc_done per issuer
+    __shared__ __align__(8) unsigned long long bars[NA + NREC + NBC + 2];
     __shared__ uint32_t tmem_slot;
     __shared__ int abort_flag;
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int32_t blk = blockIdx.x, g = blockIdx.y;
-    const uint32_t stage_base = (smem_u32(smem_dyn) + 1023u) & ~1023u;
+    const uint32_t b_base = (smem_u32(smem_dyn) + 1023u) & ~1023u;
+    const unsigned char* b_generic = smem_dyn + (b_base - smem_u32(smem_dyn));
     const uint32_t bar_base = smem_u32(bars);
     auto a_full = [&](int s) { return bar_base + 8u * (uint32_t)s; };
-    auto b_full = [&](int s) { return bar_base + 8u * (uint32_t)(NS + s); };
-    auto empty = [&](int s) { return bar_base + 8u * (uint32_t)(2 * NS + s); };
-    const uint32_t acc_done = bar_base + 8u * (uint32_t)(3 * NS);
+    auto rec_full = [&](int s) { return bar_base + 8u * (uint32_t)(NA + s); };
+    auto done = [&](int s) { return bar_base + 8u * (uint32_t)(NA + NREC + s); };
+    auto acc_done = [&](int w) { return bar_base + 8u * (uint32_t)(NA + NREC + NBC + w); };
 
     if (tid == 0) {
-        for (int s = 0; s < NS; ++s) { mbar_init(a_full(s), BQ); mbar_init(b_full(s), 1); mbar_init(empty(s), 1); }
-        mbar_init(acc_done, 1);
+        for (int s = 0; s < NA; ++s) mbar_init(a_full(s), 4);
+        for (int s = 0; s < NREC; ++s) mbar_init(rec_full(s), 1);
+        for (int s = 0; s < NBC; ++s) mbar_init(done(s), 1);
+        mbar_init(acc_done(0), 1);
+        mbar_init(acc_done(1), 1);
         abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -158,14 +192,16 @@ gather_contract_tc_kernel(int32_t N, int32_t R, const int32_t* __restrict__ rowp
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-    const uint32_t tmem_acc = tmem_slot;
+    const uint32_t tmem_base = tmem_slot;
+    const uint32_t tmem_a = tmem_base + 2u * D;     // A ring behind the two accumulators
 
     const int32_t cnt = plan_cnt[blk];
+    const int32_t ngroups = (cnt + GU - 1) / GU;
     const int32_t* ulist = plan_col + plan_off[blk];
-    const __nv_bfloat16* Sg = S + (size_t)g * R * M * D;
+    const unsigned char* recs = records + (size_t)g * R * Sh::REC_BYTES;
 
     if (warp < 4) {
-        // ------------------------------------------------------------ row threads: build A, then epilogue
+        // ------------------------------------------------------------ row threads: A operand, denominators, epilogue
         const int32_t row = blk * BQ + tid;
         const bool live = row < N;
         uint32_t q2[M / 2];
@@ -180,81 +216,89 @@ gather_contract_tc_kernel(int32_t N, int32_t R, const int32_t* __restrict__ rowp
 #pragma unroll
             for (int c = 0; c < M / 2; ++c) q2[c] = 0u;
         }
+        // this row's non-zeros of Phi, walked in step with the union list; two entries are kept ahead
         int32_t p = live ? rowptr[row] : 0;
         const int32_t pend = live ? rowptr[row + 1] : 0;
-        int32_t next_col = p < pend ? __ldg(col + p) : -1;
-        float next_val = p < pend ? __ldg(val + p) : 0.0f;
-        const float* zg = z + (size_t)g * R * M;
-        float den = 0.0f;
+        int32_t col0 = p < pend ? __ldg(col + p) : -1, col1 = p + 1 < pend ? __ldg(col + p + 1) : -1;
+        float val0 = p < pend ? __ldg(val + p) : 0.0f, val1 = p + 1 < pend ? __ldg(val + p + 1) : 0.0f;
+        const float den = live ? den_in[(size_t)g * N + row] : 0.0f;
         bool ok = true;
-        for (int32_t u = 0; u < cnt; ++u) {
-            const int s = u % NS;
-            const uint32_t ph = (uint32_t)(u / NS) & 1u;
-            if (!mbar_wait(empty(s), ph ^ 1u, &abort_flag)) { ok = false; break; }
-            const int32_t l = __ldg(ulist + u);
-            float coef = 0.0f;
-            if (next_col == l) {
-                coef = next_val;
-                ++p;
-                next_col = p < pend ? __ldg(col + p) : -1;
-                next_val = p < pend ? __ldg(val + p) : 0.0f;
-            }
-            const uint32_t a_stage = stage_base + (uint32_t)s * Sh::STAGE;
-            if (coef != 0.0f) {
-                const float4* zl = reinterpret_cast<const float4*>(zg + (size_t)l * M);
-                float dot = 0.0f;
+        int32_t l_mine = -1;
+        const uint32_t lane_field = (uint32_t)(warp * 32) << 16;
+        for (int32_t gi = 0; gi < ngroups; ++gi) {
+            const int32_t u0 = gi * GU;
+            if ((u0 & 31) == 0) l_mine = (u0 + lane < cnt) ? __ldg(ulist + u0 + lane) : -1;   // GU divides 32
+            const int st = gi % NA;
+            // the A slots of this stage are free once the group that used them NA groups ago has been multiplied
+            if (gi >= NA && !mbar_wait(done((gi - NA) % NBC), (uint32_t)((gi - NA) / NBC) & 1u, &abort_flag)) ok = false;
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
 #pragma unroll
-                for (int c = 0; c < M / 4; ++c) {
-                    const float4 zz = __ldg(zl + c);
-                    dot = fmaf(__uint_as_float(q2[2 * c] << 16), zz.x, dot);
-                    dot = fmaf(__uint_as_float(q2[2 * c] & 0xffff0000u), zz.y, dot);
-                    dot = fmaf(__uint_as_float(q2[2 * c + 1] << 16), zz.z, dot);
-                    dot = fmaf(__uint_as_float(q2[2 * c + 1] & 0xffff0000u), zz.w, dot);
-                }
-                den = fmaf(coef, dot, den);
+            for (int j = 0; j < GU; ++j) {
+                const int32_t u = u0 + j;
+                const int32_t l = __shfl_sync(0xffffffffu, l_mine, u & 31);   // -1 beyond the list: matches nothing
+                // A_l[row, :] = Phi_il * phi(q_row): zeros for most rows; products are taken in packed bf16
+                uint32_t w[M / 2];
+                if (l >= 0 && col0 == l) {
+                    const __nv_bfloat162 c2 = __float2bfloat162_rn(val0);
+                    ++p;
+                    col0 = col1; val0 = val1;
+                    col1 = p + 1 < pend ? __ldg(col + p + 1) : -1;
+                    val1 = p + 1 < pend ? __ldg(val + p + 1) : 0.0f;
 #pragma unroll
-                for (int c = 0; c < M / 8; ++c) {
-                    uint32_t w[4];
-#pragma unroll
-                    for (int e = 0; e < 4; ++e) {
-                        const float lo = coef * __uint_as_float(q2[4 * c + e] << 16);
-                        const float hi = coef * __uint_as_float(q2[4 * c + e] & 0xffff0000u);
-                        __nv_bfloat162 h = __floats2bfloat162_rn(lo, hi);
-                        w[e] = *reinterpret_cast<uint32_t*>(&h);
+                    for (int e = 0; e < M / 2; ++e) {
+                        const __nv_bfloat162 h = __hmul2(*reinterpret_cast<const __nv_bfloat162*>(&q2[e]), c2);
+                        w[e] = *reinterpret_cast<const uint32_t*>(&h);
                     }
-                    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};"
-                                 ::"r"(a_stage + (uint32_t)c * (BQ * 16) + (uint32_t)tid * 16),
-                                   "r"(w[0]), "r"(w[1]), "r"(w[2]), "r"(w[3]) : "memory");
-                }
-            } else {
+                } else {
 #pragma unroll
-                for (int c = 0; c < M / 8; ++c)
-                    asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};"
-                                 ::"r"(a_stage + (uint32_t)c * (BQ * 16) + (uint32_t)tid * 16), "r"(0u) : "memory");
+                    for (int e = 0; e < M / 2; ++e) w[e] = 0u;
+                }
+                __syncwarp();
+                const uint32_t a_slot = tmem_a + lane_field + (uint32_t)((st * GU + j) * Sh::A_COLS);
+                if constexpr (M >= 32) {
+#pragma unroll
+                    for (int c = 0; c < M / 32; ++c) {
+                        uint32_t w16[16];
+#pragma unroll
+                        for (int e = 0; e < 16; ++e) w16[e] = w[16 * c + e];
+                        tmem_st16(a_slot + (uint32_t)c * 16u, w16);
+                    }
+                } else {
+                    uint32_t w8[8];
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) w8[e] = w[e];
+                    tmem_st8(a_slot, w8);
+                }
             }
-            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-            mbar_arrive(a_full(s));
+            asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+            asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+            __syncwarp();
+            if (lane == 0) mbar_arrive(a_full(st));
         }
-        // epilogue: this thread's row of the accumulator is TMEM lane `tid`
-        if (ok && cnt > 0) ok = mbar_wait(acc_done, 0u, &abort_flag);
+        // epilogue: this thread's row of the accumulators is TMEM lane `tid`; the two issuers' partial sums are
+        // added in a fixed order
+        if (ok && ngroups > 0) ok = mbar_wait(acc_done(0), 0u, &abort_flag);
+        if (ok && ngroups > 1) ok = mbar_wait(acc_done(1), 0u, &abort_flag);
         ok = __all_sync(0xffffffffu, ok);   // the tensor-memory loads below are warp-wide
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         const float inv = (den != 0.0f) ? 1.0f / den : 0.0f;
         __nv_bfloat16* orow = out + ((size_t)g * N + row) * D;
 #pragma unroll
         for (int c0 = 0; c0 < D; c0 += 16) {
-            uint32_t r[16];
-            if (ok && cnt > 0) {
-                tmem_ld16(tmem_acc + ((uint32_t)(warp * 32) << 16) + (uint32_t)c0, r);
-            } else {
+            uint32_t r[16], r1[16];
 #pragma unroll
-                for (int e = 0; e < 16; ++e) r[e] = 0u;
-            }
+            for (int e = 0; e < 16; ++e) { r[e] = 0u; r1[e] = 0u; }
+            if (ok && ngroups > 0) tmem_ld16(tmem_base + lane_field + (uint32_t)c0, r);
+            if (ok && ngroups > 1) tmem_ld16(tmem_base + lane_field + (uint32_t)(D + c0), r1);
             if (live && ok) {
                 uint32_t w[8];
 #pragma unroll
                 for (int e = 0; e < 8; ++e) {
-                    __nv_bfloat162 h = __floats2bfloat162_rn(__uint_as_float(r[2 * e]) * inv, __uint_as_float(r[2 * e + 1]) * inv);
+                    const float x0 = (__uint_as_float(r[2 * e]) + __uint_as_float(r1[2 * e])) * inv;
+                    const float x1 = (__uint_as_float(r[2 * e + 1]) + __uint_as_float(r1[2 * e + 1])) * inv;
+                    __nv_bfloat162 h = __floats2bfloat162_rn(x0, x1);
                     w[e] = *reinterpret_cast<uint32_t*>(&h);
                 }
                 uint4* dst = reinterpret_cast<uint4*>(orow + c0);
@@ -262,68 +306,125 @@ gather_contract_tc_kernel(int32_t N, int32_t R, const int32_t* __restrict__ rowp
                 dst[1] = make_uint4(w[4], w[5], w[6], w[7]);
             }
         }
-        if (live && ok && den_out) den_out[(size_t)g * N + row] = den;
     } else if (warp == 4) {
-        // ------------------------------------------------------------ tile loader
+        // ------------------------------------------------------------ record loader (runs NBC chunks ahead)
         int32_t issued = 0;
-        for (int32_t u = 0; u < cnt; ++u) {
-            const int s = u % NS;
-            const uint32_t ph = (uint32_t)(u / NS) & 1u;
-            if (!mbar_wait(empty(s), ph ^ 1u, &abort_flag)) break;
+        for (int32_t gi = 0; gi < ngroups; ++gi) {
+            if (gi >= NBC && !mbar_wait(done(gi % NBC), (uint32_t)((gi - NBC) / NBC) & 1u, &abort_flag)) break;
+            const int32_t uend = min(cnt, (gi + 1) * GU);
             if (lane == 0) {
-                const int32_t l = __ldg(ulist + u);
-                mbar_arrive_expect_tx(b_full(s), Sh::B_BYTES);
-                bulk_copy_g2s(stage_base + (uint32_t)s * Sh::STAGE + Sh::A_BYTES, Sg + (size_t)l * M * D, Sh::B_BYTES,
-                              b_full(s));
+                for (int32_t u = gi * GU; u < uend; ++u) {
+                    // records further down the list are pulled into L2 ahead of their turn
+                    if (u + 2 * NREC < cnt)
+                        asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;"
+                                     ::"l"(recs + (size_t)__ldg(ulist + u + 2 * NREC) * Sh::REC_BYTES), "r"((uint32_t)Sh::REC_BYTES)
+                                     : "memory");
+                    const int s = u % NREC;
+                    const int32_t l = __ldg(ulist + u);
+                    mbar_arrive_expect_tx(rec_full(s), Sh::REC_BYTES);
+                    bulk_copy_g2s(b_base + (uint32_t)s * Sh::REC_BYTES, recs + (size_t)l * Sh::REC_BYTES, Sh::REC_BYTES, rec_full(s));
+                }
             }
-            ++issued;
+            issued = uend;
             __syncwarp();
         }
         if (abort_flag) {
             // gave up somewhere: let the copies that are still in flight land before the CTA exits
-            const int32_t first = issued > NS ? issued - NS : 0;
+            const int32_t first = issued > NREC ? issued - NREC : 0;
             for (int32_t u = first; u < issued; ++u) {
-                const unsigned long long t0 = global_ns();
-                while (!mbar_try_wait(b_full(u % NS), (uint32_t)(u / NS) & 1u) && global_ns() - t0 < WAIT_NS) {}
+                const long long t0 = clock64();
+                while (!mbar_try_wait(rec_full(u % NREC), (uint32_t)(u / NREC) & 1u) && clock64() - t0 < WAIT_CYCLES) {}
             }
         }
     } else {
-        // ------------------------------------------------------------ MMA issuer
+        // ------------------------------------------------------------ MMA issuers: warp 5 takes even groups, warp 6 odd
+        const int w = warp - 5;
         constexpr uint32_t idesc = instr_desc_bf16(D);
+        const uint32_t acc = tmem_base + (uint32_t)(w * D);
         bool ok = true;
-        for (int32_t u = 0; u < cnt; ++u) {
-            const int s = u % NS;
-            const uint32_t ph = (uint32_t)(u / NS) & 1u;
-            if (!mbar_wait(a_full(s), ph, &abort_flag) || !mbar_wait(b_full(s), ph, &abort_flag)) { ok = false; break; }
-            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-            if (lane == 0) {
-                const uint32_t a_stage = stage_base + (uint32_t)s * Sh::STAGE;
-                const uint32_t b_stage = a_stage + Sh::A_BYTES;
+        bool first = true;
+        for (int32_t gi = w; gi < ngroups && ok; gi += 2) {
+            const int st = gi % NA;
+            if (!mbar_wait(a_full(st), (uint32_t)(gi / NA) & 1u, &abort_flag)) { ok = false; break; }
+            const int32_t uend = min(cnt, (gi + 1) * GU);
+            for (int32_t u = gi * GU; u < uend; ++u) {
+                const int sr = u % NREC;
+                if (!mbar_wait(rec_full(sr), (uint32_t)(u / NREC) & 1u, &abort_flag)) { ok = false; break; }
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                if (lane == 0) {
+                    const uint32_t a_op = tmem_a + (uint32_t)((st * GU + (u - gi * GU)) * Sh::A_COLS);
+                    const uint32_t b_op = b_base + (uint32_t)sr * Sh::REC_BYTES;
 #pragma unroll
-                for (int k = 0; k < M / 16; ++k) {
-                    const uint64_t ad = operand_desc(a_stage + (uint32_t)k * 2u * (BQ * 16), BQ * 16, 128);
-                    const uint64_t bd = operand_desc(b_stage + (uint32_t)k * 2u * (D * 16), D * 16, 128);
-                    mma_bf16_ss(tmem_acc, ad, bd, idesc, (u > 0 || k > 0) ? 1u : 0u);
+                    for (int k = 0; k < M / 16; ++k) {
+                        const uint64_t bd = operand_desc(b_op + (uint32_t)k * 2u * (D * 16), D * 16, 128);
+                        mma_bf16_ts(acc, a_op + (uint32_t)k * 8u, bd, idesc, (first && k == 0) ? 0u : 1u);
+                    }
                 }
-                mma_commit(empty(s));
+                first = false;
+                __syncwarp();
             }
+            if (lane == 0 && ok) mma_commit(done(gi % NBC));
             __syncwarp();
         }
-        if (lane == 0 && cnt > 0) mma_commit(acc_done);
+        if (lane == 0 && ngroups > w) mma_commit(acc_done(w));
         __syncwarp();
-        if (!ok && cnt > 0) {
+        if (!ok && ngroups > w) {
             // aborted: wait (bounded) until the MMAs already issued have drained before the CTA exits
-            const unsigned long long t0 = global_ns();
-            while (!mbar_try_wait(acc_done, 0u) && global_ns() - t0 < WAIT_NS) {}
+            const long long t0 = clock64();
+            while (!mbar_try_wait(acc_done(w), 0u) && clock64() - t0 < WAIT_CYCLES) {}
         }
     }
 
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
     if (warp == 5) {
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_acc), "r"((uint32_t)Sh::TMEM_COLS) : "memory");
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)Sh::TMEM_COLS) : "memory");
     }
     if (tid == 0 && abort_flag) atomicExch(error_word, 1);
+}
+
+// ---------------------------------------------------------------------------------------------------
+// Denominators of Eq. 12 for the tensor-core path: den_i = phi(q_i) . (sum_l Phi_il z_l), one warp per
+// (problem, query), lanes across the m feature components, z_l read coalesced from the records.
+
+template <int M, int D>
+__global__ void __launch_bounds__(256)
+row_denominators_kernel(int32_t N, int32_t R, const int32_t* __restrict__ rowptr, const int32_t* __restrict__ col,
+                        const float* __restrict__ val, const __nv_bfloat16* __restrict__ phiQ,
+                        const unsigned char* __restrict__ records, float* __restrict__ den)
+{
+    constexpr int MA = (M + 31) / 32;                       // feature components per lane
+    constexpr size_t REC = (size_t)M * D * 2 + (size_t)M * 4;
+    const int lane = threadIdx.x & 31;
+    const int32_t i = blockIdx.x * 8 + (threadIdx.x >> 5);
+    const int32_t g = blockIdx.y;
+    if (i >= N) return;
+    const unsigned char* zbase = records + (size_t)g * R * REC + (size_t)M * D * 2;
+    float zbar[MA];
+#pragma unroll
+    for (int t = 0; t < MA; ++t) zbar[t] = 0.0f;
+    const int32_t beg = rowptr[i], end = rowptr[i + 1];
+    for (int32_t p0 = beg; p0 < end; p0 += 32) {
+        const int32_t n = min(32, end - p0);
+        const int32_t c_mine = lane < n ? __ldg(col + p0 + lane) : 0;
+        const float v_mine = lane < n ? __ldg(val + p0 + lane) : 0.0f;
+        for (int32_t j = 0; j < n; ++j) {
+            const int32_t l = __shfl_sync(0xffffffffu, c_mine, j);
+            const float phi = __shfl_sync(0xffffffffu, v_mine, j);
+            const float* zl = reinterpret_cast<const float*>(zbase + (size_t)l * REC);
+#pragma unroll
+            for (int t = 0; t < MA; ++t)
+                if (M >= 32 || lane < M) zbar[t] = fmaf(phi, __ldg(zl + lane + 32 * t), zbar[t]);
+        }
+    }
+    const __nv_bfloat16* q = phiQ + ((size_t)g * N + i) * M;
+    float d = 0.0f;
+#pragma unroll
+    for (int t = 0; t < MA; ++t)
+        if (M >= 32 || lane < M) d = fmaf(__bfloat162float(q[lane + 32 * t]), zbar[t], d);
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) d += __shfl_xor_sync(0xffffffffu, d, off);
+    if (lane == 0) den[(size_t)g * N + i] = d;
 }
 
 // ---------------------------------------------------------------------------------------------------
@@ -411,30 +512,41 @@ int grf_build_block_plan(grf_ctx* ctx, grf_features* feat)
 
 template <int M, int D>
 static int launch_tc(grf_ctx* ctx, const grf_features* feat, int32_t G, int32_t N,
-                     const void* phiQ, const void* S, const float* z, void* out, float* den_out)
+                     const void* phiQ, const void* records, void* out, float* den_out)
 {
     using Sh = TcShape<M, D>;
     const grf_csr_dev& phi = feat->phi;
     GRF_CUDA_TRY(cudaFuncSetAttribute(gather_contract_tc_kernel<M, D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                       (int)Sh::SMEM));
+    float* den = den_out;
+    if (!den) {
+        GRF_TRY(grf_buf_reserve(&ctx->den_scratch, sizeof(float) * (size_t)G * N));
+        den = (float*)ctx->den_scratch.ptr;
+    }
+    {
+        grf_launch_scope scope(ctx, 5);
+        row_denominators_kernel<M, D><<<dim3(grf_ceil_div(N, 8), G), 256, 0, ctx->stream>>>(
+            N, phi.cols, (const int32_t*)phi.rowptr.ptr, (const int32_t*)phi.col.ptr, (const float*)phi.val.ptr,
+            (const __nv_bfloat16*)phiQ, (const unsigned char*)records, den);
+    }
     const dim3 grid(feat->plan_blocks, G);
     {
         grf_launch_scope scope(ctx, 5);
         gather_contract_tc_kernel<M, D><<<grid, TC_THREADS, Sh::SMEM, ctx->stream>>>(
             N, phi.cols, (const int32_t*)phi.rowptr.ptr, (const int32_t*)phi.col.ptr, (const float*)phi.val.ptr,
             (const int32_t*)feat->plan_off.ptr, (const int32_t*)feat->plan_cnt.ptr, (const int32_t*)feat->plan_col.ptr,
-            (const __nv_bfloat16*)phiQ, (const __nv_bfloat16*)S, z, (__nv_bfloat16*)out, den_out, ctx->error_word);
+            (const __nv_bfloat16*)phiQ, (const unsigned char*)records, (__nv_bfloat16*)out, den, ctx->error_word);
     }
     return cudaGetLastError() == cudaSuccess ? GRF_OK : GRF_ERR_CUDA;
 }
 
 // Returns GRF_OK after launching, or 1 when this shape/object has no tensor-core path (caller falls back).
 int grf_gather_contract_tc(grf_ctx* ctx, const grf_features* feat, int32_t G, int32_t N, int32_t m, int32_t d,
-                           const void* phiQ, const void* S, const float* z, void* out, float* den_out)
+                           const void* phiQ, const void* records, void* out, float* den_out)
 {
     if (!feat->plan_ready || G > 65535) return 1;
 #define GRF_TC_CASE(MM, DD) \
-    if (m == MM && d == DD) return launch_tc<MM, DD>(ctx, feat, G, N, phiQ, S, z, out, den_out);
+    if (m == MM && d == DD) return launch_tc<MM, DD>(ctx, feat, G, N, phiQ, records, out, den_out);
     GRF_TC_CASE(16, 16) GRF_TC_CASE(16, 32) GRF_TC_CASE(16, 64) GRF_TC_CASE(16, 128)
     GRF_TC_CASE(32, 16) GRF_TC_CASE(32, 32) GRF_TC_CASE(32, 64) GRF_TC_CASE(32, 128)
     GRF_TC_CASE(64, 16) GRF_TC_CASE(64, 32) GRF_TC_CASE(64, 64) GRF_TC_CASE(64, 128)

@@ -44,7 +44,7 @@ template <typename T, int M, int D>
 __global__ void __launch_bounds__(StateTiling<T, M, D>::THREADS)
 build_states_kernel(int32_t R, int32_t N, const int32_t* __restrict__ t_rowptr, const int32_t* __restrict__ t_col,
                     const float* __restrict__ t_val, const T* __restrict__ phiK, const T* __restrict__ V,
-                    T* __restrict__ S, float* __restrict__ z)
+                    unsigned char* __restrict__ records)
 {
     using Tl = StateTiling<T, M, D>;
     constexpr int CH = Tl::CH, TXB = Tl::TXB, TB = Tl::TB, JC = Tl::JC, THREADS = Tl::THREADS;
@@ -96,11 +96,12 @@ build_states_kernel(int32_t R, int32_t N, const int32_t* __restrict__ t_rowptr, 
         __syncthreads();
     }
 
-    T* Sl = S + ((size_t)g * R + l) * M * D;
+    unsigned char* rec = records + ((size_t)g * R + l) * grf_record_bytes<T>(M, D);
+    T* Sl = reinterpret_cast<T*>(rec);
 #pragma unroll
     for (int t = 0; t < TB; ++t) store_chunk(Sl + grf_tile_index<T>(kc * CH, bx + t * TXB, D), acc[t]);
     if (bx == 0) {
-        float* zl = z + ((size_t)g * R + l) * M;
+        float* zl = reinterpret_cast<float*>(rec + (size_t)M * D * sizeof(T));
 #pragma unroll
         for (int c = 0; c < CH; ++c) zl[kc * CH + c] = zacc[c];
     }
@@ -108,14 +109,14 @@ build_states_kernel(int32_t R, int32_t N, const int32_t* __restrict__ t_rowptr, 
 
 template <typename T, int M>
 int launch_m(grf_ctx* ctx, const grf_csr_dev& psit, int32_t G, int32_t N, int32_t d,
-             const void* phiK, const void* V, void* S, float* z)
+             const void* phiK, const void* V, void* records)
 {
     const dim3 grid(psit.rows, G);
 #define GRF_STATE_CASE(DD)                                                                                  \
     case DD:                                                                                                \
         build_states_kernel<T, M, DD><<<grid, StateTiling<T, M, DD>::THREADS, 0, ctx->stream>>>(            \
             psit.rows, N, (const int32_t*)psit.rowptr.ptr, (const int32_t*)psit.col.ptr,                    \
-            (const float*)psit.val.ptr, (const T*)phiK, (const T*)V, (T*)S, z);                            \
+            (const float*)psit.val.ptr, (const T*)phiK, (const T*)V, (unsigned char*)records);                            \
         break;
     {
         grf_launch_scope scope(ctx, 4);
@@ -130,14 +131,14 @@ int launch_m(grf_ctx* ctx, const grf_csr_dev& psit, int32_t G, int32_t N, int32_
 
 template <typename T>
 int launch_t(grf_ctx* ctx, const grf_csr_dev& psit, int32_t G, int32_t N, int32_t m, int32_t d,
-             const void* phiK, const void* V, void* S, float* z)
+             const void* phiK, const void* V, void* records)
 {
     switch (m) {
-        case 8: return launch_m<T, 8>(ctx, psit, G, N, d, phiK, V, S, z);
-        case 16: return launch_m<T, 16>(ctx, psit, G, N, d, phiK, V, S, z);
-        case 32: return launch_m<T, 32>(ctx, psit, G, N, d, phiK, V, S, z);
-        case 64: return launch_m<T, 64>(ctx, psit, G, N, d, phiK, V, S, z);
-        case 128: return launch_m<T, 128>(ctx, psit, G, N, d, phiK, V, S, z);
+        case 8: return launch_m<T, 8>(ctx, psit, G, N, d, phiK, V, records);
+        case 16: return launch_m<T, 16>(ctx, psit, G, N, d, phiK, V, records);
+        case 32: return launch_m<T, 32>(ctx, psit, G, N, d, phiK, V, records);
+        case 64: return launch_m<T, 64>(ctx, psit, G, N, d, phiK, V, records);
+        case 128: return launch_m<T, 128>(ctx, psit, G, N, d, phiK, V, records);
         default: return GRF_ERR_INVALID;
     }
 }
@@ -145,10 +146,10 @@ int launch_t(grf_ctx* ctx, const grf_csr_dev& psit, int32_t G, int32_t N, int32_
 }  // namespace
 
 int grf_build_states(grf_ctx* ctx, const grf_csr_dev& psit, int32_t G, int32_t N, int32_t m, int32_t d, int dtype,
-                     const void* phiK, const void* V, void* S, float* z)
+                     const void* phiK, const void* V, void* records)
 {
     if (G > 65535) return GRF_ERR_TOO_LARGE;
-    if (dtype == GRF_DTYPE_F32) return launch_t<float>(ctx, psit, G, N, m, d, phiK, V, S, z);
-    if (dtype == GRF_DTYPE_BF16) return launch_t<__nv_bfloat16>(ctx, psit, G, N, m, d, phiK, V, S, z);
+    if (dtype == GRF_DTYPE_F32) return launch_t<float>(ctx, psit, G, N, m, d, phiK, V, records);
+    if (dtype == GRF_DTYPE_BF16) return launch_t<__nv_bfloat16>(ctx, psit, G, N, m, d, phiK, V, records);
     return GRF_ERR_INVALID;
 }

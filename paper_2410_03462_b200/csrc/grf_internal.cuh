@@ -39,6 +39,7 @@ struct grf_ctx {
     grf_buf scan_blocks;            // block totals of the two-level scan
     // transpose scratch
     grf_buf t_cursor, t_tmp_col, t_tmp_val;
+    grf_buf den_scratch;            // denominators of the tensor-core gather path when the caller wants none
     // host-buffer path
     grf_buf h_rowptr, h_col, h_w, h_q, h_k, h_v, h_out, h_ws;
     grf_features* h_feat = nullptr;
@@ -109,13 +110,13 @@ int grf_transpose_launch(grf_ctx* ctx, int32_t rows, int32_t cols, int64_t nnz,
 
 // attn_state.cu / attn_gather.cu
 int grf_build_states(grf_ctx* ctx, const grf_csr_dev& psit, int32_t G, int32_t N, int32_t m, int32_t d, int dtype,
-                     const void* phiK, const void* V, void* S, float* z);
+                     const void* phiK, const void* V, void* records);
 int grf_gather_contract_alu(grf_ctx* ctx, const grf_csr_dev& phi, int32_t G, int32_t N, int32_t m, int32_t d,
-                            int dtype, const void* phiQ, const void* S, const float* z, void* out, float* den_out);
+                            int dtype, const void* phiQ, const void* records, void* out, float* den_out);
 // attn_gather_tc.cu
 int grf_build_block_plan(grf_ctx* ctx, grf_features* feat);
 int grf_gather_contract_tc(grf_ctx* ctx, const grf_features* feat, int32_t G, int32_t N, int32_t m, int32_t d,
-                           const void* phiQ, const void* S, const float* z, void* out, float* den_out);
+                           const void* phiQ, const void* records, void* out, float* den_out);
 
 // Layout of one state tile S_l (m x d) inside the workspace: 16-byte chunks that hold CH consecutive feature
 // rows a of one column b, ordered [a / CH][b][a % CH].  With bf16 (CH = 8) this is the K-major, unswizzled
@@ -125,6 +126,13 @@ template <typename T> __host__ __device__ constexpr int grf_tile_chunk() { retur
 template <typename T> __host__ __device__ constexpr size_t grf_tile_index(int a, int b, int D)
 {
     return ((size_t)(a / grf_tile_chunk<T>()) * D + b) * grf_tile_chunk<T>() + (a % grf_tile_chunk<T>());
+}
+
+// The workspace holds one record per (problem, node): the state tile S_l followed by z_l (m fp32 values), so
+// that one contiguous copy brings both.
+template <typename T> __host__ __device__ constexpr size_t grf_record_bytes(int M, int D)
+{
+    return (size_t)M * D * sizeof(T) + (size_t)M * sizeof(float);
 }
 
 static inline int grf_ceil_div(int64_t a, int64_t b) { return (int)((a + b - 1) / b); }
