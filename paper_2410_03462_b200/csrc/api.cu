@@ -165,7 +165,7 @@ extern "C" int grf_features_free(grf_features* feat)
     cudaSetDevice(feat->device);
     csr_release(&feat->phi); csr_release(&feat->psi); csr_release(&feat->psit);
     grf_buf_release(&feat->plan_off); grf_buf_release(&feat->plan_cnt);
-    grf_buf_release(&feat->plan_col); grf_buf_release(&feat->plan_total);
+    grf_buf_release(&feat->plan_col); grf_buf_release(&feat->plan_total); grf_buf_release(&feat->plan_coef);
     delete feat;
     return GRF_OK;
 }

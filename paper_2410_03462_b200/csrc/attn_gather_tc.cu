@@ -151,9 +151,9 @@ constexpr int TC_THREADS = 224;
 
 template <int M, int D>
 __global__ void __launch_bounds__(TC_THREADS)
-gather_contract_tc_kernel(int32_t N, int32_t R, const int32_t* __restrict__ rowptr, const int32_t* __restrict__ col,
-                          const float* __restrict__ val, const int32_t* __restrict__ plan_off,
+gather_contract_tc_kernel(int32_t N, int32_t R, const int32_t* __restrict__ plan_off,
                           const int32_t* __restrict__ plan_cnt, const int32_t* __restrict__ plan_col,
+                          const uint2* __restrict__ plan_coef,
                           const __nv_bfloat16* __restrict__ phiQ, const unsigned char* __restrict__ records,
                           __nv_bfloat16* __restrict__ out, const float* __restrict__ den_in, int* __restrict__ error_word)
 {
@@ -216,18 +216,24 @@ gather_contract_tc_kernel(int32_t N, int32_t R, const int32_t* __restrict__ rowp
 #pragma unroll
             for (int c = 0; c < M / 2; ++c) q2[c] = 0u;
         }
-        // this row's non-zeros of Phi, walked in step with the union list; two entries are kept ahead
-        int32_t p = live ? rowptr[row] : 0;
-        const int32_t pend = live ? rowptr[row + 1] : 0;
-        int32_t col0 = p < pend ? __ldg(col + p) : -1, col1 = p + 1 < pend ? __ldg(col + p + 1) : -1;
-        float val0 = p < pend ? __ldg(val + p) : 0.0f, val1 = p + 1 < pend ? __ldg(val + p + 1) : 0.0f;
+        // this row's coefficients Phi_il for the block's union entries, four entries (bf16) per 8-byte word,
+        // read two words ahead of their use
+        const uint2* tab = plan_coef + (size_t)(plan_off[blk] >> 2) * BQ + tid;
+        const int32_t nquads = cnt >> 2;
+        uint2 cur = make_uint2(0u, 0u);
+        uint2 nxt1 = nquads > 0 ? __ldg(tab) : make_uint2(0u, 0u);
+        uint2 nxt2 = nquads > 1 ? __ldg(tab + BQ) : make_uint2(0u, 0u);
         const float den = live ? den_in[(size_t)g * N + row] : 0.0f;
         bool ok = true;
-        int32_t l_mine = -1;
         const uint32_t lane_field = (uint32_t)(warp * 32) << 16;
         for (int32_t gi = 0; gi < ngroups; ++gi) {
             const int32_t u0 = gi * GU;
-            if ((u0 & 31) == 0) l_mine = (u0 + lane < cnt) ? __ldg(ulist + u0 + lane) : -1;   // GU divides 32
+            if ((u0 & 3) == 0) {
+                const int32_t q = u0 >> 2;
+                cur = nxt1; nxt1 = nxt2;
+                nxt2 = q + 2 < nquads ? __ldg(tab + (size_t)(q + 2) * BQ) : make_uint2(0u, 0u);
+            }
+            const unsigned long long quad = ((unsigned long long)cur.y << 32) | cur.x;
             const int st = gi % NA;
             // the A slots of this stage are free once the group that used them NA groups ago has been multiplied
             if (gi >= NA && !mbar_wait(done((gi - NA) % NBC), (uint32_t)((gi - NA) / NBC) & 1u, &abort_flag)) ok = false;
@@ -236,16 +242,12 @@ gather_contract_tc_kernel(int32_t N, int32_t R, const int32_t* __restrict__ rowp
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
 #pragma unroll
             for (int j = 0; j < GU; ++j) {
-                const int32_t u = u0 + j;
-                const int32_t l = __shfl_sync(0xffffffffu, l_mine, u & 31);   // -1 beyond the list: matches nothing
                 // A_l[row, :] = Phi_il * phi(q_row): zeros for most rows; products are taken in packed bf16
+                const uint32_t cbits = (uint32_t)(quad >> (16 * ((u0 + j) & 3))) & 0xffffu;
                 uint32_t w[M / 2];
-                if (l >= 0 && col0 == l) {
-                    const __nv_bfloat162 c2 = __float2bfloat162_rn(val0);
-                    ++p;
-                    col0 = col1; val0 = val1;
-                    col1 = p + 1 < pend ? __ldg(col + p + 1) : -1;
-                    val1 = p + 1 < pend ? __ldg(val + p + 1) : 0.0f;
+                if (cbits != 0u) {
+                    const uint32_t cpair = cbits | (cbits << 16);
+                    const __nv_bfloat162 c2 = *reinterpret_cast<const __nv_bfloat162*>(&cpair);
 #pragma unroll
                     for (int e = 0; e < M / 2; ++e) {
                         const __nv_bfloat162 h = __hmul2(*reinterpret_cast<const __nv_bfloat162*>(&q2[e]), c2);
@@ -437,7 +439,7 @@ block_plan_kernel(int32_t N, int32_t R, const int32_t* __restrict__ rowptr, cons
 {
     extern __shared__ uint32_t bitmap[];        // one bit per column
     __shared__ int32_t warp_sums[8];
-    __shared__ int32_t base_off;
+    __shared__ int32_t base_off, block_total;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int32_t blk = blockIdx.x;
     const int32_t words = (R + 31) >> 5;
@@ -465,10 +467,12 @@ block_plan_kernel(int32_t N, int32_t R, const int32_t* __restrict__ rowptr, cons
     int32_t before = inc - mine;
     for (int w = 0; w < warp; ++w) before += warp_sums[w];
     if (tid == 255) {
-        const int32_t total = before + mine;
-        base_off = atomicAdd(plan_total, total);
+        // lists are padded to a multiple of four entries (the last column repeated, with zero coefficients)
+        const int32_t total = before + mine, padded = (total + 3) & ~3;
+        base_off = atomicAdd(plan_total, padded);
+        block_total = total;
         plan_off[blk] = base_off;
-        plan_cnt[blk] = total;
+        plan_cnt[blk] = padded;
     }
     __syncthreads();
     int32_t o = base_off + before;
@@ -480,6 +484,67 @@ block_plan_kernel(int32_t N, int32_t R, const int32_t* __restrict__ rowptr, cons
             plan_col[o++] = (x << 5) + b;
         }
     }
+    if (before + mine == block_total && block_total > 0) {
+        // the thread that holds the end of the list: w1 may be below `words` only for trailing empty ranges
+        bool last = true;
+        for (int32_t x = w1; x < words && last; ++x) last = bitmap[x] == 0u;
+        if (last && mine > 0) {
+            const int32_t last_col = plan_col[base_off + block_total - 1];
+            for (int32_t e = block_total; e < ((block_total + 3) & ~3); ++e) plan_col[base_off + e] = last_col;
+        }
+    }
+}
+
+// Second pass of the plan: the block's coefficients as a dense table, four union entries (bf16) per 8-byte
+// word, [quad][row][4], so that a row thread of the gather kernel reads its coefficients with one coalesced
+// load per four union entries.
+__global__ void __launch_bounds__(256)
+block_coef_kernel(int32_t N, int32_t R, const int32_t* __restrict__ rowptr, const int32_t* __restrict__ col,
+                  const float* __restrict__ val, const int32_t* __restrict__ plan_off,
+                  const int32_t* __restrict__ plan_cnt, __nv_bfloat16* __restrict__ plan_coef)
+{
+    extern __shared__ uint32_t smem_plan[];     // bitmap, then the number of set bits before each word
+    __shared__ int32_t warp_sums[8];
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int32_t blk = blockIdx.x;
+    const int32_t words = (R + 31) >> 5;
+    uint32_t* bitmap = smem_plan;
+    int32_t* before_word = reinterpret_cast<int32_t*>(smem_plan + words);
+    for (int32_t x = tid; x < words; x += 256) bitmap[x] = 0u;
+    __syncthreads();
+    const int32_t r0 = blk * BQ, r1 = min(N, r0 + BQ);
+    for (int32_t p = rowptr[r0] + tid; p < rowptr[r1]; p += 256) {
+        const int32_t c = col[p];
+        atomicOr(&bitmap[c >> 5], 1u << (c & 31));
+    }
+    // zero this block's part of the table meanwhile
+    const int32_t off = plan_off[blk], cnt = plan_cnt[blk];
+    uint4* tab4 = reinterpret_cast<uint4*>(plan_coef + (size_t)off * BQ);
+    for (int32_t x = tid; x < cnt * (BQ * 2 / 16); x += 256) tab4[x] = make_uint4(0u, 0u, 0u, 0u);
+    __syncthreads();
+    const int32_t per = (words + 255) / 256;
+    const int32_t w0 = min(words, tid * per), w1 = min(words, w0 + per);
+    int32_t mine = 0;
+    for (int32_t x = w0; x < w1; ++x) mine += __popc(bitmap[x]);
+    int32_t inc = mine;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const int32_t y = __shfl_up_sync(0xffffffffu, inc, o);
+        if (lane >= o) inc += y;
+    }
+    if (lane == 31) warp_sums[warp] = inc;
+    __syncthreads();
+    int32_t run = inc - mine;
+    for (int w = 0; w < warp; ++w) run += warp_sums[w];
+    for (int32_t x = w0; x < w1; ++x) { before_word[x] = run; run += __popc(bitmap[x]); }
+    __syncthreads();
+    __nv_bfloat16* tab = plan_coef + (size_t)off * BQ;
+    for (int32_t r = r0 + warp; r < r1; r += 8)
+        for (int32_t p = rowptr[r] + lane; p < rowptr[r + 1]; p += 32) {
+            const int32_t c = col[p];
+            const int32_t u = before_word[c >> 5] + __popc(bitmap[c >> 5] & ((1u << (c & 31)) - 1u));
+            tab[((size_t)(u >> 2) * BQ + (r - r0)) * 4 + (u & 3)] = __float2bfloat16_rn(val[p]);
+        }
 }
 
 }  // namespace
@@ -489,20 +554,35 @@ int grf_build_block_plan(grf_ctx* ctx, grf_features* feat)
     grf_csr_dev& phi = feat->phi;
     feat->plan_ready = false;
     const int32_t N = phi.rows, R = phi.cols;
-    const size_t bitmap_bytes = (size_t)((R + 31) / 32) * 4;
-    if (bitmap_bytes > 200 * 1024 || phi.nnz <= 0) return GRF_OK;   // no plan: the ALU kernel serves this object
+    const size_t words = (size_t)(R + 31) / 32;
+    if (words * 8 > 200 * 1024 || phi.nnz <= 0) return GRF_OK;   // no plan: the ALU kernel serves this object
     const int32_t nblocks = grf_ceil_div(N, BQ);
     GRF_TRY(grf_buf_reserve(&feat->plan_off, sizeof(int32_t) * (size_t)nblocks));
     GRF_TRY(grf_buf_reserve(&feat->plan_cnt, sizeof(int32_t) * (size_t)nblocks));
-    GRF_TRY(grf_buf_reserve(&feat->plan_col, phi.col.bytes));       // at most nnz entries in total
+    GRF_TRY(grf_buf_reserve(&feat->plan_col, phi.col.bytes + sizeof(int32_t) * 3 * (size_t)nblocks));
     GRF_TRY(grf_buf_reserve(&feat->plan_total, sizeof(int32_t)));
     GRF_CUDA_TRY(cudaMemsetAsync(feat->plan_total.ptr, 0, sizeof(int32_t), ctx->stream));
-    GRF_CUDA_TRY(cudaFuncSetAttribute(block_plan_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bitmap_bytes));
+    GRF_CUDA_TRY(cudaFuncSetAttribute(block_plan_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(words * 4)));
     {
         grf_launch_scope scope(ctx, 3);
-        block_plan_kernel<<<nblocks, 256, bitmap_bytes, ctx->stream>>>(
+        block_plan_kernel<<<nblocks, 256, words * 4, ctx->stream>>>(
             N, R, (const int32_t*)phi.rowptr.ptr, (const int32_t*)phi.col.ptr, (int32_t*)feat->plan_off.ptr,
             (int32_t*)feat->plan_cnt.ptr, (int32_t*)feat->plan_col.ptr, (int32_t*)feat->plan_total.ptr);
+    }
+    GRF_CUDA_TRY(cudaGetLastError());
+    // the table's size is known only now
+    GRF_CUDA_TRY(cudaMemcpyAsync(ctx->pinned + 4, feat->plan_total.ptr, sizeof(int32_t), cudaMemcpyDeviceToHost, ctx->stream));
+    GRF_CUDA_TRY(cudaStreamSynchronize(ctx->stream));
+    const size_t entries = (size_t)ctx->pinned[4];
+    const size_t table_bytes = entries * BQ * sizeof(__nv_bfloat16);
+    if (table_bytes > ((size_t)2 << 30)) return GRF_OK;           // too little sharing between neighbouring rows
+    if (feat->plan_coef.bytes < table_bytes) GRF_TRY(grf_buf_reserve(&feat->plan_coef, table_bytes + table_bytes / 8));
+    GRF_CUDA_TRY(cudaFuncSetAttribute(block_coef_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(words * 8)));
+    {
+        grf_launch_scope scope(ctx, 3);
+        block_coef_kernel<<<nblocks, 256, words * 8, ctx->stream>>>(
+            N, R, (const int32_t*)phi.rowptr.ptr, (const int32_t*)phi.col.ptr, (const float*)phi.val.ptr,
+            (const int32_t*)feat->plan_off.ptr, (const int32_t*)feat->plan_cnt.ptr, (__nv_bfloat16*)feat->plan_coef.ptr);
     }
     GRF_CUDA_TRY(cudaGetLastError());
     feat->plan_blocks = nblocks;
@@ -533,9 +613,8 @@ static int launch_tc(grf_ctx* ctx, const grf_features* feat, int32_t G, int32_t 
     {
         grf_launch_scope scope(ctx, 5);
         gather_contract_tc_kernel<M, D><<<grid, TC_THREADS, Sh::SMEM, ctx->stream>>>(
-            N, phi.cols, (const int32_t*)phi.rowptr.ptr, (const int32_t*)phi.col.ptr, (const float*)phi.val.ptr,
-            (const int32_t*)feat->plan_off.ptr, (const int32_t*)feat->plan_cnt.ptr, (const int32_t*)feat->plan_col.ptr,
-            (const __nv_bfloat16*)phiQ, (const unsigned char*)records, (__nv_bfloat16*)out, den, ctx->error_word);
+            N, phi.cols, (const int32_t*)feat->plan_off.ptr, (const int32_t*)feat->plan_cnt.ptr,
+            (const int32_t*)feat->plan_col.ptr, (const uint2*)feat->plan_coef.ptr, (const __nv_bfloat16*)phiQ, (const unsigned char*)records, (__nv_bfloat16*)out, den, ctx->error_word);
     }
     return cudaGetLastError() == cudaSuccess ? GRF_OK : GRF_ERR_CUDA;
 }

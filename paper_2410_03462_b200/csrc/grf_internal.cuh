@@ -76,6 +76,7 @@ struct grf_features {
     grf_csr_dev phi, psi, psit;
     // block plan of Phi: per block of GRF_PLAN_BLOCK rows, the sorted distinct columns
     grf_buf plan_off, plan_cnt, plan_col, plan_total;
+    grf_buf plan_coef;              // dense bf16 coefficients [quad of union entries][row of the block][4]
     int32_t plan_blocks = 0;
     bool plan_ready = false;
 };
