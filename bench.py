@@ -111,6 +111,10 @@ def algorithmic_bytes(w, N, nnz_phi, nnz_psi, E):
         "build_states": G * N * (m + d) * es + csr(nnz_psi) + S + z,
         # S, z, phi(Q), Phi read once; out written once
         "gather_contract": S + z + G * N * m * es + csr(nnz_phi) + G * N * d * es,
+        # z and Phi read once, denominators written once
+        "row_denominators": z + csr(nnz_phi) + G * N * m * es + G * N * 4,
+        # Phi read twice (union lists, coefficient table)
+        "block_plan": 2 * csr(nnz_phi),
     }
 
 

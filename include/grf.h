@@ -170,8 +170,9 @@ int grf_step_host(grf_ctx* ctx, int32_t N, const int32_t* rowptr, const int32_t*
  * bounded waits (GRF_ERR_TIMEOUT; the affected outputs are invalid), else GRF_OK. */
 int grf_ctx_check(grf_ctx* ctx);
 
-/* Chooses the gather-contract kernel for bf16 problems: 1 (default) = tensor-core kernel where a block plan
- * exists and m, d are multiples of 16; 0 = plain-ALU kernel always.  Results agree within the stated tolerance. */
+/* Chooses the attention kernels for bf16 problems: 1 (default) = tensor-core kernels where they apply (state
+ * build: m a multiple of 16 and d <= 64; gather-contract: a block plan exists and m, d are multiples of 16);
+ * 0 = plain-ALU kernels always.  Results agree within the stated tolerance. */
 int grf_ctx_use_tensor_cores(grf_ctx* ctx, int enable);
 
 /* Number of kernels the context has launched since it was created (for accounting in benchmarks). */
@@ -181,8 +182,9 @@ int64_t grf_ctx_launch_count(const grf_ctx* ctx);
  * bracketed by two CUDA events on the context's stream.  grf_ctx_kernel_times waits for the stream, adds
  * the elapsed times since the previous read to ms[GRF_KERNEL_CLASSES] / launches[GRF_KERNEL_CLASSES]
  * (HOST arrays, overwritten) and clears the record.  Classes: 0 walk+merge, 1 prefix scans, 2 row
- * compaction, 3 column regrouping (histogram, scatter, ordering), 4 state build (S, z), 5 gather-contract. */
-#define GRF_KERNEL_CLASSES 6
+ * compaction, 3 column regrouping (histogram, scatter, ordering), 4 state build (S, z), 5 gather-contract,
+ * 6 denominators pass of the tensor-core gather, 7 block plan of the tensor-core gather. */
+#define GRF_KERNEL_CLASSES 8
 int grf_ctx_enable_timing(grf_ctx* ctx, int enable);
 int grf_ctx_kernel_times(grf_ctx* ctx, float* ms, int64_t* launches);
 

@@ -117,7 +117,8 @@ def grf_ctx_use_tensor_cores(ctx: int, enable: bool):
     _check(lib.grf_ctx_use_tensor_cores(ctx, int(enable)), "grf_ctx_use_tensor_cores")
 
 
-KERNEL_CLASSES = ("walk_merge", "scan", "compact", "regroup", "build_states", "gather_contract")
+KERNEL_CLASSES = ("walk_merge", "scan", "compact", "regroup", "build_states", "gather_contract", "row_denominators",
+                  "block_plan")
 
 
 def grf_ctx_enable_timing(ctx: int, enable: bool):

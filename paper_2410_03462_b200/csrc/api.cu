@@ -281,7 +281,11 @@ extern "C" int grf_masked_linear_attn(grf_ctx* ctx, const grf_features* feat, in
         const char* q_ptr = (const char*)phiQ + (size_t)g0 * N * m * es;
         char* o_ptr = (char*)out + (size_t)g0 * N * d * es;
         float* den_ptr = den_out ? den_out + (size_t)g0 * N : nullptr;
-        GRF_TRY(grf_build_states(ctx, feat->psit, gc, N, m, d, dtype, k_ptr, v_ptr, workspace));
+        int rs = 1;
+        if (dtype == GRF_DTYPE_BF16 && ctx->use_tensor_cores)
+            rs = grf_build_states_tc(ctx, feat->psit, gc, N, m, d, k_ptr, v_ptr, workspace);
+        if (rs > 0) rs = grf_build_states(ctx, feat->psit, gc, N, m, d, dtype, k_ptr, v_ptr, workspace);
+        GRF_TRY(rs);
         int rc = 1;
         if (dtype == GRF_DTYPE_BF16 && ctx->use_tensor_cores)
             rc = grf_gather_contract_tc(ctx, feat, gc, N, m, d, q_ptr, workspace, o_ptr, den_ptr);

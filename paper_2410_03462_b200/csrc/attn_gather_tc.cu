@@ -564,7 +564,7 @@ int grf_build_block_plan(grf_ctx* ctx, grf_features* feat)
     GRF_CUDA_TRY(cudaMemsetAsync(feat->plan_total.ptr, 0, sizeof(int32_t), ctx->stream));
     GRF_CUDA_TRY(cudaFuncSetAttribute(block_plan_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(words * 4)));
     {
-        grf_launch_scope scope(ctx, 3);
+        grf_launch_scope scope(ctx, 7);
         block_plan_kernel<<<nblocks, 256, words * 4, ctx->stream>>>(
             N, R, (const int32_t*)phi.rowptr.ptr, (const int32_t*)phi.col.ptr, (int32_t*)feat->plan_off.ptr,
             (int32_t*)feat->plan_cnt.ptr, (int32_t*)feat->plan_col.ptr, (int32_t*)feat->plan_total.ptr);
@@ -579,7 +579,7 @@ int grf_build_block_plan(grf_ctx* ctx, grf_features* feat)
     if (feat->plan_coef.bytes < table_bytes) GRF_TRY(grf_buf_reserve(&feat->plan_coef, table_bytes + table_bytes / 8));
     GRF_CUDA_TRY(cudaFuncSetAttribute(block_coef_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(words * 8)));
     {
-        grf_launch_scope scope(ctx, 3);
+        grf_launch_scope scope(ctx, 7);
         block_coef_kernel<<<nblocks, 256, words * 8, ctx->stream>>>(
             N, R, (const int32_t*)phi.rowptr.ptr, (const int32_t*)phi.col.ptr, (const float*)phi.val.ptr,
             (const int32_t*)feat->plan_off.ptr, (const int32_t*)feat->plan_cnt.ptr, (__nv_bfloat16*)feat->plan_coef.ptr);
@@ -604,7 +604,7 @@ static int launch_tc(grf_ctx* ctx, const grf_features* feat, int32_t G, int32_t 
         den = (float*)ctx->den_scratch.ptr;
     }
     {
-        grf_launch_scope scope(ctx, 5);
+        grf_launch_scope scope(ctx, 6);
         row_denominators_kernel<M, D><<<dim3(grf_ceil_div(N, 8), G), 256, 0, ctx->stream>>>(
             N, phi.cols, (const int32_t*)phi.rowptr.ptr, (const int32_t*)phi.col.ptr, (const float*)phi.val.ptr,
             (const __nv_bfloat16*)phiQ, (const unsigned char*)records, den);

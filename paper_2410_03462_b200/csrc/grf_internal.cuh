@@ -112,6 +112,8 @@ int grf_transpose_launch(grf_ctx* ctx, int32_t rows, int32_t cols, int64_t nnz,
 // attn_state.cu / attn_gather.cu
 int grf_build_states(grf_ctx* ctx, const grf_csr_dev& psit, int32_t G, int32_t N, int32_t m, int32_t d, int dtype,
                      const void* phiK, const void* V, void* records);
+int grf_build_states_tc(grf_ctx* ctx, const grf_csr_dev& psit, int32_t G, int32_t N, int32_t m, int32_t d,
+                        const void* phiK, const void* V, void* records);
 int grf_gather_contract_alu(grf_ctx* ctx, const grf_csr_dev& phi, int32_t G, int32_t N, int32_t m, int32_t d,
                             int dtype, const void* phiQ, const void* records, void* out, float* den_out);
 // attn_gather_tc.cu
