@@ -170,66 +170,96 @@ build_states_tc_kernel(int32_t R, int32_t N, const int32_t* __restrict__ t_rowpt
 
     if (warp >= 5) {
         // ------------------------------------------------------------ producers
+        // Software pipeline over items: while item q is written to shared memory, the rows of item q+1 and
+        // the (key, Psi) pairs of item q+2 are already on their way from L2.
         const int ptid = tid - 160;            // 0..127: key row jj = ptid / 2, half h = ptid % 2 of its pieces
         const int jj = ptid >> 1, h = ptid & 1;
         const uint32_t a_row = (uint32_t)(jj / 16) * Sh::A_KSTEP + (uint32_t)((jj % 16) / 8) * Sh::A_LBO + (uint32_t)(jj % 8) * 16;
         const uint32_t b_row = (uint32_t)(jj / 16) * Sh::B_KSTEP + (uint32_t)((jj % 16) / 8) * Sh::B_LBO + (uint32_t)(jj % 8) * 16;
+        constexpr int NV = (D / 8 + 1) / 2, NK = (M / 8 + 1) / 2;
+
+        struct Walk {          // position in the CTA's item sequence
+            int32_t l, it, beg, c;
+            __device__ __forceinline__ void load(const int32_t* rp, int32_t lend) {
+                if (l < lend) { beg = __ldg(rp + l); c = __ldg(rp + l + 1) - beg; } else { beg = 0; c = 0; }
+            }
+            __device__ __forceinline__ void advance(const int32_t* rp, int32_t lend) {
+                const int32_t nitems = c > 0 ? (c + ITEM_KEYS - 1) / ITEM_KEYS : 1;
+                if (++it >= nitems) { ++l; it = 0; load(rp, lend); }
+            }
+            __device__ __forceinline__ int32_t keys() const { return min(ITEM_KEYS, c - it * ITEM_KEYS); }
+        };
+        struct Idx { int32_t j; float psi; bool real; };
+        auto fetch_idx = [&](const Walk& w) {
+            Idx x; x.j = 0; x.psi = 0.0f;
+            x.real = w.l < l1 && jj < w.keys();
+            if (x.real) { x.j = __ldg(t_col + w.beg + w.it * ITEM_KEYS + jj); x.psi = __ldg(t_val + w.beg + w.it * ITEM_KEYS + jj); }
+            return x;
+        };
+        struct Rows { uint4 v[NV], k[NK]; };
+        auto fetch_rows = [&](const Idx& x) {
+            Rows r;
+#pragma unroll
+            for (int y = 0; y < NV; ++y) r.v[y] = make_uint4(0u, 0u, 0u, 0u);
+#pragma unroll
+            for (int y = 0; y < NK; ++y) r.k[y] = make_uint4(0u, 0u, 0u, 0u);
+            if (x.real) {
+#pragma unroll
+                for (int y = 0; y < NV; ++y)
+                    if (h + 2 * y < D / 8) r.v[y] = __ldg(reinterpret_cast<const uint4*>(Vg + (size_t)x.j * D) + h + 2 * y);
+#pragma unroll
+                for (int y = 0; y < NK; ++y)
+                    if (h + 2 * y < M / 8) r.k[y] = __ldg(reinterpret_cast<const uint4*>(Kg + (size_t)x.j * M) + h + 2 * y);
+            }
+            return r;
+        };
+
+        Walk w0; w0.l = l0; w0.it = 0; w0.load(t_rowptr, l1);
+        Walk w2 = w0;
+        Idx idx_cur = fetch_idx(w2);
+        w2.advance(t_rowptr, l1);
+        Idx idx_nxt = fetch_idx(w2);
+        w2.advance(t_rowptr, l1);
+        Rows rows_cur = fetch_rows(idx_cur);
         int32_t q = 0;
         bool ok = true;
-        for (int32_t l = l0; l < l1 && ok; ++l) {
-            const int32_t beg = t_rowptr[l], c = t_rowptr[l + 1] - beg;
-            const int32_t nitems = c > 0 ? (c + ITEM_KEYS - 1) / ITEM_KEYS : 1;
-            for (int32_t it = 0; it < nitems; ++it, ++q) {
-                const int s = q % NS;
-                const int32_t n = min(ITEM_KEYS, c - it * ITEM_KEYS);       // keys of this item (may be 0)
-                const int32_t rows = n > 0 ? ((n + 15) & ~15) : 16;         // rows the MMAs will read
-                // this thread's key: fetch before waiting for the buffer
-                const bool real = jj < n;
-                int32_t j = 0;
-                float psi = 0.0f;
-                if (real) { j = __ldg(t_col + beg + it * ITEM_KEYS + jj); psi = __ldg(t_val + beg + it * ITEM_KEYS + jj); }
-                uint4 vq[(D / 8 + 1) / 2], kq[(M / 8 + 1) / 2];
-                if (real) {
+        while (w0.l < l1) {
+            const Rows rows_nxt = fetch_rows(idx_nxt);        // item q+1
+            const Idx idx_nxt2 = fetch_idx(w2);               // item q+2
+            w2.advance(t_rowptr, l1);
+            const int s = q % NS;
+            const int32_t n = w0.keys();
+            const int32_t rows = n > 0 ? ((n + 15) & ~15) : 16;         // rows the MMAs will read
+            if (!mbar_wait(empty(s), ((uint32_t)(q / NS) & 1u) ^ 1u, &abort_flag)) ok = false;
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
+            if (jj < rows) {
+                unsigned char* a_dst = stage_generic + (size_t)s * Sh::STAGE + a_row;
+                unsigned char* b_dst = stage_generic + (size_t)s * Sh::STAGE + Sh::A_BYTES + b_row;
 #pragma unroll
-                    for (int x = 0; x < (D / 8 + 1) / 2; ++x)
-                        if (h + 2 * x < D / 8) vq[x] = __ldg(reinterpret_cast<const uint4*>(Vg + (size_t)j * D) + h + 2 * x);
+                for (int y = 0; y < NV; ++y)
+                    if (h + 2 * y < D / 8) *reinterpret_cast<uint4*>(a_dst + (size_t)(h + 2 * y) * 128) = rows_cur.v[y];
 #pragma unroll
-                    for (int x = 0; x < (M / 8 + 1) / 2; ++x)
-                        if (h + 2 * x < M / 8) kq[x] = __ldg(reinterpret_cast<const uint4*>(Kg + (size_t)j * M) + h + 2 * x);
-                }
-                if (!mbar_wait(empty(s), ((uint32_t)(q / NS) & 1u) ^ 1u, &abort_flag)) ok = false;
-                ok = __all_sync(0xffffffffu, ok);
-                if (!ok) break;
-                if (jj < rows) {
-                    unsigned char* a_dst = stage_generic + (size_t)s * Sh::STAGE + a_row;
-                    unsigned char* b_dst = stage_generic + (size_t)s * Sh::STAGE + Sh::A_BYTES + b_row;
+                for (int y = 0; y < NK; ++y)
+                    if (h + 2 * y < M / 8) {
+                        const uint32_t w[4] = {rows_cur.k[y].x, rows_cur.k[y].y, rows_cur.k[y].z, rows_cur.k[y].w};
+                        uint32_t r[4];
 #pragma unroll
-                    for (int x = 0; x < (D / 8 + 1) / 2; ++x)
-                        if (h + 2 * x < D / 8)
-                            *reinterpret_cast<uint4*>(a_dst + (size_t)(h + 2 * x) * 128) = real ? vq[x] : make_uint4(0u, 0u, 0u, 0u);
-#pragma unroll
-                    for (int x = 0; x < (M / 8 + 1) / 2; ++x)
-                        if (h + 2 * x < M / 8) {
-                            uint4 o = make_uint4(0u, 0u, 0u, 0u);
-                            if (real) {
-                                const uint32_t w[4] = {kq[x].x, kq[x].y, kq[x].z, kq[x].w};
-                                uint32_t r[4];
-#pragma unroll
-                                for (int e = 0; e < 4; ++e) {
-                                    const float lo = psi * __uint_as_float(w[e] << 16);
-                                    const float hi = psi * __uint_as_float(w[e] & 0xffff0000u);
-                                    __nv_bfloat162 t2 = __floats2bfloat162_rn(lo, hi);
-                                    r[e] = *reinterpret_cast<uint32_t*>(&t2);
-                                }
-                                o = make_uint4(r[0], r[1], r[2], r[3]);
-                            }
-                            *reinterpret_cast<uint4*>(b_dst + (size_t)(h + 2 * x) * 128) = o;
+                        for (int e = 0; e < 4; ++e) {
+                            const float lo = idx_cur.psi * __uint_as_float(w[e] << 16);
+                            const float hi = idx_cur.psi * __uint_as_float(w[e] & 0xffff0000u);
+                            __nv_bfloat162 t2 = __floats2bfloat162_rn(lo, hi);
+                            r[e] = *reinterpret_cast<uint32_t*>(&t2);
                         }
-                }
-                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-                __syncwarp();
-                if (lane == 0) mbar_arrive(full(s));
+                        *reinterpret_cast<uint4*>(b_dst + (size_t)(h + 2 * y) * 128) = make_uint4(r[0], r[1], r[2], r[3]);
+                    }
             }
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            __syncwarp();
+            if (lane == 0) mbar_arrive(full(s));
+            ++q;
+            w0.advance(t_rowptr, l1);
+            idx_cur = idx_nxt; idx_nxt = idx_nxt2; rows_cur = rows_nxt;
         }
     } else if (warp == 4) {
         // ------------------------------------------------------------ MMA issuer
