@@ -51,7 +51,7 @@ def peaks():
 
 class ClockSampler:
     """nvidia-smi clock/throttle samples every 100 ms while the timed region runs (read-only queries)."""
-    FIELDS = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+    FIELDS = ("timestamp,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
               "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
               "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
 
@@ -61,11 +61,14 @@ class ClockSampler:
         try:
             self.proc = subprocess.Popen(
                 ["nvidia-smi", f"--id={device_index}", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
-                 "-lms", "100"], stdout=self.tmp, stderr=subprocess.DEVNULL)
+                 "-lms", "20"], stdout=self.tmp, stderr=subprocess.DEVNULL)
         except OSError:
             self.proc = None
 
-    def stop(self):
+    def stop(self, t_begin=None, t_end=None):
+        """Median SM clock and throttle reasons over the samples taken between the two wall-clock times
+        (all samples if none falls inside)."""
+        import datetime
         out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
         if self.proc is not None:
             self.proc.terminate()
@@ -75,22 +78,28 @@ class ClockSampler:
                 self.proc.kill()
         self.tmp.flush()
         self.tmp.seek(0)
-        sm, mx, reasons = [], [], set()
+        rows = []
         for line in self.tmp:
             parts = [x.strip() for x in line.split(",")]
             if len(parts) < 9:
                 continue
             try:
-                sm.append(float(parts[1])); mx.append(float(parts[2]))
+                ts = datetime.datetime.strptime(parts[0], "%Y/%m/%d %H:%M:%S.%f").timestamp()
+                rows.append((ts, float(parts[1]), float(parts[2]), parts[5:9]))
             except ValueError:
                 continue
-            for name, flag in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), parts[5:9]):
-                if flag.lower().startswith("active"):
-                    reasons.add(name)
         self.tmp.close()
         os.unlink(self.tmp.name)
-        if sm:
-            out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(mx), reasons=sorted(reasons), samples=len(sm))
+        inside = [r for r in rows if t_begin is not None and t_begin <= r[0] <= t_end]
+        use = inside or rows
+        reasons = set()
+        for _, _, _, flags in use:
+            for name, flag in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), flags):
+                if flag.lower().startswith("active"):
+                    reasons.add(name)
+        if use:
+            out.update(sm_mhz=statistics.median(r[1] for r in use), sm_max_mhz=max(r[2] for r in use),
+                       reasons=sorted(reasons), samples=len(use), window="timed region" if inside else "whole run")
         return out
 
 
@@ -118,6 +127,17 @@ def algorithmic_bytes(w, N, nnz_phi, nnz_psi, E):
     }
 
 
+def rank_seed(base: int, rank: int) -> int:
+    """Every rank draws its own batch: same shapes, different values."""
+    return base + rank
+
+
+def aggregate_over_ranks(local_ms: float, tokens_per_rank_step: int, steps: int, world: int, reduce_max):
+    """Whole-job throughput: all ranks' tokens over the slowest rank's device time."""
+    total_ms = reduce_max(local_ms)
+    return total_ms, tokens_per_rank_step * world * steps / (total_ms * 1e-3)
+
+
 def run_ours(args):
     import torch
     import torch.distributed as dist
@@ -141,7 +161,7 @@ def run_ours(args):
     ctx = api.Context(local)
     dg = api.DeviceGraph(g, local)
     # every rank has its own batch of the same shape (weak scaling over independent problems)
-    q, k, v = tensors.qkv(w.G, N, w.m, w.d, w.dtype, configs.QKV_SEED + rank)
+    q, k, v = tensors.qkv(w.G, N, w.m, w.d, w.dtype, rank_seed(configs.QKV_SEED, rank))
     qd, kd, vd = q.cuda(), k.cuda(), v.cuda()
     dt = B.dtype_code(qd)
     ws_bytes = B.grf_attn_workspace_bytes(w.G, N, w.m, w.d, dt)
@@ -155,11 +175,12 @@ def run_ours(args):
                                    w.max_len, f, None, feat.handle)
         B.grf_masked_linear_attn(ctx.handle, feat.handle, w.G, N, w.m, w.d, dt, qd, kd, vd, out, None, ws, ws_bytes)
 
+    sampler = ClockSampler(local) if rank == 0 else None
+    B.grf_ctx_enable_timing(ctx.handle, True)      # per-kernel events exist before the timed region starts
     for i in range(args.warmup):
         step(i)
     torch.cuda.synchronize()
-    B.grf_ctx_kernel_times(ctx.handle)
-    B.grf_ctx_enable_timing(ctx.handle, True)
+    B.grf_ctx_kernel_times(ctx.handle)             # discard the warm-up record
 
     def barrier():
         if world > 1:
@@ -168,12 +189,12 @@ def run_ours(args):
 
     # ---- timed region: K steps, each bracketed by CUDA events on the stream the kernels run on;
     # L2 is flushed between steps, outside the events
-    sampler = ClockSampler(local) if rank == 0 else None
     launches0 = ctx.launches
     evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
     ev_mid = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]
     barrier()
     t_wall0 = time.perf_counter()
+    t_epoch0 = time.time()
     for i in range(args.steps):
         flush.zero_()
         evs[i][0].record()
@@ -184,7 +205,7 @@ def run_ours(args):
         evs[i][1].record()
     barrier()
     wall = time.perf_counter() - t_wall0
-    clocks = sampler.stop() if sampler else None
+    t_epoch1 = time.time()
     launches = ctx.launches - launches0
     step_ms = [a.elapsed_time(b) for a, b in evs]
     sample_ms = [a[0].elapsed_time(mid) for a, mid in zip(evs, ev_mid)]
@@ -217,6 +238,8 @@ def run_ours(args):
     h2d = (rp_h.numel() + c_h.numel() + w_h.numel()) * 4 + sum(t.numel() * t.element_size() for t in (qh, kh, vh))
     d2h = oh.numel() * oh.element_size()
 
+    clocks = sampler.stop(t_epoch0, t_epoch1) if sampler else None
+
     # ---- max over ranks
     def rmax(x):
         if world == 1:
@@ -225,10 +248,9 @@ def run_ours(args):
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
         return float(t.item())
 
-    total_ms = rmax(total_ms)
+    total_ms, value = aggregate_over_ranks(total_ms, w.batch * N, args.steps, world, rmax)
     e2e_ms = rmax(e2e_ms)
     tokens_per_step = w.batch * N * world
-    value = tokens_per_step * args.steps / (total_ms * 1e-3)
 
     result = None
     if rank == 0:

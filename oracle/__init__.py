@@ -207,15 +207,18 @@ def attn_bruteforce(phiQ, phiK, V, Mhat: np.ndarray, rows=None):
     Vd = np.asarray(V, dtype=np.float64)
     G, N, _ = Q.shape
     rows = np.arange(N) if rows is None else np.asarray(rows)
-    Mr = np.asarray(Mhat, dtype=np.float64)[rows]
+    Mr = np.asarray(Mhat[rows], dtype=np.float64)      # only the requested rows of the mask are touched
     num = np.empty((G, len(rows), Vd.shape[2])); den = np.empty((G, len(rows)))
+    num_abs = np.empty_like(num); den_abs = np.empty_like(den)
     for g in range(G):
         A = (Q[g][rows] @ K[g].T) * Mr
         num[g] = A @ Vd[g]
         den[g] = A.sum(axis=1)
+        num_abs[g] = np.abs(A) @ np.abs(Vd[g])      # sums of the absolute values of the terms
+        den_abs[g] = np.abs(A).sum(axis=1)
     with np.errstate(divide="ignore", invalid="ignore"):
         out = np.where(den[..., None] != 0.0, num / den[..., None], 0.0)
-    return dict(num=num, den=den, out=out)
+    return dict(num=num, den=den, out=out, num_abs=num_abs, den_abs=den_abs)
 
 
 def mask_rows(Phi: CSR, Psi: CSR, rows) -> np.ndarray:

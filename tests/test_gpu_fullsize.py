@@ -1,0 +1,62 @@
+"""Parity at the benchmark's full size and launch configuration (N = 32768 point cloud, 8 heads, m = 32,
+d = 64, bf16): the sampler's output bit for bit against the oracle, and the attention on sampled query rows
+against the O(N) brute force of Eqs. 1-2 restricted to those rows."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from tests import helpers
+from workloads import configs, tensors
+
+pytestmark = pytest.mark.gpu
+
+
+def test_bench_workload_sampler_and_sampled_attention_rows():
+    from paper_2410_03462_b200 import api, binding as B
+    w = configs.point_cloud_32768()
+    g = w.graph()
+    ctx = api.Context(0)
+    f = oracle.deconvolve(w.alpha).astype(np.float32)
+    feat = api.sample(ctx, api.DeviceGraph(g), configs.WALK_SEED, w.n_walks, w.p_halt, w.max_len, f)
+    Phi, Psi, PsiT, _, _ = helpers.oracle_features(w, g, configs.WALK_SEED, f)
+    for which, want in ((0, Phi), (1, Psi), (2, PsiT)):
+        rp, c, v = feat.to_host(which)
+        assert np.array_equal(rp, want.rowptr) and np.array_equal(c, want.col)
+        assert np.array_equal(v.view(np.uint32), want.val.view(np.uint32))
+
+    q, k, v = tensors.qkv(w.G, g.N, w.m, w.d, w.dtype, configs.QKV_SEED)
+    qd, kd, vd = q.cuda(), k.cuda(), v.cuda()
+    rng = np.random.default_rng(5)
+    rows = np.unique(np.concatenate([[0, 127, 128, g.N - 1], rng.integers(0, g.N, 60)]))
+    Mrows = oracle.mask_rows(Phi, Psi, rows)
+    ref = oracle.attn_bruteforce(tensors.widen(q), tensors.widen(k), tensors.widen(v), Mrows_full(Mrows, rows, g.N), rows=rows)
+    for tensor_cores in (True, False):
+        B.grf_ctx_use_tensor_cores(ctx.handle, tensor_cores)
+        out, den = api.masked_linear_attn(ctx, feat, qd, kd, vd, want_den=True)
+        B.grf_ctx_check(ctx.handle)
+        out_rows = out[:, rows].float().cpu().numpy()
+        den_rows = den[:, rows].cpu().numpy()
+        helpers.assert_attn_close(out_rows, ref, helpers.TOL["bf16"], den_rows, f"full size tensor_cores={tensor_cores}")
+        # properties that hold at any size: finite outputs, positive denominators (all terms are >= 0 here)
+        assert torch.isfinite(out.float()).all()
+        assert (den > 0).all()
+    B.grf_ctx_use_tensor_cores(ctx.handle, True)
+    # run-to-run determinism of the whole path at full size
+    out2 = api.masked_linear_attn(ctx, feat, qd, kd, vd)
+    out3 = api.masked_linear_attn(ctx, feat, qd, kd, vd)
+    assert torch.equal(out2, out3)
+    feat.free()
+    ctx.close()
+
+
+def Mrows_full(Mrows, rows, N):
+    """attn_bruteforce indexes the mask by absolute row: place the sampled rows into an N x N frame lazily."""
+    class _Rows:
+        def __init__(self):
+            self.pos = {int(r): i for i, r in enumerate(rows)}
+        def __getitem__(self, idx):
+            return np.stack([Mrows[self.pos[int(r)]] for r in np.atleast_1d(idx)])
+        def __array__(self, dtype=None, copy=None):
+            raise TypeError("dense N x N mask is never formed")
+    return _Rows()
