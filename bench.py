@@ -61,7 +61,7 @@ class ClockSampler:
         try:
             self.proc = subprocess.Popen(
                 ["nvidia-smi", f"--id={device_index}", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
-                 "-lms", "20"], stdout=self.tmp, stderr=subprocess.DEVNULL)
+                 "-lms", "50"], stdout=self.tmp, stderr=subprocess.DEVNULL)
         except OSError:
             self.proc = None
 
@@ -155,6 +155,9 @@ def run_ours(args):
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
 
     w = make_workload(args.workload)
+    if args.heads > 0:
+        w.heads = args.heads
+        w.name += f"-heads{args.heads}"
     g = w.graph()
     N, E = g.N, g.E
     f = B.grf_deconvolve(w.alpha).astype(np.float32)
@@ -353,6 +356,7 @@ def main():
     ap.add_argument("--workload", default="pc32768")
     ap.add_argument("--cpu-heads", type=int, default=1, help="problems of the batch the CPU baseline really runs")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--heads", type=int, default=0, help="override the workload's head count (profiling of a smaller case)")
     args = ap.parse_args()
     if args.warmup < 3 and args.impl == "ours":
         args.warmup = 3
