@@ -29,6 +29,17 @@ if ROOT not in sys.path:
 METRIC = "grf_masked_linear_attention_tokens_per_s"
 UNIT = "tokens/s"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0}
+# DRAM bytes (read + write) of one launch at the default workload, from the ncu capture summarised in
+# profiles/kernels_pointcloud32768_2heads.md (taken with 2 of the 8 heads; traffic grows in proportion to the
+# heads, so the figures are scaled by 4).  Set an entry to None when its kernel changes after the capture.
+NCU_TRAFFIC_BYTES = {
+    "pointcloud-gmm16-N32768": {
+        "gather_contract": 4 * (1.368350e9 + 9.472768e6),
+        "build_states": 4 * (0.062359e9 + 220.503552e6),
+        "row_denominators": 4 * (0.037773e9 + 0.019712e6),
+        "walk_merge": 0.004971e9 + 5.708288e6,
+    }
+}
 
 
 def make_workload(name: str):
@@ -283,8 +294,9 @@ def run_ours(args):
             "e2e": {"value": tokens_per_step / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
                     "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms, "entry_point": "grf_step_host"},
             "roofline": {"kernel": dom, "bound": "hbm", "achieved": achieved, "peak": peak_gbs, "unit": "GB/s",
-                         "frac": achieved / peak_gbs, "peak_source": peak_kind, "traffic": None,
-                         "ms_per_launch": dom_ms},
+                         "frac": achieved / peak_gbs, "peak_source": peak_kind,
+                         "traffic": NCU_TRAFFIC_BYTES.get(w.name, {}).get(dom),
+                         "algorithmic_bytes": alg[dom], "ms_per_launch": dom_ms},
             "phases": {"sample_ms": statistics.mean(sample_ms), "attn_ms": statistics.mean(attn_ms),
                        "sample_ms_min_med_max": [min(sample_ms), statistics.median(sample_ms), max(sample_ms)],
                        "attn_ms_min_med_max": [min(attn_ms), statistics.median(attn_ms), max(attn_ms)],
