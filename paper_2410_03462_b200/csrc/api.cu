@@ -66,6 +66,7 @@ extern "C" int grf_ctx_destroy(grf_ctx* ctx)
     if (ctx->h_feat) grf_features_free(ctx->h_feat);
     if (ctx->pinned) cudaFreeHost(ctx->pinned);
     if (ctx->error_word) cudaFree(ctx->error_word);
+    if (ctx->copy_stream) { cudaStreamSynchronize(ctx->copy_stream); cudaStreamDestroy(ctx->copy_stream); cudaEventDestroy(ctx->copy_done); }
     for (auto& t : ctx->timed) { cudaEventDestroy(t.beg); cudaEventDestroy(t.end); }
     for (cudaEvent_t e : ctx->free_events) cudaEventDestroy(e);
     delete ctx;
@@ -331,9 +332,15 @@ extern "C" int grf_step_host(grf_ctx* ctx, int32_t N, const int32_t* rowptr, con
         GRF_CUDA_TRY(cudaMemcpyAsync(ctx->h_col.ptr, col, E * 4, cudaMemcpyHostToDevice, s));
         GRF_CUDA_TRY(cudaMemcpyAsync(ctx->h_w.ptr, w, E * 4, cudaMemcpyHostToDevice, s));
     }
-    GRF_CUDA_TRY(cudaMemcpyAsync(ctx->h_q.ptr, phiQ, qk_bytes, cudaMemcpyHostToDevice, s));
-    GRF_CUDA_TRY(cudaMemcpyAsync(ctx->h_k.ptr, phiK, qk_bytes, cudaMemcpyHostToDevice, s));
-    GRF_CUDA_TRY(cudaMemcpyAsync(ctx->h_v.ptr, V, v_bytes, cudaMemcpyHostToDevice, s));
+    // phi(Q), phi(K), V travel on a second stream while the features are sampled on the context's stream
+    if (!ctx->copy_stream) {
+        GRF_CUDA_TRY(cudaStreamCreateWithFlags(&ctx->copy_stream, cudaStreamNonBlocking));
+        GRF_CUDA_TRY(cudaEventCreateWithFlags(&ctx->copy_done, cudaEventDisableTiming));
+    }
+    GRF_CUDA_TRY(cudaMemcpyAsync(ctx->h_q.ptr, phiQ, qk_bytes, cudaMemcpyHostToDevice, ctx->copy_stream));
+    GRF_CUDA_TRY(cudaMemcpyAsync(ctx->h_k.ptr, phiK, qk_bytes, cudaMemcpyHostToDevice, ctx->copy_stream));
+    GRF_CUDA_TRY(cudaMemcpyAsync(ctx->h_v.ptr, V, v_bytes, cudaMemcpyHostToDevice, ctx->copy_stream));
+    GRF_CUDA_TRY(cudaEventRecord(ctx->copy_done, ctx->copy_stream));
     GRF_TRY(grf_sample(ctx, N, (const int32_t*)ctx->h_rowptr.ptr, (const int32_t*)ctx->h_col.ptr,
                        (const float*)ctx->h_w.ptr, seed, n_walks, p_halt, max_len, f_phi, f_psi, &ctx->h_feat));
     // workspace: everything if it is modest, else chunks of about 1 GiB
@@ -342,6 +349,7 @@ extern "C" int grf_step_host(grf_ctx* ctx, int32_t N, const int32_t* rowptr, con
     const size_t cap = (size_t)1 << 31;
     if (want > cap) want = per * (cap / per > 0 ? cap / per : 1);
     GRF_TRY(grf_buf_reserve(&ctx->h_ws, want));
+    GRF_CUDA_TRY(cudaStreamWaitEvent(s, ctx->copy_done, 0));
     GRF_TRY(grf_masked_linear_attn(ctx, ctx->h_feat, G, N, m, d, dtype, ctx->h_q.ptr, ctx->h_k.ptr, ctx->h_v.ptr,
                                    ctx->h_out.ptr, nullptr, ctx->h_ws.ptr, ctx->h_ws.bytes));
     GRF_CUDA_TRY(cudaMemcpyAsync(out, ctx->h_out.ptr, v_bytes, cudaMemcpyDeviceToHost, s));

@@ -43,6 +43,8 @@ struct grf_ctx {
     // host-buffer path
     grf_buf h_rowptr, h_col, h_w, h_q, h_k, h_v, h_out, h_ws;
     grf_features* h_feat = nullptr;
+    cudaStream_t copy_stream = nullptr;   // host-buffer path: inputs of the attention are uploaded beside the sampler
+    cudaEvent_t copy_done = nullptr;
     int32_t* pinned = nullptr;      // small pinned host block for read-backs
     int* error_word = nullptr;      // device word set by a kernel that gave up a bounded wait
     bool use_tensor_cores = true;
