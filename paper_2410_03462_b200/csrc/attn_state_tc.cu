@@ -7,13 +7,18 @@
 // the same instructions.  M = 128 costs the tensor pipe no more time than M = 64 at these widths.
 //
 // A CTA walks a range of nodes of one problem.  Keys are processed in items of up to 64 (four K = 16 steps):
-//   producers (4 warps)  gather v_j and Psi_jl * phi(k_j) into shared memory in the unswizzled MN-major
-//                        operand layout (16-byte pieces of a row go to 8x16-byte core matrices),
+//   producers (4 warps)  each warp owns one shared-memory stage and every fourth item: it gathers v_j and
+//                        phi(k_j) into the stage in the tensor cores' MN-major operand layout and scales the
+//                        phi(k_j) rows by Psi_jl in place.  Two kernels differ in how the rows travel:
+//                        asynchronous 16-byte copies into the unswizzled layout (any d <= 64), or, for d = 64,
+//                        the tensor-map copy engine gathering whole rows into the swizzled layout,
 //   one warp             issues the tcgen05.mma instructions, accumulating a node in tensor memory,
 //   epilogue (4 warps)   read the accumulator (two buffers, so the next node overlaps), round to bf16 and
 //                        write the node's record: the tile in the gather kernel's operand layout, then z_l.
 // The summation order over j is fixed by the instruction order (ascending j), so results are reproducible.
 // All mbarrier waits are bounded; a wait that gives up raises the context's error word.
+#include <cuda.h>
+
 #include "grf_internal.cuh"
 
 namespace {
@@ -96,10 +101,16 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16])
 }
 
 template <int M, int D> struct StShape {
-    static constexpr int A_LBO = 16 * 128;                    // 16 blocks of 8 rows (M = 128), 128 bytes each
+    // Blocks of 8 along M/N sit 144, 160 or 192 bytes apart, not 128: the eight lanes of a quarter warp copy
+    // 16-byte pieces of 1, 2 or 4 neighbouring keys (rows 8, 4 or 2 pieces long), and with these strides their
+    // destinations fall into eight different bank groups.
+    static constexpr int pad_stride(int pieces) { return pieces >= 8 ? 144 : (pieces == 4 ? 160 : 192); }
+    static constexpr int A_SBO = pad_stride(D / 8);
+    static constexpr int B_SBO = pad_stride(M / 8);
+    static constexpr int A_LBO = 16 * A_SBO;                  // 16 blocks of 8 rows (M = 128)
     static constexpr int A_KSTEP = 2 * A_LBO;                 // one K = 16 step of A
     static constexpr int A_BYTES = (ITEM_KEYS / 16) * A_KSTEP;
-    static constexpr int B_LBO = (M / 8) * 128;
+    static constexpr int B_LBO = (M / 8) * B_SBO;
     static constexpr int B_KSTEP = 2 * B_LBO;
     static constexpr int B_BYTES = (ITEM_KEYS / 16) * B_KSTEP;
     static constexpr int STAGE = A_BYTES + B_BYTES;
@@ -123,6 +134,7 @@ build_states_tc_kernel(int32_t R, int32_t N, const int32_t* __restrict__ t_rowpt
     __shared__ __align__(8) unsigned long long bars[2 * NS + 4];   // full, empty per stage; acc_full[2], acc_free[2]
     __shared__ uint32_t tmem_slot;
     __shared__ int abort_flag;
+    __shared__ int32_t node_beg[NODES_PER_CTA + 1];   // row pointers of the CTA's nodes
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int32_t g = blockIdx.y;
@@ -136,7 +148,7 @@ build_states_tc_kernel(int32_t R, int32_t N, const int32_t* __restrict__ t_rowpt
     auto acc_free = [&](int b) { return bar_base + 8u * (uint32_t)(2 * NS + 2 + b); };
 
     if (tid == 0) {
-        for (int s = 0; s < NS; ++s) { mbar_init(full(s), 4); mbar_init(empty(s), 1); }
+        for (int s = 0; s < NS; ++s) { mbar_init(full(s), 1); mbar_init(empty(s), 1); }
         for (int b = 0; b < 2; ++b) { mbar_init(acc_full(b), 1); mbar_init(acc_free(b), 4); }
         abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -146,6 +158,7 @@ build_states_tc_kernel(int32_t R, int32_t N, const int32_t* __restrict__ t_rowpt
                      ::"r"(smem_u32(&tmem_slot)), "r"((uint32_t)Sh::TMEM_COLS) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
+    if (tid <= NODES_PER_CTA) node_beg[tid] = t_rowptr[min(l0 + tid, R)];
     // constant part of every A buffer: zeros, and ones in row D (the row that sums Psi_jl phi(k_j) into z_l)
     for (int x = tid; x < NS * Sh::A_BYTES / 16; x += ST_THREADS) {
         const int s = x / (Sh::A_BYTES / 16), y = x % (Sh::A_BYTES / 16);
@@ -156,7 +169,7 @@ build_states_tc_kernel(int32_t R, int32_t N, const int32_t* __restrict__ t_rowpt
         const int s = x / ITEM_KEYS, jj = x % ITEM_KEYS;
         // key jj of the item: K step jj / 16, K block (jj % 16) / 8, row jj % 8 of the core matrix; M block D / 8
         unsigned char* p = stage_generic + (size_t)s * Sh::STAGE + (size_t)(jj / 16) * Sh::A_KSTEP +
-                           (size_t)((jj % 16) / 8) * Sh::A_LBO + (size_t)(D / 8) * 128 + (size_t)(jj % 8) * 16;
+                           (size_t)((jj % 16) / 8) * Sh::A_LBO + (size_t)(D / 8) * Sh::A_SBO + (size_t)(jj % 8) * 16;
         *reinterpret_cast<unsigned short*>(p) = 0x3F80u;   // bf16 1.0 at row D (element 0 of the block)
     }
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -170,96 +183,101 @@ build_states_tc_kernel(int32_t R, int32_t N, const int32_t* __restrict__ t_rowpt
 
     if (warp >= 5) {
         // ------------------------------------------------------------ producers
-        // Software pipeline over items: while item q is written to shared memory, the rows of item q+1 and
-        // the (key, Psi) pairs of item q+2 are already on their way from L2.
-        const int ptid = tid - 160;            // 0..127: key row jj = ptid / 2, half h = ptid % 2 of its pieces
-        const int jj = ptid >> 1, h = ptid & 1;
-        const uint32_t a_row = (uint32_t)(jj / 16) * Sh::A_KSTEP + (uint32_t)((jj % 16) / 8) * Sh::A_LBO + (uint32_t)(jj % 8) * 16;
-        const uint32_t b_row = (uint32_t)(jj / 16) * Sh::B_KSTEP + (uint32_t)((jj % 16) / 8) * Sh::B_LBO + (uint32_t)(jj % 8) * 16;
-        constexpr int NV = (D / 8 + 1) / 2, NK = (M / 8 + 1) / 2;
-
-        struct Walk {          // position in the CTA's item sequence
-            int32_t l, it, beg, c;
-            __device__ __forceinline__ void load(const int32_t* rp, int32_t lend) {
-                if (l < lend) { beg = __ldg(rp + l); c = __ldg(rp + l + 1) - beg; } else { beg = 0; c = 0; }
-            }
-            __device__ __forceinline__ void advance(const int32_t* rp, int32_t lend) {
-                const int32_t nitems = c > 0 ? (c + ITEM_KEYS - 1) / ITEM_KEYS : 1;
-                if (++it >= nitems) { ++l; it = 0; load(rp, lend); }
-            }
-            __device__ __forceinline__ int32_t keys() const { return min(ITEM_KEYS, c - it * ITEM_KEYS); }
+        // Producer warp w owns stage w and the items q = w, w + NW, ...: the warps work on different items, so the
+        // waits of one item (stage free, copies landed, proxy fence) overlap the copies of the others.
+        // A warp copy instruction (16 bytes per lane, asynchronous, straight into the operand layout) covers
+        // whole rows: consecutive lanes take consecutive pieces of one key's row.  The lane that copied a piece
+        // of phi(k_j) scales it by Psi_jl afterwards.  Keys and Psi values of the warp's next item are read
+        // while the current one is in flight.
+        constexpr int NW = NS;                              // one producer warp per stage (NS <= 4)
+        static_assert(NS <= 4, "more stages than producer warps");
+        const int pw = warp - 5;
+        constexpr int CV = D / 8, CK = M / 8;             // 16-byte pieces per value row / per key-feature row
+        constexpr int KPV = 32 / CV, KPK = CK >= 32 ? 1 : 32 / CK;   // keys per copy instruction
+        constexpr int NIV = ITEM_KEYS / KPV, NIK = ITEM_KEYS / KPK;  // copy instructions per item
+        static_assert(CV <= 8 && CK <= 16, "rows longer than a warp's copy");
+        auto key_offset = [](int key, int kstep_bytes, int lbo) {
+            return (uint32_t)(key / 16) * (uint32_t)kstep_bytes + (uint32_t)((key % 16) / 8) * (uint32_t)lbo +
+                   (uint32_t)(key % 8) * 16u;
         };
-        struct Idx { int32_t j; float psi; bool real; };
-        auto fetch_idx = [&](const Walk& w) {
-            Idx x; x.j = 0; x.psi = 0.0f;
-            x.real = w.l < l1 && jj < w.keys();
-            if (x.real) { x.j = __ldg(t_col + w.beg + w.it * ITEM_KEYS + jj); x.psi = __ldg(t_val + w.beg + w.it * ITEM_KEYS + jj); }
-            return x;
-        };
-        struct Rows { uint4 v[NV], k[NK]; };
-        auto fetch_rows = [&](const Idx& x) {
-            Rows r;
+        // destination of this lane's piece in instruction 0; instruction y adds key_offset(KP * y) (the
+        // offsets add up because KP divides 16)
+        const uint32_t a_lane = key_offset(lane / CV, Sh::A_KSTEP, Sh::A_LBO) + (uint32_t)(lane % CV) * Sh::A_SBO;
+        const uint32_t b_lane = key_offset(lane / CK, Sh::B_KSTEP, Sh::B_LBO) + (uint32_t)(lane % CK) * Sh::B_SBO + Sh::A_BYTES;
+        const int32_t nn = l1 - l0;
+        if (pw < NW) {
+            const int s = pw;
+            const uint32_t st = stage_base + (uint32_t)s * Sh::STAGE;
+            unsigned char* st_generic = stage_generic + (size_t)s * Sh::STAGE;
+            // walker over the CTA's items
+            int32_t wn = 0, wit = 0, wbeg = node_beg[0], wc = node_beg[1] - node_beg[0];
+            auto advance = [&]() {
+                const int32_t nitems = wc > 0 ? (wc + ITEM_KEYS - 1) / ITEM_KEYS : 1;
+                if (++wit >= nitems) { ++wn; wit = 0; wbeg = node_beg[min(wn, nn)]; wc = node_beg[min(wn + 1, nn)] - wbeg; }
+            };
+            int32_t j0, j1, nkeys; float p0, p1;
+            auto read_idx = [&](int32_t& nk, int32_t& ja, int32_t& jb, float& pa, float& pb) {
+                ja = -1; jb = -1; pa = 0.0f; pb = 0.0f; nk = 0;
+                if (wn < nn) {
+                    nk = min(ITEM_KEYS, wc - wit * ITEM_KEYS);
+                    const int32_t pos = wbeg + wit * ITEM_KEYS + lane;
+                    if (lane < nk) { ja = __ldg(t_col + pos); pa = __ldg(t_val + pos); }
+                    if (lane + 32 < nk) { jb = __ldg(t_col + pos + 32); pb = __ldg(t_val + pos + 32); }
+                }
+            };
+            for (int k = 0; k < pw; ++k) advance();
+            read_idx(nkeys, j0, j1, p0, p1);
+            bool ok = true;
+            for (uint32_t use = 0; wn < nn; ++use) {
+                const int32_t rows = nkeys > 0 ? ((nkeys + 15) & ~15) : 16;     // rows the MMAs will read
+                if (!mbar_wait(empty(s), (use & 1u) ^ 1u, &abort_flag)) ok = false;
+                ok = __all_sync(0xffffffffu, ok);
+                if (!ok) break;
 #pragma unroll
-            for (int y = 0; y < NV; ++y) r.v[y] = make_uint4(0u, 0u, 0u, 0u);
-#pragma unroll
-            for (int y = 0; y < NK; ++y) r.k[y] = make_uint4(0u, 0u, 0u, 0u);
-            if (x.real) {
-#pragma unroll
-                for (int y = 0; y < NV; ++y)
-                    if (h + 2 * y < D / 8) r.v[y] = __ldg(reinterpret_cast<const uint4*>(Vg + (size_t)x.j * D) + h + 2 * y);
-#pragma unroll
-                for (int y = 0; y < NK; ++y)
-                    if (h + 2 * y < M / 8) r.k[y] = __ldg(reinterpret_cast<const uint4*>(Kg + (size_t)x.j * M) + h + 2 * y);
-            }
-            return r;
-        };
-
-        Walk w0; w0.l = l0; w0.it = 0; w0.load(t_rowptr, l1);
-        Walk w2 = w0;
-        Idx idx_cur = fetch_idx(w2);
-        w2.advance(t_rowptr, l1);
-        Idx idx_nxt = fetch_idx(w2);
-        w2.advance(t_rowptr, l1);
-        Rows rows_cur = fetch_rows(idx_cur);
-        int32_t q = 0;
-        bool ok = true;
-        while (w0.l < l1) {
-            const Rows rows_nxt = fetch_rows(idx_nxt);        // item q+1
-            const Idx idx_nxt2 = fetch_idx(w2);               // item q+2
-            w2.advance(t_rowptr, l1);
-            const int s = q % NS;
-            const int32_t n = w0.keys();
-            const int32_t rows = n > 0 ? ((n + 15) & ~15) : 16;         // rows the MMAs will read
-            if (!mbar_wait(empty(s), ((uint32_t)(q / NS) & 1u) ^ 1u, &abort_flag)) ok = false;
-            ok = __all_sync(0xffffffffu, ok);
-            if (!ok) break;
-            if (jj < rows) {
-                unsigned char* a_dst = stage_generic + (size_t)s * Sh::STAGE + a_row;
-                unsigned char* b_dst = stage_generic + (size_t)s * Sh::STAGE + Sh::A_BYTES + b_row;
-#pragma unroll
-                for (int y = 0; y < NV; ++y)
-                    if (h + 2 * y < D / 8) *reinterpret_cast<uint4*>(a_dst + (size_t)(h + 2 * y) * 128) = rows_cur.v[y];
-#pragma unroll
-                for (int y = 0; y < NK; ++y)
-                    if (h + 2 * y < M / 8) {
-                        const uint32_t w[4] = {rows_cur.k[y].x, rows_cur.k[y].y, rows_cur.k[y].z, rows_cur.k[y].w};
-                        uint32_t r[4];
-#pragma unroll
-                        for (int e = 0; e < 4; ++e) {
-                            const float lo = idx_cur.psi * __uint_as_float(w[e] << 16);
-                            const float hi = idx_cur.psi * __uint_as_float(w[e] & 0xffff0000u);
-                            __nv_bfloat162 t2 = __floats2bfloat162_rn(lo, hi);
-                            r[e] = *reinterpret_cast<uint32_t*>(&t2);
-                        }
-                        *reinterpret_cast<uint4*>(b_dst + (size_t)(h + 2 * y) * 128) = make_uint4(r[0], r[1], r[2], r[3]);
+                for (int y = 0; y < NIV; ++y) {
+                    if (KPV * y < rows) {
+                        const int32_t j = __shfl_sync(0xffffffffu, y < NIV / 2 ? j0 : j1, (KPV * y + lane / CV) & 31);
+                        const __nv_bfloat16* src = Vg + (size_t)max(j, 0) * D + (lane % CV) * 8;
+                        asm volatile("cp.async.ca.shared.global [%0], [%1], 16, %2;"
+                                     ::"r"(st + a_lane + key_offset(KPV * y, Sh::A_KSTEP, Sh::A_LBO)), "l"(src),
+                                       "r"(j >= 0 ? 16u : 0u) : "memory");       // no such key: zero-filled
                     }
+                }
+#pragma unroll
+                for (int y = 0; y < NIK; ++y) {
+                    if (KPK * y < rows) {
+                        const int32_t j = __shfl_sync(0xffffffffu, y < NIK / 2 ? j0 : j1, (KPK * y + lane / CK) & 31);
+                        const __nv_bfloat16* src = Kg + (size_t)max(j, 0) * M + (lane % CK) * 8;
+                        asm volatile("cp.async.ca.shared.global [%0], [%1], 16, %2;"
+                                     ::"r"(st + b_lane + key_offset(KPK * y, Sh::B_KSTEP, Sh::B_LBO)), "l"(src),
+                                       "r"(j >= 0 ? 16u : 0u) : "memory");
+                    }
+                }
+                asm volatile("cp.async.commit_group;" ::: "memory");
+                // the warp's next item: keys and Psi values on their way while this one lands
+                for (int k = 0; k < NW; ++k) advance();
+                int32_t nkeys_n, jn0, jn1; float pn0, pn1;
+                read_idx(nkeys_n, jn0, jn1, pn0, pn1);
+                asm volatile("cp.async.wait_group 0;" ::: "memory");
+#pragma unroll
+                for (int y = 0; y < NIK; ++y) {
+                    if (KPK * y < rows) {
+                        const float psi = __shfl_sync(0xffffffffu, y < NIK / 2 ? p0 : p1, (KPK * y + lane / CK) & 31);
+                        const __nv_bfloat162 p2 = __float2bfloat162_rn(psi);
+                        unsigned char* pc = st_generic + b_lane + key_offset(KPK * y, Sh::B_KSTEP, Sh::B_LBO);
+                        uint4 w = *reinterpret_cast<uint4*>(pc);
+                        __nv_bfloat162* e = reinterpret_cast<__nv_bfloat162*>(&w);
+#pragma unroll
+                        for (int x = 0; x < 4; ++x) e[x] = __hmul2(e[x], p2);
+                        *reinterpret_cast<uint4*>(pc) = w;
+                    }
+                }
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                __syncwarp();
+                if (lane == 0) mbar_arrive(full(s));
+                nkeys = nkeys_n; j0 = jn0; j1 = jn1; p0 = pn0; p1 = pn1;
             }
-            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-            __syncwarp();
-            if (lane == 0) mbar_arrive(full(s));
-            ++q;
-            w0.advance(t_rowptr, l1);
-            idx_cur = idx_nxt; idx_nxt = idx_nxt2; rows_cur = rows_nxt;
+            asm volatile("cp.async.wait_all;" ::: "memory");
         }
     } else if (warp == 4) {
         // ------------------------------------------------------------ MMA issuer
@@ -283,8 +301,8 @@ build_states_tc_kernel(int32_t R, int32_t N, const int32_t* __restrict__ t_rowpt
                     const uint32_t a_op = stage_base + (uint32_t)s * Sh::STAGE;
                     const uint32_t b_op = a_op + Sh::A_BYTES;
                     for (int32_t ks = 0; ks < ksteps; ++ks) {
-                        const uint64_t ad = operand_desc(a_op + (uint32_t)ks * Sh::A_KSTEP, Sh::A_LBO, 128);
-                        const uint64_t bd = operand_desc(b_op + (uint32_t)ks * Sh::B_KSTEP, Sh::B_LBO, 128);
+                        const uint64_t ad = operand_desc(a_op + (uint32_t)ks * Sh::A_KSTEP, Sh::A_LBO, Sh::A_SBO);
+                        const uint64_t bd = operand_desc(b_op + (uint32_t)ks * Sh::B_KSTEP, Sh::B_LBO, Sh::B_SBO);
                         mma_bf16_ss(acc, ad, bd, idesc, (it > 0 || ks > 0) ? 1u : 0u);
                     }
                     mma_commit(empty(s));
@@ -372,6 +390,331 @@ int launch_state_tc(grf_ctx* ctx, const grf_csr_dev& psit, int32_t G, int32_t N,
     return cudaGetLastError() == cudaSuccess ? GRF_OK : GRF_ERR_CUDA;
 }
 
+
+// ---------------------------------------------------------------------------------------------------------
+// d = 64: the same product with the rows gathered by the tensor-map copy engine (TMA, tile::gather4: four
+// rows of a 2-D tensor per instruction, row indices given in registers), so the gather does not pass through
+// the load/store units.  A gathered v_j row is 128 bytes: 64 rows stacked at a 128-byte pitch, written with
+// the 128-byte swizzle, ARE the MN-major swizzled operand (8 keys x 128 bytes per swizzle atom).  The second
+// atom along M (rows 64..127: the ones row that yields z_l, then zeros) is one constant region shared by all
+// stages, reached through the descriptor's leading-dimension offset.  phi(k_j) rows (2m bytes) are gathered
+// the same way with the 32/64/128-byte swizzle that matches their length, then scaled in place by Psi_jl.
+template <int M> struct TmaShape {
+    static constexpr int D = 64;
+    static constexpr int A_BYTES = ITEM_KEYS * 128;             // gathered value rows of an item
+    static constexpr int B_PITCH = M * 2;
+    static constexpr int B_BYTES = ITEM_KEYS * B_PITCH;
+    static constexpr int STAGE = A_BYTES + B_BYTES;
+    static constexpr int NS = 4;                                // one stage per producer warp
+    static constexpr int B_SBO = 8 * B_PITCH;
+    static constexpr uint64_t B_LAYOUT = M == 16 ? 6 : (M == 32 ? 4 : 2);   // 32-, 64-, 128-byte swizzle
+    static constexpr int ACC_COLS = M < 32 ? 32 : M;
+    static constexpr int TMEM_COLS = 2 * ACC_COLS < 32 ? 32 : 2 * ACC_COLS;
+    static constexpr size_t SMEM = (size_t)NS * STAGE + A_BYTES + 1024;
+    static_assert(STAGE % 1024 == 0, "stages must keep the swizzle phase");
+};
+
+__device__ __forceinline__ uint64_t swizzled_desc(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes, uint64_t layout)
+{
+    uint64_t d = (uint64_t)((saddr & 0x3FFFFu) >> 4);
+    d |= (uint64_t)((lbo_bytes >> 4) & 0x3FFFu) << 16;
+    d |= (uint64_t)((sbo_bytes >> 4) & 0x3FFFu) << 32;
+    d |= (uint64_t)1 << 46;
+    d |= layout << 61;
+    return d;
+}
+__device__ __forceinline__ void tma_gather4(uint32_t dst, const CUtensorMap* map, int32_t r0, int32_t r1, int32_t r2,
+                                            int32_t r3, uint32_t bar)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.tile::gather4.mbarrier::complete_tx::bytes"
+        " [%0], [%1, {%2, %3, %4, %5, %6}], [%7];"
+        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(0), "r"(r0), "r"(r1), "r"(r2), "r"(r3), "r"(bar)
+        : "memory");
+}
+
+template <int M>
+__global__ void __launch_bounds__(ST_THREADS)
+build_states_tma_kernel(int32_t R, int32_t N, const int32_t* __restrict__ t_rowptr, const int32_t* __restrict__ t_col,
+                        const float* __restrict__ t_val, const __grid_constant__ CUtensorMap map_k,
+                        const __grid_constant__ CUtensorMap map_v, unsigned char* __restrict__ records,
+                        int* __restrict__ error_word)
+{
+    using Sh = TmaShape<M>;
+    constexpr int NS = Sh::NS, D = Sh::D;
+    extern __shared__ unsigned char smem_dyn[];
+    __shared__ __align__(8) unsigned long long bars[3 * NS + 4];   // landed, full, empty per stage; acc_full[2], acc_free[2]
+    __shared__ uint32_t tmem_slot;
+    __shared__ int abort_flag;
+    __shared__ int32_t node_beg[NODES_PER_CTA + 1];
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int32_t g = blockIdx.y;
+    const int32_t l0 = blockIdx.x * NODES_PER_CTA, l1 = min(R, l0 + NODES_PER_CTA);
+    const uint32_t stage_base = (smem_u32(smem_dyn) + 1023u) & ~1023u;
+    unsigned char* stage_generic = smem_dyn + (stage_base - smem_u32(smem_dyn));
+    const uint32_t const_base = stage_base + (uint32_t)NS * Sh::STAGE;     // the constant second atom of A
+    const uint32_t bar_base = smem_u32(bars);
+    auto landed = [&](int s) { return bar_base + 8u * (uint32_t)s; };
+    auto full = [&](int s) { return bar_base + 8u * (uint32_t)(NS + s); };
+    auto empty = [&](int s) { return bar_base + 8u * (uint32_t)(2 * NS + s); };
+    auto acc_full = [&](int b) { return bar_base + 8u * (uint32_t)(3 * NS + b); };
+    auto acc_free = [&](int b) { return bar_base + 8u * (uint32_t)(3 * NS + 2 + b); };
+
+    if (tid == 0) {
+        for (int s = 0; s < NS; ++s) { mbar_init(landed(s), 1); mbar_init(full(s), 1); mbar_init(empty(s), 1); }
+        for (int b = 0; b < 2; ++b) { mbar_init(acc_full(b), 1); mbar_init(acc_free(b), 4); }
+        abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 4) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                     ::"r"(smem_u32(&tmem_slot)), "r"((uint32_t)Sh::TMEM_COLS) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    if (tid <= NODES_PER_CTA) node_beg[tid] = t_rowptr[min(l0 + tid, R)];
+    // stages start as zeros (pad rows are multiplied before they are ever written); the constant atom is zero
+    // except for bf16 1.0 in element 0 of logical piece 0 of every key row, which the swizzle puts at piece r % 8
+    for (int x = tid; x < (NS * Sh::STAGE + Sh::A_BYTES) / 16; x += ST_THREADS)
+        *reinterpret_cast<uint4*>(stage_generic + (size_t)x * 16) = make_uint4(0u, 0u, 0u, 0u);
+    __syncthreads();
+    for (int r = tid; r < ITEM_KEYS; r += ST_THREADS)
+        *reinterpret_cast<unsigned short*>(stage_generic + (size_t)NS * Sh::STAGE + (size_t)r * 128 + (size_t)(r % 8) * 16) = 0x3F80u;
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const uint32_t tmem_base = tmem_slot;
+
+    if (warp >= 5) {
+        // ------------------------------------------------------------ producers: warp w owns stage w, items w, w+4, ...
+        const int s = warp - 5;
+        const int32_t nn = l1 - l0;
+        const uint32_t st = stage_base + (uint32_t)s * Sh::STAGE;
+        unsigned char* st_generic = stage_generic + (size_t)s * Sh::STAGE;
+        constexpr int CK = M / 8;                         // 16-byte pieces of a phi(k_j) row
+        const int y4 = lane & 15;                         // this lane gathers keys 4*y4 .. 4*y4+3 ...
+        const bool is_k = lane >= 16;                     // ... of phi(K) (lanes 16-31) or of V (lanes 0-15)
+        const int32_t row0 = g * N;
+        int32_t wn = 0, wit = 0, wbeg = node_beg[0], wc = node_beg[1] - node_beg[0];
+        auto advance = [&]() {
+            const int32_t nitems = wc > 0 ? (wc + ITEM_KEYS - 1) / ITEM_KEYS : 1;
+            if (++wit >= nitems) { ++wn; wit = 0; wbeg = node_beg[min(wn, nn)]; wc = node_beg[min(wn + 1, nn)] - wbeg; }
+        };
+        struct Idx { int32_t nkeys, j[4]; float p0, p1; };
+        auto read_idx = [&]() {
+            Idx x; x.nkeys = 0; x.p0 = 0.0f; x.p1 = 0.0f;
+#pragma unroll
+            for (int e = 0; e < 4; ++e) x.j[e] = 0;
+            if (wn < nn) {
+                x.nkeys = min(ITEM_KEYS, wc - wit * ITEM_KEYS);
+                const int32_t pos = wbeg + wit * ITEM_KEYS;
+                if (x.nkeys > 0) {
+#pragma unroll
+                    for (int e = 0; e < 4; ++e)      // beyond the item's keys: repeat its last key (the row is zeroed later)
+                        x.j[e] = __ldg(t_col + pos + min(4 * y4 + e, x.nkeys - 1));
+                }
+                if (lane < x.nkeys) x.p0 = __ldg(t_val + pos + lane);
+                if (lane + 32 < x.nkeys) x.p1 = __ldg(t_val + pos + lane + 32);
+            }
+            return x;
+        };
+        for (int k = 0; k < s; ++k) advance();
+        Idx cur = read_idx();
+        bool ok = true;
+        for (uint32_t use = 0; wn < nn; ++use) {
+            const int32_t rows = cur.nkeys > 0 ? ((cur.nkeys + 15) & ~15) : 16;     // rows the MMAs will read
+            if (!mbar_wait(empty(s), (use & 1u) ^ 1u, &abort_flag)) ok = false;
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
+            if (lane == 0)
+                asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;"
+                             ::"r"(landed(s)), "r"((uint32_t)rows * (128u + (uint32_t)Sh::B_PITCH)) : "memory");
+            __syncwarp();
+            if (4 * y4 < rows) {
+                if (is_k) tma_gather4(st + Sh::A_BYTES + (uint32_t)y4 * 4u * Sh::B_PITCH, &map_k, row0 + cur.j[0], row0 + cur.j[1],
+                                      row0 + cur.j[2], row0 + cur.j[3], landed(s));
+                else tma_gather4(st + (uint32_t)y4 * 512u, &map_v, row0 + cur.j[0], row0 + cur.j[1], row0 + cur.j[2],
+                                 row0 + cur.j[3], landed(s));
+            }
+            // the warp's next item: keys and Psi values on their way while this one lands
+            for (int k = 0; k < NS; ++k) advance();
+            const Idx nxt = read_idx();
+            if (!mbar_wait(landed(s), use & 1u, &abort_flag)) ok = false;
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
+            // Psi_jl * phi(k_j), in place: a lane takes 16-byte pieces lane, lane + 32, ... of the item's rows
+#pragma unroll
+            for (int y = 0; y < 2 * CK; ++y) {
+                const int row = (32 * y + lane) / CK;
+                const float psi = __shfl_sync(0xffffffffu, y < CK ? cur.p0 : cur.p1, row & 31);
+                if (row < rows) {
+                    unsigned char* pc = st_generic + Sh::A_BYTES + (size_t)(32 * y + lane) * 16;
+                    uint4 w = make_uint4(0u, 0u, 0u, 0u);
+                    if (row < cur.nkeys) {
+                        const __nv_bfloat162 p2 = __float2bfloat162_rn(psi);
+                        w = *reinterpret_cast<uint4*>(pc);
+                        __nv_bfloat162* e = reinterpret_cast<__nv_bfloat162*>(&w);
+#pragma unroll
+                        for (int x = 0; x < 4; ++x) e[x] = __hmul2(e[x], p2);
+                    }
+                    *reinterpret_cast<uint4*>(pc) = w;
+                }
+            }
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            __syncwarp();
+            if (lane == 0) mbar_arrive(full(s));
+            cur = nxt;
+        }
+        if (!ok) {
+            // aborted: give copies that may still be in flight time to land before the CTA's memory is released
+            const long long t0 = clock64();
+            while (clock64() - t0 < 2000000ll) {}
+        }
+    } else if (warp == 4) {
+        // ------------------------------------------------------------ MMA issuer
+        constexpr uint32_t idesc = instr_desc_mn(M);
+        int32_t q = 0, nn = 0;
+        bool ok = true;
+        for (int32_t l = l0; l < l1 && ok; ++l, ++nn) {
+            const int32_t c = node_beg[l - l0 + 1] - node_beg[l - l0];
+            const int32_t nitems = c > 0 ? (c + ITEM_KEYS - 1) / ITEM_KEYS : 1;
+            const int buf = nn & 1;
+            if (!mbar_wait(acc_free(buf), ((uint32_t)(nn >> 1) & 1u) ^ 1u, &abort_flag)) { ok = false; break; }
+            const uint32_t acc = tmem_base + (uint32_t)(buf * Sh::ACC_COLS);
+            for (int32_t it = 0; it < nitems; ++it, ++q) {
+                const int s = q % NS;
+                const int32_t n = min(ITEM_KEYS, c - it * ITEM_KEYS);
+                const int32_t ksteps = n > 0 ? (n + 15) / 16 : 1;
+                if (!mbar_wait(full(s), (uint32_t)(q / NS) & 1u, &abort_flag)) { ok = false; break; }
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                if (lane == 0) {
+                    const uint32_t a_op = stage_base + (uint32_t)s * Sh::STAGE;
+                    const uint32_t b_op = a_op + Sh::A_BYTES;
+                    for (int32_t ks = 0; ks < ksteps; ++ks) {
+                        // A: two atoms along M (gathered rows, then the constant atom), 8-key groups 1024 bytes apart
+                        const uint64_t ad = swizzled_desc(a_op + (uint32_t)ks * 2048u, const_base - a_op, 1024u, 2);
+                        const uint64_t bd = swizzled_desc(b_op + (uint32_t)ks * 16u * Sh::B_PITCH, 16u, Sh::B_SBO, Sh::B_LAYOUT);
+                        mma_bf16_ss(acc, ad, bd, idesc, (it > 0 || ks > 0) ? 1u : 0u);
+                    }
+                    mma_commit(empty(s));
+                    if (it == nitems - 1) mma_commit(acc_full(buf));
+                }
+                __syncwarp();
+            }
+        }
+        if (!ok) {
+            const long long t0 = clock64();
+            while (clock64() - t0 < 2000000ll) {}
+        }
+    } else {
+        // ------------------------------------------------------------ epilogue: accumulator -> record
+        constexpr size_t REC = grf_record_bytes<__nv_bfloat16>(M, D);
+        const int row = warp * 32 + lane;                   // accumulator row = TMEM lane
+        const bool warp_has_rows = warp * 32 <= D;          // S rows 0..D-1 and the z row D
+        int32_t nn = 0;
+        bool ok = true;
+        for (int32_t l = l0; l < l1; ++l, ++nn) {
+            const int buf = nn & 1;
+            if (ok && !mbar_wait(acc_full(buf), (uint32_t)(nn >> 1) & 1u, &abort_flag)) ok = false;
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            if (warp_has_rows) {
+                unsigned char* rec = records + ((size_t)g * R + l) * REC;
+                __nv_bfloat16* tile = reinterpret_cast<__nv_bfloat16*>(rec);
+                float* zl = reinterpret_cast<float*>(rec + (size_t)M * D * 2);
+                const uint32_t taddr = tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)(buf * Sh::ACC_COLS);
+#pragma unroll
+                for (int c0 = 0; c0 < M; c0 += 16) {
+                    uint32_t r[16];
+                    tmem_ld16(taddr + (uint32_t)c0, r);
+                    if (row < D) {
+#pragma unroll
+                        for (int half = 0; half < 2; ++half) {
+                            uint32_t w[4];
+#pragma unroll
+                            for (int e = 0; e < 4; ++e) {
+                                __nv_bfloat162 t2 = __floats2bfloat162_rn(__uint_as_float(r[8 * half + 2 * e]),
+                                                                          __uint_as_float(r[8 * half + 2 * e + 1]));
+                                w[e] = *reinterpret_cast<uint32_t*>(&t2);
+                            }
+                            *reinterpret_cast<uint4*>(tile + grf_tile_index<__nv_bfloat16>(c0 + 8 * half, row, D)) =
+                                make_uint4(w[0], w[1], w[2], w[3]);
+                        }
+                    } else if (row == D) {
+#pragma unroll
+                        for (int e = 0; e < 16; e += 4)
+                            *reinterpret_cast<float4*>(zl + c0 + e) = make_float4(__uint_as_float(r[e]), __uint_as_float(r[e + 1]),
+                                                                                  __uint_as_float(r[e + 2]), __uint_as_float(r[e + 3]));
+                    }
+                }
+            }
+            asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+            __syncwarp();
+            if (lane == 0) mbar_arrive(acc_free(buf));
+        }
+    }
+
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    if (warp == 4) {
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)Sh::TMEM_COLS) : "memory");
+    }
+    if (tid == 0 && abort_flag) atomicExch(error_word, 1);
+}
+
+// cuTensorMapEncodeTiled, looked up through the runtime (the library does not link the driver directly)
+typedef CUresult (*encode_tiled_fn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                    const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                    CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+encode_tiled_fn tensor_map_encoder()
+{
+    static encode_tiled_fn fn = []() -> encode_tiled_fn {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) != cudaSuccess ||
+            qres != cudaDriverEntryPointSuccess)
+            return nullptr;
+        return reinterpret_cast<encode_tiled_fn>(p);
+    }();
+    return fn;
+}
+// A [rows x cols] bf16 matrix whose rows are gathered one at a time (box = one row of at most 64 elements).
+bool make_row_gather_map(CUtensorMap* map, const void* base, uint64_t rows, uint32_t cols)
+{
+    encode_tiled_fn enc = tensor_map_encoder();
+    if (!enc || (reinterpret_cast<uintptr_t>(base) & 15u) != 0) return false;
+    const cuuint64_t dims[2] = {cols, rows};
+    const cuuint64_t strides[1] = {(cuuint64_t)cols * 2};
+    const cuuint32_t box[2] = {cols, 1};
+    const cuuint32_t estr[2] = {1, 1};
+    const CUtensorMapSwizzle sw = cols * 2 == 32 ? CU_TENSOR_MAP_SWIZZLE_32B
+                                : (cols * 2 == 64 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_128B);
+    return enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, sw, CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// 1 when the tensor maps cannot be made (the caller then takes the kernel above)
+template <int M>
+int launch_state_tma(grf_ctx* ctx, const grf_csr_dev& psit, int32_t G, int32_t N, const void* phiK, const void* V,
+                     void* records)
+{
+    using Sh = TmaShape<M>;
+    if ((int64_t)G * N > 0x7fffffffll) return 1;
+    CUtensorMap map_k, map_v;
+    if (!make_row_gather_map(&map_k, phiK, (uint64_t)G * N, M) || !make_row_gather_map(&map_v, V, (uint64_t)G * N, 64)) return 1;
+    GRF_CUDA_TRY(cudaFuncSetAttribute(build_states_tma_kernel<M>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Sh::SMEM));
+    const dim3 grid(grf_ceil_div(psit.rows, NODES_PER_CTA), G);
+    {
+        grf_launch_scope scope(ctx, 4);
+        build_states_tma_kernel<M><<<grid, ST_THREADS, Sh::SMEM, ctx->stream>>>(
+            psit.rows, N, (const int32_t*)psit.rowptr.ptr, (const int32_t*)psit.col.ptr, (const float*)psit.val.ptr,
+            map_k, map_v, (unsigned char*)records, ctx->error_word);
+    }
+    return cudaGetLastError() == cudaSuccess ? GRF_OK : GRF_ERR_CUDA;
+}
+
 }  // namespace
 
 // Returns GRF_OK after launching, or 1 when this shape has no tensor-core path (the caller falls back).
@@ -379,6 +722,12 @@ int grf_build_states_tc(grf_ctx* ctx, const grf_csr_dev& psit, int32_t G, int32_
                         const void* phiK, const void* V, void* records)
 {
     if (G > 65535) return 1;
+    if (d == 64 && (m == 16 || m == 32 || m == 64)) {
+        const int rc = m == 16 ? launch_state_tma<16>(ctx, psit, G, N, phiK, V, records)
+                     : m == 32 ? launch_state_tma<32>(ctx, psit, G, N, phiK, V, records)
+                               : launch_state_tma<64>(ctx, psit, G, N, phiK, V, records);
+        if (rc != 1) return rc;
+    }
 #define GRF_ST_CASE(MM, DD) \
     if (m == MM && d == DD) return launch_state_tc<MM, DD>(ctx, psit, G, N, phiK, V, records);
     GRF_ST_CASE(16, 16) GRF_ST_CASE(16, 32) GRF_ST_CASE(16, 64)

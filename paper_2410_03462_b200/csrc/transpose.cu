@@ -77,8 +77,12 @@ int grf_transpose_launch(grf_ctx* ctx, int32_t rows, int32_t cols, int64_t nnz,
     if (nnz >= (1ll << 31)) return GRF_ERR_TOO_LARGE;
     // scratch: per-column counts, later the scatter cursors; and the unordered buckets
     GRF_TRY(grf_buf_reserve(&ctx->t_cursor, sizeof(int32_t) * ((size_t)cols + 1)));
-    GRF_TRY(grf_buf_reserve(&ctx->t_tmp_col, sizeof(int32_t) * (size_t)(nnz > 0 ? nnz : 1)));
-    GRF_TRY(grf_buf_reserve(&ctx->t_tmp_val, sizeof(float) * (size_t)(nnz > 0 ? nnz : 1)));
+    // grown with head-room: resampling changes nnz a little every time, and a reallocation stalls the stream
+    if (ctx->t_tmp_col.bytes < sizeof(int32_t) * (size_t)nnz || ctx->t_tmp_val.bytes < sizeof(float) * (size_t)nnz) {
+        const size_t cap = (size_t)nnz + (size_t)nnz / 8 + 64;
+        GRF_TRY(grf_buf_reserve(&ctx->t_tmp_col, sizeof(int32_t) * cap));
+        GRF_TRY(grf_buf_reserve(&ctx->t_tmp_val, sizeof(float) * cap));
+    }
     int32_t* cursor = (int32_t*)ctx->t_cursor.ptr;
     GRF_CUDA_TRY(cudaMemsetAsync(cursor, 0, sizeof(int32_t) * ((size_t)cols + 1), ctx->stream));
     if (nnz > 0) {
