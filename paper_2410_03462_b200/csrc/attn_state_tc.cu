@@ -397,17 +397,19 @@ int launch_state_tc(grf_ctx* ctx, const grf_csr_dev& psit, int32_t G, int32_t N,
 // the load/store units.  A gathered v_j row is 128 bytes: 64 rows stacked at a 128-byte pitch, written with
 // the 128-byte swizzle, ARE the MN-major swizzled operand (8 keys x 128 bytes per swizzle atom).  The second
 // atom along M (rows 64..127: the ones row that yields z_l, then zeros) is one constant region shared by all
-// stages, reached through the descriptor's leading-dimension offset.  phi(k_j) rows (2m bytes) are gathered
-// the same way with the 32/64/128-byte swizzle that matches their length, then scaled in place by Psi_jl.
+// stages, reached through the descriptor's leading-dimension offset.  The copy engine sustains about one
+// four-row gather per 15 cycles per SM whatever the rows' length, so the shorter phi(k_j) rows do not go
+// through it as well: they travel as asynchronous 16-byte copies through the load/store units (which would
+// otherwise idle) into the padded unswizzled layout of the kernel above, and are scaled in place by Psi_jl.
 template <int M> struct TmaShape {
     static constexpr int D = 64;
     static constexpr int A_BYTES = ITEM_KEYS * 128;             // gathered value rows of an item
-    static constexpr int B_PITCH = M * 2;
-    static constexpr int B_BYTES = ITEM_KEYS * B_PITCH;
+    static constexpr int B_SBO = StShape<M, 64>::B_SBO;
+    static constexpr int B_LBO = (M / 8) * B_SBO;
+    static constexpr int B_KSTEP = 2 * B_LBO;
+    static constexpr int B_BYTES = (ITEM_KEYS / 16) * B_KSTEP;
     static constexpr int STAGE = A_BYTES + B_BYTES;
     static constexpr int NS = 4;                                // one stage per producer warp
-    static constexpr int B_SBO = 8 * B_PITCH;
-    static constexpr uint64_t B_LAYOUT = M == 16 ? 6 : (M == 32 ? 4 : 2);   // 32-, 64-, 128-byte swizzle
     static constexpr int ACC_COLS = M < 32 ? 32 : M;
     static constexpr int TMEM_COLS = 2 * ACC_COLS < 32 ? 32 : 2 * ACC_COLS;
     static constexpr size_t SMEM = (size_t)NS * STAGE + A_BYTES + 1024;
@@ -436,7 +438,7 @@ __device__ __forceinline__ void tma_gather4(uint32_t dst, const CUtensorMap* map
 template <int M>
 __global__ void __launch_bounds__(ST_THREADS)
 build_states_tma_kernel(int32_t R, int32_t N, const int32_t* __restrict__ t_rowptr, const int32_t* __restrict__ t_col,
-                        const float* __restrict__ t_val, const __grid_constant__ CUtensorMap map_k,
+                        const float* __restrict__ t_val, const __nv_bfloat16* __restrict__ phiK,
                         const __grid_constant__ CUtensorMap map_v, unsigned char* __restrict__ records,
                         int* __restrict__ error_word)
 {
@@ -493,17 +495,24 @@ build_states_tma_kernel(int32_t R, int32_t N, const int32_t* __restrict__ t_rowp
         const uint32_t st = stage_base + (uint32_t)s * Sh::STAGE;
         unsigned char* st_generic = stage_generic + (size_t)s * Sh::STAGE;
         constexpr int CK = M / 8;                         // 16-byte pieces of a phi(k_j) row
-        const int y4 = lane & 15;                         // this lane gathers keys 4*y4 .. 4*y4+3 ...
-        const bool is_k = lane >= 16;                     // ... of phi(K) (lanes 16-31) or of V (lanes 0-15)
+        constexpr int KPK = 32 / CK, NIK = ITEM_KEYS / KPK;   // keys per copy instruction, instructions per item
+        const int y4 = lane & 15;                         // lanes 0-15 gather the value rows of keys 4*y4 .. 4*y4+3
         const int32_t row0 = g * N;
+        auto key_offset = [](int key) {
+            return (uint32_t)(key / 16) * (uint32_t)Sh::B_KSTEP + (uint32_t)((key % 16) / 8) * (uint32_t)Sh::B_LBO +
+                   (uint32_t)(key % 8) * 16u;
+        };
+        // this lane's piece of phi(k_j) in copy instruction 0; instruction y adds key_offset(KPK * y)
+        const uint32_t b_lane = Sh::A_BYTES + key_offset(lane / CK) + (uint32_t)(lane % CK) * Sh::B_SBO;
+        const __nv_bfloat16* Kg = phiK + (size_t)g * N * M + (lane % CK) * 8;
         int32_t wn = 0, wit = 0, wbeg = node_beg[0], wc = node_beg[1] - node_beg[0];
         auto advance = [&]() {
             const int32_t nitems = wc > 0 ? (wc + ITEM_KEYS - 1) / ITEM_KEYS : 1;
             if (++wit >= nitems) { ++wn; wit = 0; wbeg = node_beg[min(wn, nn)]; wc = node_beg[min(wn + 1, nn)] - wbeg; }
         };
-        struct Idx { int32_t nkeys, j[4]; float p0, p1; };
+        struct Idx { int32_t nkeys, j[4], jlo, jhi; float p0, p1; };
         auto read_idx = [&]() {
-            Idx x; x.nkeys = 0; x.p0 = 0.0f; x.p1 = 0.0f;
+            Idx x; x.nkeys = 0; x.p0 = 0.0f; x.p1 = 0.0f; x.jlo = -1; x.jhi = -1;
 #pragma unroll
             for (int e = 0; e < 4; ++e) x.j[e] = 0;
             if (wn < nn) {
@@ -511,11 +520,11 @@ build_states_tma_kernel(int32_t R, int32_t N, const int32_t* __restrict__ t_rowp
                 const int32_t pos = wbeg + wit * ITEM_KEYS;
                 if (x.nkeys > 0) {
 #pragma unroll
-                    for (int e = 0; e < 4; ++e)      // beyond the item's keys: repeat its last key (the row is zeroed later)
+                    for (int e = 0; e < 4; ++e)      // beyond the item's keys: repeat its last key (it meets a zero row)
                         x.j[e] = __ldg(t_col + pos + min(4 * y4 + e, x.nkeys - 1));
                 }
-                if (lane < x.nkeys) x.p0 = __ldg(t_val + pos + lane);
-                if (lane + 32 < x.nkeys) x.p1 = __ldg(t_val + pos + lane + 32);
+                if (lane < x.nkeys) { x.jlo = __ldg(t_col + pos + lane); x.p0 = __ldg(t_val + pos + lane); }
+                if (lane + 32 < x.nkeys) { x.jhi = __ldg(t_col + pos + lane + 32); x.p1 = __ldg(t_val + pos + lane + 32); }
             }
             return x;
         };
@@ -529,43 +538,53 @@ build_states_tma_kernel(int32_t R, int32_t N, const int32_t* __restrict__ t_rowp
             if (!ok) break;
             if (lane == 0)
                 asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;"
-                             ::"r"(landed(s)), "r"((uint32_t)rows * (128u + (uint32_t)Sh::B_PITCH)) : "memory");
+                             ::"r"(landed(s)), "r"((uint32_t)rows * 128u) : "memory");
             __syncwarp();
-            if (4 * y4 < rows) {
-                if (is_k) tma_gather4(st + Sh::A_BYTES + (uint32_t)y4 * 4u * Sh::B_PITCH, &map_k, row0 + cur.j[0], row0 + cur.j[1],
-                                      row0 + cur.j[2], row0 + cur.j[3], landed(s));
-                else tma_gather4(st + (uint32_t)y4 * 512u, &map_v, row0 + cur.j[0], row0 + cur.j[1], row0 + cur.j[2],
-                                 row0 + cur.j[3], landed(s));
+            if (lane < 16 && 4 * y4 < rows)
+                tma_gather4(st + (uint32_t)y4 * 512u, &map_v, row0 + cur.j[0], row0 + cur.j[1], row0 + cur.j[2],
+                            row0 + cur.j[3], landed(s));
+#pragma unroll
+            for (int y = 0; y < NIK; ++y) {
+                const int32_t j = __shfl_sync(0xffffffffu, y < NIK / 2 ? cur.jlo : cur.jhi, (KPK * y + lane / CK) & 31);
+                if (KPK * y < rows)
+                    asm volatile("cp.async.ca.shared.global [%0], [%1], 16, %2;"
+                                 ::"r"(st + b_lane + key_offset(KPK * y)), "l"(Kg + (size_t)max(j, 0) * M),
+                                   "r"(j >= 0 ? 16u : 0u) : "memory");       // no such key: zero-filled
             }
+            asm volatile("cp.async.commit_group;" ::: "memory");
             // the warp's next item: keys and Psi values on their way while this one lands
             for (int k = 0; k < NS; ++k) advance();
             const Idx nxt = read_idx();
+            asm volatile("cp.async.wait_group 0;" ::: "memory");
+            // Psi_jl * phi(k_j), in place: every lane scales the pieces it copied
+            constexpr int BATCH = NIK < 8 ? NIK : 8;
+#pragma unroll
+            for (int y0 = 0; y0 < NIK; y0 += BATCH) {
+                uint4 w[BATCH];
+#pragma unroll
+                for (int u = 0; u < BATCH; ++u)
+                    w[u] = *reinterpret_cast<const uint4*>(st_generic + b_lane + key_offset(KPK * (y0 + u)));
+#pragma unroll
+                for (int u = 0; u < BATCH; ++u) {
+                    const float psi = __shfl_sync(0xffffffffu, y0 + u < NIK / 2 ? cur.p0 : cur.p1, (KPK * (y0 + u) + lane / CK) & 31);
+                    const __nv_bfloat162 p2 = __float2bfloat162_rn(psi);
+                    __nv_bfloat162* e = reinterpret_cast<__nv_bfloat162*>(&w[u]);
+#pragma unroll
+                    for (int x = 0; x < 4; ++x) e[x] = __hmul2(e[x], p2);
+                }
+#pragma unroll
+                for (int u = 0; u < BATCH; ++u)
+                    if (KPK * (y0 + u) < rows) *reinterpret_cast<uint4*>(st_generic + b_lane + key_offset(KPK * (y0 + u))) = w[u];
+            }
             if (!mbar_wait(landed(s), use & 1u, &abort_flag)) ok = false;
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
-            // Psi_jl * phi(k_j), in place: a lane takes 16-byte pieces lane, lane + 32, ... of the item's rows
-#pragma unroll
-            for (int y = 0; y < 2 * CK; ++y) {
-                const int row = (32 * y + lane) / CK;
-                const float psi = __shfl_sync(0xffffffffu, y < CK ? cur.p0 : cur.p1, row & 31);
-                if (row < rows) {
-                    unsigned char* pc = st_generic + Sh::A_BYTES + (size_t)(32 * y + lane) * 16;
-                    uint4 w = make_uint4(0u, 0u, 0u, 0u);
-                    if (row < cur.nkeys) {
-                        const __nv_bfloat162 p2 = __float2bfloat162_rn(psi);
-                        w = *reinterpret_cast<uint4*>(pc);
-                        __nv_bfloat162* e = reinterpret_cast<__nv_bfloat162*>(&w);
-#pragma unroll
-                        for (int x = 0; x < 4; ++x) e[x] = __hmul2(e[x], p2);
-                    }
-                    *reinterpret_cast<uint4*>(pc) = w;
-                }
-            }
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
             __syncwarp();
             if (lane == 0) mbar_arrive(full(s));
             cur = nxt;
         }
+        asm volatile("cp.async.wait_all;" ::: "memory");
         if (!ok) {
             // aborted: give copies that may still be in flight time to land before the CTA's memory is released
             const long long t0 = clock64();
@@ -594,7 +613,7 @@ build_states_tma_kernel(int32_t R, int32_t N, const int32_t* __restrict__ t_rowp
                     for (int32_t ks = 0; ks < ksteps; ++ks) {
                         // A: two atoms along M (gathered rows, then the constant atom), 8-key groups 1024 bytes apart
                         const uint64_t ad = swizzled_desc(a_op + (uint32_t)ks * 2048u, const_base - a_op, 1024u, 2);
-                        const uint64_t bd = swizzled_desc(b_op + (uint32_t)ks * 16u * Sh::B_PITCH, 16u, Sh::B_SBO, Sh::B_LAYOUT);
+                        const uint64_t bd = operand_desc(b_op + (uint32_t)ks * Sh::B_KSTEP, Sh::B_LBO, Sh::B_SBO);
                         mma_bf16_ss(acc, ad, bd, idesc, (it > 0 || ks > 0) ? 1u : 0u);
                     }
                     mma_commit(empty(s));
@@ -702,15 +721,15 @@ int launch_state_tma(grf_ctx* ctx, const grf_csr_dev& psit, int32_t G, int32_t N
 {
     using Sh = TmaShape<M>;
     if ((int64_t)G * N > 0x7fffffffll) return 1;
-    CUtensorMap map_k, map_v;
-    if (!make_row_gather_map(&map_k, phiK, (uint64_t)G * N, M) || !make_row_gather_map(&map_v, V, (uint64_t)G * N, 64)) return 1;
+    CUtensorMap map_v;
+    if ((reinterpret_cast<uintptr_t>(phiK) & 15u) != 0 || !make_row_gather_map(&map_v, V, (uint64_t)G * N, 64)) return 1;
     GRF_CUDA_TRY(cudaFuncSetAttribute(build_states_tma_kernel<M>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Sh::SMEM));
     const dim3 grid(grf_ceil_div(psit.rows, NODES_PER_CTA), G);
     {
         grf_launch_scope scope(ctx, 4);
         build_states_tma_kernel<M><<<grid, ST_THREADS, Sh::SMEM, ctx->stream>>>(
             psit.rows, N, (const int32_t*)psit.rowptr.ptr, (const int32_t*)psit.col.ptr, (const float*)psit.val.ptr,
-            map_k, map_v, (unsigned char*)records, ctx->error_word);
+            (const __nv_bfloat16*)phiK, map_v, (unsigned char*)records, ctx->error_word);
     }
     return cudaGetLastError() == cudaSuccess ? GRF_OK : GRF_ERR_CUDA;
 }
