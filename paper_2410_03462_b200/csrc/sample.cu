@@ -3,8 +3,9 @@
 // One warp owns one feature row (ensemble e, source node i); its lanes are walkers.  Every decision
 // of a walk is integer (Philox words against a threshold, multiply-high neighbour pick), the load is
 // fp32 with a fixed operation order, so the walks do not depend on the launch geometry.  Deposits
-// stay in shared memory: the warp sorts them by (column, walk, step) with a bitonic network, adds
-// equal columns in that order and writes the merged row once.
+// stay in shared memory: the warp sorts their keys by (column, walk, step) with a bitonic network (in
+// registers and shuffles for rows of up to 512 deposits), adds equal columns in that order and writes the
+// merged row once.
 #include <new>
 
 #include "grf_internal.cuh"
@@ -59,6 +60,44 @@ struct Walker {
     }
 };
 
+// Bitonic sort of 32 * E keys held E per lane (key x = lane * E + r sits in register r of its lane): partners
+// closer than E are registers of the same lane, the others are reached with one shuffle.  Same network as
+// the shared-memory loop it replaces, so the result is the same sorted row.
+template <int E>
+__device__ __forceinline__ void sort_in_registers(uint32_t* keys, int lane)
+{
+    uint32_t v[E];
+#pragma unroll
+    for (int r = 0; r < E; ++r) v[r] = keys[lane * E + r];
+#pragma unroll
+    for (int k = 2; k <= 32 * E; k <<= 1) {
+#pragma unroll
+        for (int j = k >> 1; j > 0; j >>= 1) {
+            if (j >= E) {
+                const int lj = j / E;
+                const bool keep_min = ((lane & lj) == 0) == (((lane * E) & k) == 0);
+#pragma unroll
+                for (int r = 0; r < E; ++r) {
+                    const uint32_t p = __shfl_xor_sync(0xffffffffu, v[r], lj);
+                    v[r] = keep_min ? min(v[r], p) : max(v[r], p);
+                }
+            } else {
+#pragma unroll
+                for (int r = 0; r < E; ++r) {
+                    if ((r & j) == 0) {
+                        const bool up = k < E ? (r & k) == 0 : ((lane * E) & k) == 0;
+                        const uint32_t mn = min(v[r], v[r | j]), mx = max(v[r], v[r | j]);
+                        v[r] = up ? mn : mx;
+                        v[r | j] = up ? mx : mn;
+                    }
+                }
+            }
+        }
+    }
+#pragma unroll
+    for (int r = 0; r < E; ++r) keys[lane * E + r] = v[r];
+}
+
 __global__ void __launch_bounds__(256)
 walk_merge_kernel(const __grid_constant__ grf_walk_params P,
                   const int32_t* __restrict__ rowptr, const int32_t* __restrict__ col, const float* __restrict__ w,
@@ -109,6 +148,16 @@ walk_merge_kernel(const __grid_constant__ grf_walk_params P,
     while (Psort < cnt) Psort <<= 1;
     for (int32_t x = cnt + lane; x < Psort; x += 32) keys[x] = 0xffffffffu;
     __syncwarp();
+    if (Psort <= 512) {
+        switch (Psort) {
+            case 32: sort_in_registers<1>(keys, lane); break;
+            case 64: sort_in_registers<2>(keys, lane); break;
+            case 128: sort_in_registers<4>(keys, lane); break;
+            case 256: sort_in_registers<8>(keys, lane); break;
+            default: sort_in_registers<16>(keys, lane); break;
+        }
+        __syncwarp();
+    } else
     for (int32_t k = 2; k <= Psort; k <<= 1)
         for (int32_t j = k >> 1; j > 0; j >>= 1) {
             for (int32_t idx = lane; idx < (Psort >> 1); idx += 32) {
