@@ -88,9 +88,30 @@ __host__ __device__ constexpr uint32_t instr_desc_bf16(int n)
     return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
 }
 
+// The issuing helpers below are called by ALL lanes of a converged warp with the same arguments; elect.sync
+// picks the lane that issues.  (Issued from a branch that only one lane takes, the same instruction costs
+// its thread about three times as many cycles: the operands of these instructions are warp-uniform.)
 __device__ __forceinline__ void mma_commit(uint32_t bar)
 {
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+    asm volatile(
+        "{\n\t.reg .pred q;\n\t"
+        "elect.sync _|q, 0xffffffff;\n\t"
+        "@q tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n\t}"
+        ::"r"(bar) : "memory");
+}
+// expect-tx arrival, bulk copy of one record into its slot and an L2 prefetch of a later record, by one elected lane
+__device__ __forceinline__ void load_record_elected(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar,
+                                                    const void* prefetch_src, uint32_t prefetch_bytes)
+{
+    asm volatile(
+        "{\n\t.reg .pred q, r;\n\t"
+        "elect.sync _|q, 0xffffffff;\n\t"
+        "setp.ne.u32 r, %5, 0;\n\t"
+        "and.pred r, r, q;\n\t"
+        "@r cp.async.bulk.prefetch.L2.global [%4], %5;\n\t"
+        "@q mbarrier.arrive.expect_tx.shared::cta.b64 _, [%3], %2;\n\t"
+        "@q cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];\n\t}"
+        ::"r"(dst), "l"(src), "r"(bytes), "r"(bar), "l"(prefetch_src), "r"(prefetch_bytes) : "memory");
 }
 
 __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16])
@@ -124,9 +145,10 @@ __device__ __forceinline__ void mma_bf16_ts(uint32_t d_tmem, uint32_t a_tmem, ui
                                             uint32_t accumulate)
 {
     asm volatile(
-        "{\n\t.reg .pred p;\n\t"
+        "{\n\t.reg .pred p, q;\n\t"
         "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+        "elect.sync _|q, 0xffffffff;\n\t"
+        "@q tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
         ::"r"(d_tmem), "r"(a_tmem), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
 }
 
@@ -310,25 +332,21 @@ gather_contract_tc_kernel(int32_t N, int32_t R, const int32_t* __restrict__ plan
         }
     } else if (warp == 4) {
         // ------------------------------------------------------------ record loader (runs NBC chunks ahead)
+        // (the whole warp runs the loop in step; one elected lane issues)
         int32_t issued = 0;
         for (int32_t gi = 0; gi < ngroups; ++gi) {
-            if (gi >= NBC && !mbar_wait(done(gi % NBC), (uint32_t)((gi - NBC) / NBC) & 1u, &abort_flag)) break;
+            if (gi >= NBC && !__all_sync(0xffffffffu, mbar_wait(done(gi % NBC), (uint32_t)((gi - NBC) / NBC) & 1u, &abort_flag))) break;
             const int32_t uend = min(cnt, (gi + 1) * GU);
-            if (lane == 0) {
-                for (int32_t u = gi * GU; u < uend; ++u) {
-                    // records further down the list are pulled into L2 ahead of their turn
-                    if (u + 2 * NREC < cnt)
-                        asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;"
-                                     ::"l"(recs + (size_t)__ldg(ulist + u + 2 * NREC) * Sh::REC_BYTES), "r"((uint32_t)Sh::REC_BYTES)
-                                     : "memory");
-                    const int s = u % NREC;
-                    const int32_t l = __ldg(ulist + u);
-                    mbar_arrive_expect_tx(rec_full(s), Sh::REC_BYTES);
-                    bulk_copy_g2s(b_base + (uint32_t)s * Sh::REC_BYTES, recs + (size_t)l * Sh::REC_BYTES, Sh::REC_BYTES, rec_full(s));
-                }
+            for (int32_t u = gi * GU; u < uend; ++u) {
+                // records further down the list are pulled into L2 ahead of their turn
+                const bool pf = u + 2 * NREC < cnt;
+                const int32_t lp = pf ? __ldg(ulist + u + 2 * NREC) : 0;
+                const int s = u % NREC;
+                const int32_t l = __ldg(ulist + u);
+                load_record_elected(b_base + (uint32_t)s * Sh::REC_BYTES, recs + (size_t)l * Sh::REC_BYTES, Sh::REC_BYTES, rec_full(s),
+                                    recs + (size_t)lp * Sh::REC_BYTES, pf ? (uint32_t)Sh::REC_BYTES : 0u);
             }
             issued = uend;
-            __syncwarp();
         }
         if (abort_flag) {
             // gave up somewhere: let the copies that are still in flight land before the CTA exits
@@ -340,6 +358,8 @@ gather_contract_tc_kernel(int32_t N, int32_t R, const int32_t* __restrict__ plan
         }
     } else {
         // ------------------------------------------------------------ MMA issuers: warp 5 takes even groups, warp 6 odd
+        // The whole warp runs the loop in step (every exit is voted on), so that the issuing helpers meet a
+        // converged warp.
         const int w = warp - 5;
         constexpr uint32_t idesc = instr_desc_bf16(D);
         const uint32_t acc = tmem_base + (uint32_t)(w * D);
@@ -347,34 +367,30 @@ gather_contract_tc_kernel(int32_t N, int32_t R, const int32_t* __restrict__ plan
         bool first = true;
         for (int32_t gi = w; gi < ngroups && ok; gi += 2) {
             const int st = gi % NA;
-            if (!mbar_wait(a_full(st), (uint32_t)(gi / NA) & 1u, &abort_flag)) { ok = false; break; }
+            if (!__all_sync(0xffffffffu, mbar_wait(a_full(st), (uint32_t)(gi / NA) & 1u, &abort_flag))) { ok = false; break; }
             const int32_t uend = min(cnt, (gi + 1) * GU);
             for (int32_t u = gi * GU; u < uend; ++u) {
                 const int sr = u % NREC;
-                if (!mbar_wait(rec_full(sr), (uint32_t)(u / NREC) & 1u, &abort_flag)) { ok = false; break; }
+                if (!__all_sync(0xffffffffu, mbar_wait(rec_full(sr), (uint32_t)(u / NREC) & 1u, &abort_flag))) { ok = false; break; }
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                if (lane == 0) {
-                    const uint32_t a_op = tmem_a + (uint32_t)((st * GU + (u - gi * GU)) * Sh::A_COLS);
-                    const uint32_t b_op = b_base + (uint32_t)sr * Sh::REC_BYTES;
+                const uint32_t a_op = tmem_a + (uint32_t)((st * GU + (u - gi * GU)) * Sh::A_COLS);
+                const uint32_t b_op = b_base + (uint32_t)sr * Sh::REC_BYTES;
 #pragma unroll
-                    for (int k = 0; k < M / 16; ++k) {
-                        const uint64_t bd = operand_desc(b_op + (uint32_t)k * 2u * (D * 16), D * 16, 128);
-                        mma_bf16_ts(acc, a_op + (uint32_t)k * 8u, bd, idesc, (first && k == 0) ? 0u : 1u);
-                    }
+                for (int k = 0; k < M / 16; ++k) {
+                    const uint64_t bd = operand_desc(b_op + (uint32_t)k * 2u * (D * 16), D * 16, 128);
+                    mma_bf16_ts(acc, a_op + (uint32_t)k * 8u, bd, idesc, (first && k == 0) ? 0u : 1u);
                 }
                 first = false;
-                __syncwarp();
             }
-            if (lane == 0 && ok) mma_commit(done(gi % NBC));
-            __syncwarp();
+            if (ok) mma_commit(done(gi % NBC));
         }
-        if (lane == 0 && ngroups > w) mma_commit(acc_done(w));
-        __syncwarp();
+        if (ngroups > w) mma_commit(acc_done(w));
         if (!ok && ngroups > w) {
             // aborted: wait (bounded) until the MMAs already issued have drained before the CTA exits
             const long long t0 = clock64();
             while (!mbar_try_wait(acc_done(w), 0u) && clock64() - t0 < WAIT_CYCLES) {}
         }
+        __syncwarp();
     }
 
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
