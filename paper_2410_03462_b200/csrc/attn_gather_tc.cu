@@ -99,7 +99,15 @@ __device__ __forceinline__ void mma_commit(uint32_t bar)
         "@q tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n\t}"
         ::"r"(bar) : "memory");
 }
-// expect-tx arrival, bulk copy of one record into its slot and an L2 prefetch of a later record, by one elected lane
+// bulk copy of one record into its slot and an L2 prefetch of a later record, by one elected lane
+__device__ __forceinline__ void expect_tx_elected(uint32_t bar, uint32_t bytes)
+{
+    asm volatile(
+        "{\n\t.reg .pred q;\n\t"
+        "elect.sync _|q, 0xffffffff;\n\t"
+        "@q mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;\n\t}"
+        ::"r"(bar), "r"(bytes) : "memory");
+}
 __device__ __forceinline__ void load_record_elected(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar,
                                                     const void* prefetch_src, uint32_t prefetch_bytes)
 {
@@ -109,7 +117,6 @@ __device__ __forceinline__ void load_record_elected(uint32_t dst, const void* sr
         "setp.ne.u32 r, %5, 0;\n\t"
         "and.pred r, r, q;\n\t"
         "@r cp.async.bulk.prefetch.L2.global [%4], %5;\n\t"
-        "@q mbarrier.arrive.expect_tx.shared::cta.b64 _, [%3], %2;\n\t"
         "@q cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];\n\t}"
         ::"r"(dst), "l"(src), "r"(bytes), "r"(bar), "l"(prefetch_src), "r"(prefetch_bytes) : "memory");
 }
@@ -182,8 +189,8 @@ gather_contract_tc_kernel(int32_t N, int32_t R, const int32_t* __restrict__ plan
     using Sh = TcShape<M, D>;
     constexpr int NA = Sh::NA, NBC = Sh::NBC, GU = Sh::GU, NREC = NBC * GU;
     extern __shared__ unsigned char smem_dyn[];
-    // a_full per A stage; rec_full per record slot; done per record chunk (= per group); acc_done per issuer
-    __shared__ __align__(8) unsigned long long bars[NA + NREC + NBC + 2];
+    // a_full per A stage; rec_full and done per record chunk (= per group of GU union entries); acc_done per issuer
+    __shared__ __align__(8) unsigned long long bars[NA + NBC + NBC + 2];
     __shared__ uint32_t tmem_slot;
     __shared__ int abort_flag;
 
@@ -194,12 +201,12 @@ gather_contract_tc_kernel(int32_t N, int32_t R, const int32_t* __restrict__ plan
     const uint32_t bar_base = smem_u32(bars);
     auto a_full = [&](int s) { return bar_base + 8u * (uint32_t)s; };
     auto rec_full = [&](int s) { return bar_base + 8u * (uint32_t)(NA + s); };
-    auto done = [&](int s) { return bar_base + 8u * (uint32_t)(NA + NREC + s); };
-    auto acc_done = [&](int w) { return bar_base + 8u * (uint32_t)(NA + NREC + NBC + w); };
+    auto done = [&](int s) { return bar_base + 8u * (uint32_t)(NA + NBC + s); };
+    auto acc_done = [&](int w) { return bar_base + 8u * (uint32_t)(NA + NBC + NBC + w); };
 
     if (tid == 0) {
         for (int s = 0; s < NA; ++s) mbar_init(a_full(s), 4);
-        for (int s = 0; s < NREC; ++s) mbar_init(rec_full(s), 1);
+        for (int s = 0; s < NBC; ++s) mbar_init(rec_full(s), 1);
         for (int s = 0; s < NBC; ++s) mbar_init(done(s), 1);
         mbar_init(acc_done(0), 1);
         mbar_init(acc_done(1), 1);
@@ -337,23 +344,25 @@ gather_contract_tc_kernel(int32_t N, int32_t R, const int32_t* __restrict__ plan
         for (int32_t gi = 0; gi < ngroups; ++gi) {
             if (gi >= NBC && !__all_sync(0xffffffffu, mbar_wait(done(gi % NBC), (uint32_t)((gi - NBC) / NBC) & 1u, &abort_flag))) break;
             const int32_t uend = min(cnt, (gi + 1) * GU);
+            // one barrier per chunk: it completes when all of the chunk's records have landed
+            expect_tx_elected(rec_full(gi % NBC), (uint32_t)(uend - gi * GU) * Sh::REC_BYTES);
             for (int32_t u = gi * GU; u < uend; ++u) {
                 // records further down the list are pulled into L2 ahead of their turn
                 const bool pf = u + 2 * NREC < cnt;
                 const int32_t lp = pf ? __ldg(ulist + u + 2 * NREC) : 0;
                 const int s = u % NREC;
                 const int32_t l = __ldg(ulist + u);
-                load_record_elected(b_base + (uint32_t)s * Sh::REC_BYTES, recs + (size_t)l * Sh::REC_BYTES, Sh::REC_BYTES, rec_full(s),
+                load_record_elected(b_base + (uint32_t)s * Sh::REC_BYTES, recs + (size_t)l * Sh::REC_BYTES, Sh::REC_BYTES, rec_full(gi % NBC),
                                     recs + (size_t)lp * Sh::REC_BYTES, pf ? (uint32_t)Sh::REC_BYTES : 0u);
             }
             issued = uend;
         }
         if (abort_flag) {
             // gave up somewhere: let the copies that are still in flight land before the CTA exits
-            const int32_t first = issued > NREC ? issued - NREC : 0;
-            for (int32_t u = first; u < issued; ++u) {
+            const int32_t glast = (issued + GU - 1) / GU;
+            for (int32_t gq = glast > NBC ? glast - NBC : 0; gq < glast; ++gq) {
                 const long long t0 = clock64();
-                while (!mbar_try_wait(rec_full(u % NREC), (uint32_t)(u / NREC) & 1u) && clock64() - t0 < WAIT_CYCLES) {}
+                while (!mbar_try_wait(rec_full(gq % NBC), (uint32_t)(gq / NBC) & 1u) && clock64() - t0 < WAIT_CYCLES) {}
             }
         }
     } else {
@@ -368,11 +377,11 @@ gather_contract_tc_kernel(int32_t N, int32_t R, const int32_t* __restrict__ plan
         for (int32_t gi = w; gi < ngroups && ok; gi += 2) {
             const int st = gi % NA;
             if (!__all_sync(0xffffffffu, mbar_wait(a_full(st), (uint32_t)(gi / NA) & 1u, &abort_flag))) { ok = false; break; }
+            if (!__all_sync(0xffffffffu, mbar_wait(rec_full(gi % NBC), (uint32_t)(gi / NBC) & 1u, &abort_flag))) { ok = false; break; }
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
             const int32_t uend = min(cnt, (gi + 1) * GU);
             for (int32_t u = gi * GU; u < uend; ++u) {
                 const int sr = u % NREC;
-                if (!__all_sync(0xffffffffu, mbar_wait(rec_full(sr), (uint32_t)(u / NREC) & 1u, &abort_flag))) { ok = false; break; }
-                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                 const uint32_t a_op = tmem_a + (uint32_t)((st * GU + (u - gi * GU)) * Sh::A_COLS);
                 const uint32_t b_op = b_base + (uint32_t)sr * Sh::REC_BYTES;
 #pragma unroll
