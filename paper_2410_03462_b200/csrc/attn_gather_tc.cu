@@ -164,8 +164,8 @@ constexpr int pow2_at_least(int x) { return x <= 32 ? 32 : (x <= 64 ? 64 : (x <=
 template <int M, int D> struct TcShape {
     static constexpr int A_COLS = M / 2;                      // TMEM columns of one union entry's A operand
     static constexpr int GU = M <= 32 ? 4 : (M == 64 ? 2 : 1); // union entries per group (one commit per group)
-    static constexpr int NA = 2;                              // A stages (groups in flight on the row-thread side)
-    static constexpr int TMEM_COLS = pow2_at_least(2 * D + NA * GU * A_COLS);   // two accumulators + A ring
+    static constexpr int NA = 3;                              // A stages: groups written ahead of the one being multiplied
+    static constexpr int TMEM_COLS = pow2_at_least(D + NA * GU * A_COLS);       // accumulator + A ring
     static constexpr int TILE_BYTES = M * D * 2;
     static constexpr int REC_BYTES = TILE_BYTES + M * 4;      // state tile followed by z
     static constexpr int CHUNK_BYTES = GU * REC_BYTES;
@@ -175,8 +175,8 @@ template <int M, int D> struct TcShape {
     static constexpr size_t SMEM = (size_t)NBC * CHUNK_BYTES + 1024;                  // + alignment slack
 };
 
-// warps 0-3: row threads (A operand, denominators, epilogue); warp 4: record loader; warps 5, 6: MMA issuers
-constexpr int TC_THREADS = 224;
+// warps 0-3: row threads (A operand, epilogue); warp 4: record loader; warp 5: MMA issuer
+constexpr int TC_THREADS = 192;
 
 template <int M, int D>
 __global__ void __launch_bounds__(TC_THREADS)
@@ -190,7 +190,7 @@ gather_contract_tc_kernel(int32_t N, int32_t R, const int32_t* __restrict__ plan
     constexpr int NA = Sh::NA, NBC = Sh::NBC, GU = Sh::GU, NREC = NBC * GU;
     extern __shared__ unsigned char smem_dyn[];
     // a_full per A stage; rec_full and done per record chunk (= per group of GU union entries); acc_done per issuer
-    __shared__ __align__(8) unsigned long long bars[NA + NBC + NBC + 2];
+    __shared__ __align__(8) unsigned long long bars[NA + NBC + NBC + 1];
     __shared__ uint32_t tmem_slot;
     __shared__ int abort_flag;
 
@@ -202,14 +202,13 @@ gather_contract_tc_kernel(int32_t N, int32_t R, const int32_t* __restrict__ plan
     auto a_full = [&](int s) { return bar_base + 8u * (uint32_t)s; };
     auto rec_full = [&](int s) { return bar_base + 8u * (uint32_t)(NA + s); };
     auto done = [&](int s) { return bar_base + 8u * (uint32_t)(NA + NBC + s); };
-    auto acc_done = [&](int w) { return bar_base + 8u * (uint32_t)(NA + NBC + NBC + w); };
+    const uint32_t acc_done = bar_base + 8u * (uint32_t)(NA + NBC + NBC);
 
     if (tid == 0) {
         for (int s = 0; s < NA; ++s) mbar_init(a_full(s), 4);
         for (int s = 0; s < NBC; ++s) mbar_init(rec_full(s), 1);
         for (int s = 0; s < NBC; ++s) mbar_init(done(s), 1);
-        mbar_init(acc_done(0), 1);
-        mbar_init(acc_done(1), 1);
+        mbar_init(acc_done, 1);
         abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -222,7 +221,7 @@ gather_contract_tc_kernel(int32_t N, int32_t R, const int32_t* __restrict__ plan
     __syncthreads();
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     const uint32_t tmem_base = tmem_slot;
-    const uint32_t tmem_a = tmem_base + 2u * D;     // A ring behind the two accumulators
+    const uint32_t tmem_a = tmem_base + (uint32_t)D;   // A ring behind the accumulator
 
     const int32_t cnt = plan_cnt[blk];
     const int32_t ngroups = (cnt + GU - 1) / GU;
@@ -308,28 +307,23 @@ gather_contract_tc_kernel(int32_t N, int32_t R, const int32_t* __restrict__ plan
             __syncwarp();
             if (lane == 0) mbar_arrive(a_full(st));
         }
-        // epilogue: this thread's row of the accumulators is TMEM lane `tid`; the two issuers' partial sums are
-        // added in a fixed order
-        if (ok && ngroups > 0) ok = mbar_wait(acc_done(0), 0u, &abort_flag);
-        if (ok && ngroups > 1) ok = mbar_wait(acc_done(1), 0u, &abort_flag);
+        // epilogue: this thread's row of the accumulator is TMEM lane `tid`
+        if (ok && ngroups > 0) ok = mbar_wait(acc_done, 0u, &abort_flag);
         ok = __all_sync(0xffffffffu, ok);   // the tensor-memory loads below are warp-wide
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         const float inv = (den != 0.0f) ? 1.0f / den : 0.0f;
         __nv_bfloat16* orow = out + ((size_t)g * N + row) * D;
 #pragma unroll
         for (int c0 = 0; c0 < D; c0 += 16) {
-            uint32_t r[16], r1[16];
+            uint32_t r[16];
 #pragma unroll
-            for (int e = 0; e < 16; ++e) { r[e] = 0u; r1[e] = 0u; }
+            for (int e = 0; e < 16; ++e) r[e] = 0u;
             if (ok && ngroups > 0) tmem_ld16(tmem_base + lane_field + (uint32_t)c0, r);
-            if (ok && ngroups > 1) tmem_ld16(tmem_base + lane_field + (uint32_t)(D + c0), r1);
             if (live && ok) {
                 uint32_t w[8];
 #pragma unroll
                 for (int e = 0; e < 8; ++e) {
-                    const float x0 = (__uint_as_float(r[2 * e]) + __uint_as_float(r1[2 * e])) * inv;
-                    const float x1 = (__uint_as_float(r[2 * e + 1]) + __uint_as_float(r1[2 * e + 1])) * inv;
-                    __nv_bfloat162 h = __floats2bfloat162_rn(x0, x1);
+                    __nv_bfloat162 h = __floats2bfloat162_rn(__uint_as_float(r[2 * e]) * inv, __uint_as_float(r[2 * e + 1]) * inv);
                     w[e] = *reinterpret_cast<uint32_t*>(&h);
                 }
                 uint4* dst = reinterpret_cast<uint4*>(orow + c0);
@@ -339,23 +333,39 @@ gather_contract_tc_kernel(int32_t N, int32_t R, const int32_t* __restrict__ plan
         }
     } else if (warp == 4) {
         // ------------------------------------------------------------ record loader (runs NBC chunks ahead)
-        // (the whole warp runs the loop in step; one elected lane issues)
+        // (the whole warp runs the loop in step; one elected lane issues).  The node indices of a group are
+        // read one group ahead of their use, all at once, so that no copy waits for an index load.
         int32_t issued = 0;
+        int32_t l_cur[GU], p_cur[GU], l_nxt[GU], p_nxt[GU];
+        auto read_indices = [&](int32_t gq, int32_t (&l)[GU], int32_t (&pf)[GU]) {
+#pragma unroll
+            for (int j = 0; j < GU; ++j) {
+                const int32_t u = gq * GU + j;
+                l[j] = u < cnt ? __ldg(ulist + u) : 0;
+                pf[j] = u + 2 * NREC < cnt ? __ldg(ulist + u + 2 * NREC) : -1;
+            }
+        };
+        read_indices(0, l_cur, p_cur);
         for (int32_t gi = 0; gi < ngroups; ++gi) {
+            read_indices(gi + 1, l_nxt, p_nxt);
             if (gi >= NBC && !__all_sync(0xffffffffu, mbar_wait(done(gi % NBC), (uint32_t)((gi - NBC) / NBC) & 1u, &abort_flag))) break;
             const int32_t uend = min(cnt, (gi + 1) * GU);
             // one barrier per chunk: it completes when all of the chunk's records have landed
             expect_tx_elected(rec_full(gi % NBC), (uint32_t)(uend - gi * GU) * Sh::REC_BYTES);
-            for (int32_t u = gi * GU; u < uend; ++u) {
-                // records further down the list are pulled into L2 ahead of their turn
-                const bool pf = u + 2 * NREC < cnt;
-                const int32_t lp = pf ? __ldg(ulist + u + 2 * NREC) : 0;
-                const int s = u % NREC;
-                const int32_t l = __ldg(ulist + u);
-                load_record_elected(b_base + (uint32_t)s * Sh::REC_BYTES, recs + (size_t)l * Sh::REC_BYTES, Sh::REC_BYTES, rec_full(gi % NBC),
-                                    recs + (size_t)lp * Sh::REC_BYTES, pf ? (uint32_t)Sh::REC_BYTES : 0u);
+#pragma unroll
+            for (int j = 0; j < GU; ++j) {
+                const int32_t u = gi * GU + j;
+                if (u < uend) {
+                    // records further down the list are pulled into L2 ahead of their turn
+                    const int s = u % NREC;
+                    load_record_elected(b_base + (uint32_t)s * Sh::REC_BYTES, recs + (size_t)l_cur[j] * Sh::REC_BYTES, Sh::REC_BYTES,
+                                        rec_full(gi % NBC), recs + (size_t)max(p_cur[j], 0) * Sh::REC_BYTES,
+                                        p_cur[j] >= 0 ? (uint32_t)Sh::REC_BYTES : 0u);
+                }
             }
             issued = uend;
+#pragma unroll
+            for (int j = 0; j < GU; ++j) { l_cur[j] = l_nxt[j]; p_cur[j] = p_nxt[j]; }
         }
         if (abort_flag) {
             // gave up somewhere: let the copies that are still in flight land before the CTA exits
@@ -366,15 +376,14 @@ gather_contract_tc_kernel(int32_t N, int32_t R, const int32_t* __restrict__ plan
             }
         }
     } else {
-        // ------------------------------------------------------------ MMA issuers: warp 5 takes even groups, warp 6 odd
+        // ------------------------------------------------------------ MMA issuer: all groups, in list order
         // The whole warp runs the loop in step (every exit is voted on), so that the issuing helpers meet a
         // converged warp.
-        const int w = warp - 5;
         constexpr uint32_t idesc = instr_desc_bf16(D);
-        const uint32_t acc = tmem_base + (uint32_t)(w * D);
+        const uint32_t acc = tmem_base;
         bool ok = true;
         bool first = true;
-        for (int32_t gi = w; gi < ngroups && ok; gi += 2) {
+        for (int32_t gi = 0; gi < ngroups && ok; ++gi) {
             const int st = gi % NA;
             if (!__all_sync(0xffffffffu, mbar_wait(a_full(st), (uint32_t)(gi / NA) & 1u, &abort_flag))) { ok = false; break; }
             if (!__all_sync(0xffffffffu, mbar_wait(rec_full(gi % NBC), (uint32_t)(gi / NBC) & 1u, &abort_flag))) { ok = false; break; }
@@ -393,11 +402,11 @@ gather_contract_tc_kernel(int32_t N, int32_t R, const int32_t* __restrict__ plan
             }
             if (ok) mma_commit(done(gi % NBC));
         }
-        if (ngroups > w) mma_commit(acc_done(w));
-        if (!ok && ngroups > w) {
+        if (ngroups > 0) mma_commit(acc_done);
+        if (!ok && ngroups > 0) {
             // aborted: wait (bounded) until the MMAs already issued have drained before the CTA exits
             const long long t0 = clock64();
-            while (!mbar_try_wait(acc_done(w), 0u) && clock64() - t0 < WAIT_CYCLES) {}
+            while (!mbar_try_wait(acc_done, 0u) && clock64() - t0 < WAIT_CYCLES) {}
         }
         __syncwarp();
     }
