@@ -99,7 +99,6 @@ __device__ __forceinline__ void mma_commit(uint32_t bar)
         "@q tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n\t}"
         ::"r"(bar) : "memory");
 }
-// bulk copy of one record into its slot and an L2 prefetch of a later record, by one elected lane
 __device__ __forceinline__ void expect_tx_elected(uint32_t bar, uint32_t bytes)
 {
     asm volatile(
@@ -108,17 +107,14 @@ __device__ __forceinline__ void expect_tx_elected(uint32_t bar, uint32_t bytes)
         "@q mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;\n\t}"
         ::"r"(bar), "r"(bytes) : "memory");
 }
-__device__ __forceinline__ void load_record_elected(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar,
-                                                    const void* prefetch_src, uint32_t prefetch_bytes)
+// bulk copy of one record into its slot, by one elected lane
+__device__ __forceinline__ void load_record_elected(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar)
 {
     asm volatile(
-        "{\n\t.reg .pred q, r;\n\t"
+        "{\n\t.reg .pred q;\n\t"
         "elect.sync _|q, 0xffffffff;\n\t"
-        "setp.ne.u32 r, %5, 0;\n\t"
-        "and.pred r, r, q;\n\t"
-        "@r cp.async.bulk.prefetch.L2.global [%4], %5;\n\t"
         "@q cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];\n\t}"
-        ::"r"(dst), "l"(src), "r"(bytes), "r"(bar), "l"(prefetch_src), "r"(prefetch_bytes) : "memory");
+        ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
 }
 
 __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16])
@@ -334,20 +330,17 @@ gather_contract_tc_kernel(int32_t N, int32_t R, const int32_t* __restrict__ plan
     } else if (warp == 4) {
         // ------------------------------------------------------------ record loader (runs NBC chunks ahead)
         // (the whole warp runs the loop in step; one elected lane issues).  The node indices of a group are
-        // read one group ahead of their use, all at once, so that no copy waits for an index load.
+        // read one group ahead of their use, all at once, so that no copy waits for an index load.  The ring is
+        // deep enough to cover the latency of HBM: separate L2 prefetches only cost issue slots.
         int32_t issued = 0;
-        int32_t l_cur[GU], p_cur[GU], l_nxt[GU], p_nxt[GU];
-        auto read_indices = [&](int32_t gq, int32_t (&l)[GU], int32_t (&pf)[GU]) {
+        int32_t l_cur[GU], l_nxt[GU];
+        auto read_indices = [&](int32_t gq, int32_t (&l)[GU]) {
 #pragma unroll
-            for (int j = 0; j < GU; ++j) {
-                const int32_t u = gq * GU + j;
-                l[j] = u < cnt ? __ldg(ulist + u) : 0;
-                pf[j] = u + 2 * NREC < cnt ? __ldg(ulist + u + 2 * NREC) : -1;
-            }
+            for (int j = 0; j < GU; ++j) l[j] = gq * GU + j < cnt ? __ldg(ulist + gq * GU + j) : 0;
         };
-        read_indices(0, l_cur, p_cur);
+        read_indices(0, l_cur);
         for (int32_t gi = 0; gi < ngroups; ++gi) {
-            read_indices(gi + 1, l_nxt, p_nxt);
+            read_indices(gi + 1, l_nxt);
             if (gi >= NBC && !__all_sync(0xffffffffu, mbar_wait(done(gi % NBC), (uint32_t)((gi - NBC) / NBC) & 1u, &abort_flag))) break;
             const int32_t uend = min(cnt, (gi + 1) * GU);
             // one barrier per chunk: it completes when all of the chunk's records have landed
@@ -355,17 +348,13 @@ gather_contract_tc_kernel(int32_t N, int32_t R, const int32_t* __restrict__ plan
 #pragma unroll
             for (int j = 0; j < GU; ++j) {
                 const int32_t u = gi * GU + j;
-                if (u < uend) {
-                    // records further down the list are pulled into L2 ahead of their turn
-                    const int s = u % NREC;
-                    load_record_elected(b_base + (uint32_t)s * Sh::REC_BYTES, recs + (size_t)l_cur[j] * Sh::REC_BYTES, Sh::REC_BYTES,
-                                        rec_full(gi % NBC), recs + (size_t)max(p_cur[j], 0) * Sh::REC_BYTES,
-                                        p_cur[j] >= 0 ? (uint32_t)Sh::REC_BYTES : 0u);
-                }
+                if (u < uend)
+                    load_record_elected(b_base + (uint32_t)(u % NREC) * Sh::REC_BYTES, recs + (size_t)l_cur[j] * Sh::REC_BYTES,
+                                        Sh::REC_BYTES, rec_full(gi % NBC));
             }
             issued = uend;
 #pragma unroll
-            for (int j = 0; j < GU; ++j) { l_cur[j] = l_nxt[j]; p_cur[j] = p_nxt[j]; }
+            for (int j = 0; j < GU; ++j) l_cur[j] = l_nxt[j];
         }
         if (abort_flag) {
             // gave up somewhere: let the copies that are still in flight land before the CTA exits
