@@ -164,7 +164,7 @@ template <int M, int D> struct TcShape {
     static constexpr int TMEM_COLS = pow2_at_least(D + NA * GU * A_COLS);       // accumulator + A ring
     static constexpr int TILE_BYTES = M * D * 2;
     static constexpr int REC_BYTES = TILE_BYTES + M * 4;      // state tile followed by z
-    static constexpr int CHUNK_BYTES = GU * REC_BYTES;
+    static constexpr int CHUNK_BYTES = GU * TILE_BYTES;        // only the tiles are copied to shared memory
     static constexpr int SMEM_BUDGET = TMEM_COLS <= 256 ? 104 * 1024 : 200 * 1024;   // two CTAs per SM, or one
     static constexpr int NBC_WANT = SMEM_BUDGET / CHUNK_BYTES;
     static constexpr int NBC = NBC_WANT > 8 ? 8 : (NBC_WANT < 2 ? 2 : NBC_WANT);     // record chunks in flight
@@ -344,13 +344,13 @@ gather_contract_tc_kernel(int32_t N, int32_t R, const int32_t* __restrict__ plan
             if (gi >= NBC && !__all_sync(0xffffffffu, mbar_wait(done(gi % NBC), (uint32_t)((gi - NBC) / NBC) & 1u, &abort_flag))) break;
             const int32_t uend = min(cnt, (gi + 1) * GU);
             // one barrier per chunk: it completes when all of the chunk's records have landed
-            expect_tx_elected(rec_full(gi % NBC), (uint32_t)(uend - gi * GU) * Sh::REC_BYTES);
+            expect_tx_elected(rec_full(gi % NBC), (uint32_t)(uend - gi * GU) * Sh::TILE_BYTES);
 #pragma unroll
             for (int j = 0; j < GU; ++j) {
                 const int32_t u = gi * GU + j;
                 if (u < uend)
-                    load_record_elected(b_base + (uint32_t)(u % NREC) * Sh::REC_BYTES, recs + (size_t)l_cur[j] * Sh::REC_BYTES,
-                                        Sh::REC_BYTES, rec_full(gi % NBC));
+                    load_record_elected(b_base + (uint32_t)(u % NREC) * Sh::TILE_BYTES, recs + (size_t)l_cur[j] * Sh::REC_BYTES,
+                                        Sh::TILE_BYTES, rec_full(gi % NBC));
             }
             issued = uend;
 #pragma unroll
@@ -381,7 +381,7 @@ gather_contract_tc_kernel(int32_t N, int32_t R, const int32_t* __restrict__ plan
             for (int32_t u = gi * GU; u < uend; ++u) {
                 const int sr = u % NREC;
                 const uint32_t a_op = tmem_a + (uint32_t)((st * GU + (u - gi * GU)) * Sh::A_COLS);
-                const uint32_t b_op = b_base + (uint32_t)sr * Sh::REC_BYTES;
+                const uint32_t b_op = b_base + (uint32_t)sr * Sh::TILE_BYTES;
 #pragma unroll
                 for (int k = 0; k < M / 16; ++k) {
                     const uint64_t bd = operand_desc(b_op + (uint32_t)k * 2u * (D * 16), D * 16, 128);
