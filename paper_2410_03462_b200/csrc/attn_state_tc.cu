@@ -77,18 +77,26 @@ __host__ __device__ constexpr uint32_t instr_desc_mn(int n)
     return (1u << 4) | (1u << 7) | (1u << 10) | (1u << 15) | (1u << 16) | ((uint32_t)(n >> 3) << 17) |
            ((uint32_t)(128 >> 4) << 24);
 }
+// The two issuing helpers are called by ALL lanes of a converged warp with the same arguments; elect.sync
+// picks the lane that issues.  (Issued from a branch that only one lane takes, the same instruction costs
+// its thread about three times as many cycles: the operands of tcgen05 instructions are warp-uniform.)
 __device__ __forceinline__ void mma_bf16_ss(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
                                             uint32_t accumulate)
 {
     asm volatile(
-        "{\n\t.reg .pred p;\n\t"
+        "{\n\t.reg .pred p, q;\n\t"
         "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        "elect.sync _|q, 0xffffffff;\n\t"
+        "@q tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
         ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
 }
 __device__ __forceinline__ void mma_commit(uint32_t bar)
 {
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+    asm volatile(
+        "{\n\t.reg .pred q;\n\t"
+        "elect.sync _|q, 0xffffffff;\n\t"
+        "@q tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n\t}"
+        ::"r"(bar) : "memory");
 }
 __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16])
 {
@@ -289,26 +297,23 @@ build_states_tc_kernel(int32_t R, int32_t N, const int32_t* __restrict__ t_rowpt
             const int32_t nitems = c > 0 ? (c + ITEM_KEYS - 1) / ITEM_KEYS : 1;
             const int buf = nn & 1;
             // the accumulator buffer must have been read out by the epilogue of the node two back
-            if (!mbar_wait(acc_free(buf), ((uint32_t)(nn >> 1) & 1u) ^ 1u, &abort_flag)) { ok = false; break; }
+            if (!__all_sync(0xffffffffu, mbar_wait(acc_free(buf), ((uint32_t)(nn >> 1) & 1u) ^ 1u, &abort_flag))) { ok = false; break; }
             const uint32_t acc = tmem_base + (uint32_t)(buf * Sh::ACC_COLS);
             for (int32_t it = 0; it < nitems; ++it, ++q) {
                 const int s = q % NS;
                 const int32_t n = min(ITEM_KEYS, c - it * ITEM_KEYS);
                 const int32_t ksteps = n > 0 ? (n + 15) / 16 : 1;
-                if (!mbar_wait(full(s), (uint32_t)(q / NS) & 1u, &abort_flag)) { ok = false; break; }
+                if (!__all_sync(0xffffffffu, mbar_wait(full(s), (uint32_t)(q / NS) & 1u, &abort_flag))) { ok = false; break; }
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                if (lane == 0) {
-                    const uint32_t a_op = stage_base + (uint32_t)s * Sh::STAGE;
-                    const uint32_t b_op = a_op + Sh::A_BYTES;
-                    for (int32_t ks = 0; ks < ksteps; ++ks) {
-                        const uint64_t ad = operand_desc(a_op + (uint32_t)ks * Sh::A_KSTEP, Sh::A_LBO, Sh::A_SBO);
-                        const uint64_t bd = operand_desc(b_op + (uint32_t)ks * Sh::B_KSTEP, Sh::B_LBO, Sh::B_SBO);
-                        mma_bf16_ss(acc, ad, bd, idesc, (it > 0 || ks > 0) ? 1u : 0u);
-                    }
-                    mma_commit(empty(s));
-                    if (it == nitems - 1) mma_commit(acc_full(buf));
+                const uint32_t a_op = stage_base + (uint32_t)s * Sh::STAGE;
+                const uint32_t b_op = a_op + Sh::A_BYTES;
+                for (int32_t ks = 0; ks < ksteps; ++ks) {
+                    const uint64_t ad = operand_desc(a_op + (uint32_t)ks * Sh::A_KSTEP, Sh::A_LBO, Sh::A_SBO);
+                    const uint64_t bd = operand_desc(b_op + (uint32_t)ks * Sh::B_KSTEP, Sh::B_LBO, Sh::B_SBO);
+                    mma_bf16_ss(acc, ad, bd, idesc, (it > 0 || ks > 0) ? 1u : 0u);
                 }
-                __syncwarp();
+                mma_commit(empty(s));
+                if (it == nitems - 1) mma_commit(acc_full(buf));
             }
         }
         if (!ok) {
@@ -599,27 +604,24 @@ build_states_tma_kernel(int32_t R, int32_t N, const int32_t* __restrict__ t_rowp
             const int32_t c = node_beg[l - l0 + 1] - node_beg[l - l0];
             const int32_t nitems = c > 0 ? (c + ITEM_KEYS - 1) / ITEM_KEYS : 1;
             const int buf = nn & 1;
-            if (!mbar_wait(acc_free(buf), ((uint32_t)(nn >> 1) & 1u) ^ 1u, &abort_flag)) { ok = false; break; }
+            if (!__all_sync(0xffffffffu, mbar_wait(acc_free(buf), ((uint32_t)(nn >> 1) & 1u) ^ 1u, &abort_flag))) { ok = false; break; }
             const uint32_t acc = tmem_base + (uint32_t)(buf * Sh::ACC_COLS);
             for (int32_t it = 0; it < nitems; ++it, ++q) {
                 const int s = q % NS;
                 const int32_t n = min(ITEM_KEYS, c - it * ITEM_KEYS);
                 const int32_t ksteps = n > 0 ? (n + 15) / 16 : 1;
-                if (!mbar_wait(full(s), (uint32_t)(q / NS) & 1u, &abort_flag)) { ok = false; break; }
+                if (!__all_sync(0xffffffffu, mbar_wait(full(s), (uint32_t)(q / NS) & 1u, &abort_flag))) { ok = false; break; }
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                if (lane == 0) {
-                    const uint32_t a_op = stage_base + (uint32_t)s * Sh::STAGE;
-                    const uint32_t b_op = a_op + Sh::A_BYTES;
-                    for (int32_t ks = 0; ks < ksteps; ++ks) {
-                        // A: two atoms along M (gathered rows, then the constant atom), 8-key groups 1024 bytes apart
-                        const uint64_t ad = swizzled_desc(a_op + (uint32_t)ks * 2048u, const_base - a_op, 1024u, 2);
-                        const uint64_t bd = operand_desc(b_op + (uint32_t)ks * Sh::B_KSTEP, Sh::B_LBO, Sh::B_SBO);
-                        mma_bf16_ss(acc, ad, bd, idesc, (it > 0 || ks > 0) ? 1u : 0u);
-                    }
-                    mma_commit(empty(s));
-                    if (it == nitems - 1) mma_commit(acc_full(buf));
+                const uint32_t a_op = stage_base + (uint32_t)s * Sh::STAGE;
+                const uint32_t b_op = a_op + Sh::A_BYTES;
+                for (int32_t ks = 0; ks < ksteps; ++ks) {
+                    // A: two atoms along M (gathered rows, then the constant atom), 8-key groups 1024 bytes apart
+                    const uint64_t ad = swizzled_desc(a_op + (uint32_t)ks * 2048u, const_base - a_op, 1024u, 2);
+                    const uint64_t bd = operand_desc(b_op + (uint32_t)ks * Sh::B_KSTEP, Sh::B_LBO, Sh::B_SBO);
+                    mma_bf16_ss(acc, ad, bd, idesc, (it > 0 || ks > 0) ? 1u : 0u);
                 }
-                __syncwarp();
+                mma_commit(empty(s));
+                if (it == nitems - 1) mma_commit(acc_full(buf));
             }
         }
         if (!ok) {
