@@ -34,10 +34,10 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0}
 # heads, so the figures are scaled by 4).  Set an entry to None when its kernel changes after the capture.
 NCU_TRAFFIC_BYTES = {
     "pointcloud-gmm16-N32768": {
-        "gather_contract": 4 * (1.368350e9 + 9.472768e6),
-        "build_states": 4 * (0.062359e9 + 220.503552e6),
-        "row_denominators": 4 * (0.037773e9 + 0.019712e6),
-        "walk_merge": 0.004971e9 + 5.708288e6,
+        "gather_contract": 4 * (1.129637e9 + 10.195200e6),
+        "build_states": 4 * (0.063099e9 + 222.010880e6),
+        "row_denominators": 4 * (0.037773e9 + 0.017152e6),
+        "walk_merge": 0.005111e9 + 5.981440e6,
     }
 }
 
