@@ -268,20 +268,15 @@ gather_contract_tc_kernel(int32_t N, int32_t R, const int32_t* __restrict__ plan
             for (int j = 0; j < GU; ++j) {
                 // A_l[row, :] = Phi_il * phi(q_row): zeros for most rows; products are taken in packed bf16
                 const uint32_t cbits = (uint32_t)(quad >> (16 * ((u0 + j) & 3))) & 0xffffu;
+                // (no branch on a zero coefficient: the product is then a signed zero, which adds nothing)
+                const uint32_t cpair = cbits | (cbits << 16);
+                const __nv_bfloat162 c2 = *reinterpret_cast<const __nv_bfloat162*>(&cpair);
                 uint32_t w[M / 2];
-                if (cbits != 0u) {
-                    const uint32_t cpair = cbits | (cbits << 16);
-                    const __nv_bfloat162 c2 = *reinterpret_cast<const __nv_bfloat162*>(&cpair);
 #pragma unroll
-                    for (int e = 0; e < M / 2; ++e) {
-                        const __nv_bfloat162 h = __hmul2(*reinterpret_cast<const __nv_bfloat162*>(&q2[e]), c2);
-                        w[e] = *reinterpret_cast<const uint32_t*>(&h);
-                    }
-                } else {
-#pragma unroll
-                    for (int e = 0; e < M / 2; ++e) w[e] = 0u;
+                for (int e = 0; e < M / 2; ++e) {
+                    const __nv_bfloat162 h = __hmul2(*reinterpret_cast<const __nv_bfloat162*>(&q2[e]), c2);
+                    w[e] = *reinterpret_cast<const uint32_t*>(&h);
                 }
-                __syncwarp();
                 const uint32_t a_slot = tmem_a + lane_field + (uint32_t)((st * GU + j) * Sh::A_COLS);
                 if constexpr (M >= 32) {
 #pragma unroll
