@@ -66,7 +66,12 @@ extern "C" int grf_ctx_destroy(grf_ctx* ctx)
     if (ctx->h_feat) grf_features_free(ctx->h_feat);
     if (ctx->pinned) cudaFreeHost(ctx->pinned);
     if (ctx->error_word) cudaFree(ctx->error_word);
-    if (ctx->copy_stream) { cudaStreamSynchronize(ctx->copy_stream); cudaStreamDestroy(ctx->copy_stream); cudaEventDestroy(ctx->copy_done); }
+    if (ctx->copy_stream) {
+        cudaStreamSynchronize(ctx->copy_stream); cudaStreamSynchronize(ctx->down_stream);
+        cudaStreamDestroy(ctx->copy_stream); cudaStreamDestroy(ctx->down_stream);
+        for (int p = 0; p < grf_ctx::HOST_PARTS; ++p) { cudaEventDestroy(ctx->up_done[p]); cudaEventDestroy(ctx->part_done[p]); }
+        cudaEventDestroy(ctx->down_done);
+    }
     for (auto& t : ctx->timed) { cudaEventDestroy(t.beg); cudaEventDestroy(t.end); }
     for (cudaEvent_t e : ctx->free_events) cudaEventDestroy(e);
     delete ctx;
@@ -332,27 +337,52 @@ extern "C" int grf_step_host(grf_ctx* ctx, int32_t N, const int32_t* rowptr, con
         GRF_CUDA_TRY(cudaMemcpyAsync(ctx->h_col.ptr, col, E * 4, cudaMemcpyHostToDevice, s));
         GRF_CUDA_TRY(cudaMemcpyAsync(ctx->h_w.ptr, w, E * 4, cudaMemcpyHostToDevice, s));
     }
-    // phi(Q), phi(K), V travel on a second stream while the features are sampled on the context's stream
+    // The problems are handled in parts: the inputs of part p travel on a second stream while the features are
+    // sampled and the earlier parts are computed; its outputs leave on a third stream while the next part runs.
     if (!ctx->copy_stream) {
         GRF_CUDA_TRY(cudaStreamCreateWithFlags(&ctx->copy_stream, cudaStreamNonBlocking));
-        GRF_CUDA_TRY(cudaEventCreateWithFlags(&ctx->copy_done, cudaEventDisableTiming));
+        GRF_CUDA_TRY(cudaStreamCreateWithFlags(&ctx->down_stream, cudaStreamNonBlocking));
+        for (int p = 0; p < grf_ctx::HOST_PARTS; ++p) {
+            GRF_CUDA_TRY(cudaEventCreateWithFlags(&ctx->up_done[p], cudaEventDisableTiming));
+            GRF_CUDA_TRY(cudaEventCreateWithFlags(&ctx->part_done[p], cudaEventDisableTiming));
+        }
+        GRF_CUDA_TRY(cudaEventCreateWithFlags(&ctx->down_done, cudaEventDisableTiming));
     }
-    GRF_CUDA_TRY(cudaMemcpyAsync(ctx->h_q.ptr, phiQ, qk_bytes, cudaMemcpyHostToDevice, ctx->copy_stream));
-    GRF_CUDA_TRY(cudaMemcpyAsync(ctx->h_k.ptr, phiK, qk_bytes, cudaMemcpyHostToDevice, ctx->copy_stream));
-    GRF_CUDA_TRY(cudaMemcpyAsync(ctx->h_v.ptr, V, v_bytes, cudaMemcpyHostToDevice, ctx->copy_stream));
-    GRF_CUDA_TRY(cudaEventRecord(ctx->copy_done, ctx->copy_stream));
+    const int parts = G >= 2 * grf_ctx::HOST_PARTS ? grf_ctx::HOST_PARTS : (G >= 2 ? 2 : 1);
+    const int32_t gp = (G + parts - 1) / parts;           // problems per part
+    for (int p = 0; p < parts; ++p) {
+        const int32_t g0 = p * gp, gc = g0 + gp <= G ? gp : G - g0;
+        if (gc <= 0) break;
+        const size_t qo = (size_t)g0 * N * m * es, vo = (size_t)g0 * N * d * es;
+        const size_t qb = (size_t)gc * N * m * es, vb = (size_t)gc * N * d * es;
+        GRF_CUDA_TRY(cudaMemcpyAsync((char*)ctx->h_q.ptr + qo, (const char*)phiQ + qo, qb, cudaMemcpyHostToDevice, ctx->copy_stream));
+        GRF_CUDA_TRY(cudaMemcpyAsync((char*)ctx->h_k.ptr + qo, (const char*)phiK + qo, qb, cudaMemcpyHostToDevice, ctx->copy_stream));
+        GRF_CUDA_TRY(cudaMemcpyAsync((char*)ctx->h_v.ptr + vo, (const char*)V + vo, vb, cudaMemcpyHostToDevice, ctx->copy_stream));
+        GRF_CUDA_TRY(cudaEventRecord(ctx->up_done[p], ctx->copy_stream));
+    }
     GRF_TRY(grf_sample(ctx, N, (const int32_t*)ctx->h_rowptr.ptr, (const int32_t*)ctx->h_col.ptr,
                        (const float*)ctx->h_w.ptr, seed, n_walks, p_halt, max_len, f_phi, f_psi, &ctx->h_feat));
-    // workspace: everything if it is modest, else chunks of about 1 GiB
+    // workspace: one part's records if that is modest, else chunks of about 1 GiB
     const size_t per = ws_per_problem(N, m, d, dtype);
-    size_t want = per * (size_t)G;
+    size_t want = per * (size_t)gp;
     const size_t cap = (size_t)1 << 31;
     if (want > cap) want = per * (cap / per > 0 ? cap / per : 1);
     GRF_TRY(grf_buf_reserve(&ctx->h_ws, want));
-    GRF_CUDA_TRY(cudaStreamWaitEvent(s, ctx->copy_done, 0));
-    GRF_TRY(grf_masked_linear_attn(ctx, ctx->h_feat, G, N, m, d, dtype, ctx->h_q.ptr, ctx->h_k.ptr, ctx->h_v.ptr,
-                                   ctx->h_out.ptr, nullptr, ctx->h_ws.ptr, ctx->h_ws.bytes));
-    GRF_CUDA_TRY(cudaMemcpyAsync(out, ctx->h_out.ptr, v_bytes, cudaMemcpyDeviceToHost, s));
+    for (int p = 0; p < parts; ++p) {
+        const int32_t g0 = p * gp, gc = g0 + gp <= G ? gp : G - g0;
+        if (gc <= 0) break;
+        const size_t qo = (size_t)g0 * N * m * es, vo = (size_t)g0 * N * d * es;
+        GRF_CUDA_TRY(cudaStreamWaitEvent(s, ctx->up_done[p], 0));
+        GRF_TRY(grf_masked_linear_attn(ctx, ctx->h_feat, gc, N, m, d, dtype, (const char*)ctx->h_q.ptr + qo,
+                                       (const char*)ctx->h_k.ptr + qo, (const char*)ctx->h_v.ptr + vo,
+                                       (char*)ctx->h_out.ptr + vo, nullptr, ctx->h_ws.ptr, ctx->h_ws.bytes));
+        GRF_CUDA_TRY(cudaEventRecord(ctx->part_done[p], s));
+        GRF_CUDA_TRY(cudaStreamWaitEvent(ctx->down_stream, ctx->part_done[p], 0));
+        GRF_CUDA_TRY(cudaMemcpyAsync((char*)out + vo, (const char*)ctx->h_out.ptr + vo, (size_t)gc * N * d * es,
+                                     cudaMemcpyDeviceToHost, ctx->down_stream));
+    }
+    GRF_CUDA_TRY(cudaEventRecord(ctx->down_done, ctx->down_stream));
+    GRF_CUDA_TRY(cudaStreamWaitEvent(s, ctx->down_done, 0));
     return grf_ctx_check(ctx);
 }
 

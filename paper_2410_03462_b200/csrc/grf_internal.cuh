@@ -43,8 +43,11 @@ struct grf_ctx {
     // host-buffer path
     grf_buf h_rowptr, h_col, h_w, h_q, h_k, h_v, h_out, h_ws;
     grf_features* h_feat = nullptr;
-    cudaStream_t copy_stream = nullptr;   // host-buffer path: inputs of the attention are uploaded beside the sampler
-    cudaEvent_t copy_done = nullptr;
+    // host-buffer path: phi(Q), phi(K), V are uploaded on one stream and the outputs downloaded on another, in
+    // parts of a few problems each, beside the sampler and the attention of the other parts
+    static constexpr int HOST_PARTS = 2;
+    cudaStream_t copy_stream = nullptr, down_stream = nullptr;
+    cudaEvent_t up_done[HOST_PARTS] = {}, part_done[HOST_PARTS] = {}, down_done = nullptr;
     int32_t* pinned = nullptr;      // small pinned host block for read-backs
     int* error_word = nullptr;      // device word set by a kernel that gave up a bounded wait
     bool use_tensor_cores = true;
