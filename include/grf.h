@@ -135,7 +135,8 @@ int grf_csr_transpose_noalloc(int device, void* cuda_stream, int32_t rows, int32
                               int32_t* t_rowptr, int32_t* t_col, float* t_val);
 
 /* Bytes of DEVICE workspace with which grf_masked_linear_attn processes all G problems in one pass
- * (per problem and node one record: the state S_l, m x d in the storage type, followed by z_l, m fp32 values).  A smaller workspace is accepted
+ * (per problem and node one record: the state S_l, m x d in the storage type, followed by z_l, m fp32 values,
+ * and with bf16 storage by z_l once more in bf16).  A smaller workspace is accepted
  * as long as it holds one problem; the call then works through G in chunks.  0 on invalid arguments. */
 size_t grf_attn_workspace_bytes(int32_t G, int32_t R, int32_t m, int32_t d, int dtype);
 

@@ -258,7 +258,9 @@ static size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
 // per-problem workspace: R records (state tile in the storage type, then z in fp32), 256-byte aligned
 static size_t ws_per_problem(int32_t R, int32_t m, int32_t d, int dtype)
 {
-    return align256((size_t)R * ((size_t)m * d * elem_size(dtype) + (size_t)m * sizeof(float)));
+    // one record per node: the state tile, z (fp32) and, with bf16 storage, z once more in bf16
+    return align256((size_t)R * ((size_t)m * d * elem_size(dtype) + (size_t)m * sizeof(float) +
+                                 (dtype == GRF_DTYPE_BF16 ? (size_t)m * 2 : 0)));
 }
 
 extern "C" size_t grf_attn_workspace_bytes(int32_t G, int32_t R, int32_t m, int32_t d, int dtype)

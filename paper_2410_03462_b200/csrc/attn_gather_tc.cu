@@ -163,7 +163,7 @@ template <int M, int D> struct TcShape {
     static constexpr int NA = 3;                              // A stages: groups written ahead of the one being multiplied
     static constexpr int TMEM_COLS = pow2_at_least(D + NA * GU * A_COLS);       // accumulator + A ring
     static constexpr int TILE_BYTES = M * D * 2;
-    static constexpr int REC_BYTES = TILE_BYTES + M * 4;      // state tile followed by z
+    static constexpr int REC_BYTES = TILE_BYTES + M * 4 + M * 2;   // state tile, z (fp32), z (bf16)
     static constexpr int CHUNK_BYTES = GU * TILE_BYTES;        // only the tiles are copied to shared memory
     static constexpr int SMEM_BUDGET = TMEM_COLS <= 256 ? 104 * 1024 : 200 * 1024;   // two CTAs per SM, or one
     static constexpr int NBC_WANT = SMEM_BUDGET / CHUNK_BYTES;
@@ -406,7 +406,8 @@ gather_contract_tc_kernel(int32_t N, int32_t R, const int32_t* __restrict__ plan
 
 // ---------------------------------------------------------------------------------------------------
 // Denominators of Eq. 12 for the tensor-core path: den_i = phi(q_i) . (sum_l Phi_il z_l), one warp per
-// (problem, query), lanes across the m feature components, z_l read coalesced from the records.
+// (problem, query); m/2 lanes take one node's z_l (its bf16 copy in the record, two components per lane), so a
+// warp handles 64/m nodes side by side.
 
 template <int M, int D>
 __global__ void __launch_bounds__(256)
@@ -414,35 +415,47 @@ row_denominators_kernel(int32_t N, int32_t R, const int32_t* __restrict__ rowptr
                         const float* __restrict__ val, const __nv_bfloat16* __restrict__ phiQ,
                         const unsigned char* __restrict__ records, float* __restrict__ den)
 {
-    constexpr int MA = (M + 31) / 32;                       // feature components per lane
-    constexpr size_t REC = (size_t)M * D * 2 + (size_t)M * 4;
+    constexpr int LPL = M / 2 < 32 ? M / 2 : 32;            // lanes per node: each takes pairs of components (bf16 x 2)
+    constexpr int LPW = 32 / LPL;                           // nodes handled side by side in a warp
+    constexpr int NT = (M / 2) / LPL;                       // pairs per lane
+    constexpr size_t REC = (size_t)M * D * 2 + (size_t)M * 4 + (size_t)M * 2;
     const int lane = threadIdx.x & 31;
+    const int sub = lane / LPL, pl = lane % LPL;
     const int32_t i = blockIdx.x * 8 + (threadIdx.x >> 5);
     const int32_t g = blockIdx.y;
     if (i >= N) return;
-    const unsigned char* zbase = records + (size_t)g * R * REC + (size_t)M * D * 2;
-    float zbar[MA];
+    const unsigned char* zbase = records + (size_t)g * R * REC + (size_t)M * D * 2 + (size_t)M * 4;   // the bf16 copy of z
+    float z0[NT], z1[NT];
 #pragma unroll
-    for (int t = 0; t < MA; ++t) zbar[t] = 0.0f;
+    for (int t = 0; t < NT; ++t) { z0[t] = 0.0f; z1[t] = 0.0f; }
     const int32_t beg = rowptr[i], end = rowptr[i + 1];
     for (int32_t p0 = beg; p0 < end; p0 += 32) {
         const int32_t n = min(32, end - p0);
         const int32_t c_mine = lane < n ? __ldg(col + p0 + lane) : 0;
         const float v_mine = lane < n ? __ldg(val + p0 + lane) : 0.0f;
-        for (int32_t j = 0; j < n; ++j) {
-            const int32_t l = __shfl_sync(0xffffffffu, c_mine, j);
-            const float phi = __shfl_sync(0xffffffffu, v_mine, j);
-            const float* zl = reinterpret_cast<const float*>(zbase + (size_t)l * REC);
+        for (int32_t j = 0; j < n; j += LPW) {
+            const int32_t jj = j + sub;
+            const int32_t l = __shfl_sync(0xffffffffu, c_mine, jj & 31);
+            const float phi = __shfl_sync(0xffffffffu, v_mine, jj & 31);
+            if (jj < n) {
+                const uint32_t* zl = reinterpret_cast<const uint32_t*>(zbase + (size_t)l * REC);
 #pragma unroll
-            for (int t = 0; t < MA; ++t)
-                if (M >= 32 || lane < M) zbar[t] = fmaf(phi, __ldg(zl + lane + 32 * t), zbar[t]);
+                for (int t = 0; t < NT; ++t) {
+                    const uint32_t w = __ldg(zl + pl + LPL * t);
+                    z0[t] = fmaf(phi, __uint_as_float(w << 16), z0[t]);
+                    z1[t] = fmaf(phi, __uint_as_float(w & 0xffff0000u), z1[t]);
+                }
+            }
         }
     }
-    const __nv_bfloat16* q = phiQ + ((size_t)g * N + i) * M;
+    const uint32_t* q = reinterpret_cast<const uint32_t*>(phiQ + ((size_t)g * N + i) * M);
     float d = 0.0f;
 #pragma unroll
-    for (int t = 0; t < MA; ++t)
-        if (M >= 32 || lane < M) d = fmaf(__bfloat162float(q[lane + 32 * t]), zbar[t], d);
+    for (int t = 0; t < NT; ++t) {
+        const uint32_t w = __ldg(q + pl + LPL * t);
+        d = fmaf(__uint_as_float(w << 16), z0[t], d);
+        d = fmaf(__uint_as_float(w & 0xffff0000u), z1[t], d);
+    }
 #pragma unroll
     for (int off = 1; off < 32; off <<= 1) d += __shfl_xor_sync(0xffffffffu, d, off);
     if (lane == 0) den[(size_t)g * N + i] = d;

@@ -104,6 +104,11 @@ build_states_kernel(int32_t R, int32_t N, const int32_t* __restrict__ t_rowptr, 
         float* zl = reinterpret_cast<float*>(rec + (size_t)M * D * sizeof(T));
 #pragma unroll
         for (int c = 0; c < CH; ++c) zl[kc * CH + c] = zacc[c];
+        if constexpr (sizeof(T) == 2) {
+            __nv_bfloat16* zb = reinterpret_cast<__nv_bfloat16*>(rec + (size_t)M * D * sizeof(T) + (size_t)M * sizeof(float));
+#pragma unroll
+            for (int c = 0; c < CH; ++c) zb[kc * CH + c] = __float2bfloat16_rn(zacc[c]);
+        }
     }
 }
 

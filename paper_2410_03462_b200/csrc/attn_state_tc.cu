@@ -362,6 +362,16 @@ build_states_tc_kernel(int32_t R, int32_t N, const int32_t* __restrict__ t_rowpt
                         for (int e = 0; e < 16; e += 4)
                             *reinterpret_cast<float4*>(zl + c0 + e) = make_float4(__uint_as_float(r[e]), __uint_as_float(r[e + 1]),
                                                                                   __uint_as_float(r[e + 2]), __uint_as_float(r[e + 3]));
+                        // and once more in bf16, for the denominators kernel
+                        uint32_t zw[8];
+#pragma unroll
+                        for (int e = 0; e < 8; ++e) {
+                            __nv_bfloat162 t2 = __floats2bfloat162_rn(__uint_as_float(r[2 * e]), __uint_as_float(r[2 * e + 1]));
+                            zw[e] = *reinterpret_cast<uint32_t*>(&t2);
+                        }
+                        uint4* zb = reinterpret_cast<uint4*>(rec + (size_t)M * D * 2 + (size_t)M * 4 + (size_t)c0 * 2);
+                        zb[0] = make_uint4(zw[0], zw[1], zw[2], zw[3]);
+                        zb[1] = make_uint4(zw[4], zw[5], zw[6], zw[7]);
                     }
                 }
             }
@@ -668,6 +678,16 @@ build_states_tma_kernel(int32_t R, int32_t N, const int32_t* __restrict__ t_rowp
                         for (int e = 0; e < 16; e += 4)
                             *reinterpret_cast<float4*>(zl + c0 + e) = make_float4(__uint_as_float(r[e]), __uint_as_float(r[e + 1]),
                                                                                   __uint_as_float(r[e + 2]), __uint_as_float(r[e + 3]));
+                        // and once more in bf16, for the denominators kernel
+                        uint32_t zw[8];
+#pragma unroll
+                        for (int e = 0; e < 8; ++e) {
+                            __nv_bfloat162 t2 = __floats2bfloat162_rn(__uint_as_float(r[2 * e]), __uint_as_float(r[2 * e + 1]));
+                            zw[e] = *reinterpret_cast<uint32_t*>(&t2);
+                        }
+                        uint4* zb = reinterpret_cast<uint4*>(rec + (size_t)M * D * 2 + (size_t)M * 4 + (size_t)c0 * 2);
+                        zb[0] = make_uint4(zw[0], zw[1], zw[2], zw[3]);
+                        zb[1] = make_uint4(zw[4], zw[5], zw[6], zw[7]);
                     }
                 }
             }

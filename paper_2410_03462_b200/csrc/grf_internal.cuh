@@ -140,11 +140,12 @@ template <typename T> __host__ __device__ constexpr size_t grf_tile_index(int a,
     return ((size_t)(a / grf_tile_chunk<T>()) * D + b) * grf_tile_chunk<T>() + (a % grf_tile_chunk<T>());
 }
 
-// The workspace holds one record per (problem, node): the state tile S_l followed by z_l (m fp32 values), so
-// that one contiguous copy brings both.
+// The workspace holds one record per (problem, node): the state tile S_l, then z_l (m fp32 values) and, with
+// bf16 storage, z_l once more rounded to bf16 (the denominators kernel of the tensor-core path reads that copy:
+// half the bytes per (query, node) pair).
 template <typename T> __host__ __device__ constexpr size_t grf_record_bytes(int M, int D)
 {
-    return (size_t)M * D * sizeof(T) + (size_t)M * sizeof(float);
+    return (size_t)M * D * sizeof(T) + (size_t)M * sizeof(float) + (sizeof(T) == 2 ? (size_t)M * 2 : 0);
 }
 
 static inline int grf_ceil_div(int64_t a, int64_t b) { return (int)((a + b - 1) / b); }
