@@ -66,10 +66,6 @@ extern "C" int grf_ctx_destroy(grf_ctx* ctx)
     if (ctx->h_feat) grf_features_free(ctx->h_feat);
     if (ctx->pinned) cudaFreeHost(ctx->pinned);
     if (ctx->error_word) cudaFree(ctx->error_word);
-    if (ctx->aux_stream) {
-        cudaStreamSynchronize(ctx->aux_stream); cudaStreamDestroy(ctx->aux_stream);
-        cudaEventDestroy(ctx->aux_fork); cudaEventDestroy(ctx->aux_join);
-    }
     if (ctx->copy_stream) {
         cudaStreamSynchronize(ctx->copy_stream); cudaStreamSynchronize(ctx->down_stream);
         cudaStreamDestroy(ctx->copy_stream); cudaStreamDestroy(ctx->down_stream);
@@ -90,19 +86,18 @@ static cudaEvent_t take_event(grf_ctx* c)
     return e;
 }
 
-grf_launch_scope::grf_launch_scope(grf_ctx* c, int cls_, int n_launches, cudaStream_t on)
-    : ctx(c), cls(cls_), n(n_launches), stream(on ? on : c->stream)
+grf_launch_scope::grf_launch_scope(grf_ctx* c, int cls_, int n_launches) : ctx(c), cls(cls_), n(n_launches)
 {
     if (!ctx->timing) return;
     beg = take_event(ctx); end = take_event(ctx);
-    if (beg && end) cudaEventRecord(beg, stream);
+    if (beg && end) cudaEventRecord(beg, ctx->stream);
 }
 
 grf_launch_scope::~grf_launch_scope()
 {
     ctx->launches += n;
     if (!ctx->timing || !beg || !end) return;
-    cudaEventRecord(end, stream);
+    cudaEventRecord(end, ctx->stream);
     ctx->timed.push_back({cls, beg, end});
 }
 

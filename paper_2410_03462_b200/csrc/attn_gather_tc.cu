@@ -247,8 +247,7 @@ gather_contract_tc_kernel(int32_t N, int32_t R, const int32_t* __restrict__ plan
         uint2 cur = make_uint2(0u, 0u);
         uint2 nxt1 = nquads > 0 ? __ldg(tab) : make_uint2(0u, 0u);
         uint2 nxt2 = nquads > 1 ? __ldg(tab + BQ) : make_uint2(0u, 0u);
-        // den_in == nullptr: the sums are written as they are and divided by a later kernel
-        const float den = !den_in ? 1.0f : (live ? den_in[(size_t)g * N + row] : 0.0f);
+        const float den = live ? den_in[(size_t)g * N + row] : 0.0f;
         bool ok = true;
         const uint32_t lane_field = (uint32_t)(warp * 32) << 16;
         for (int32_t gi = 0; gi < ngroups; ++gi) {
@@ -622,26 +621,6 @@ int grf_build_block_plan(grf_ctx* ctx, grf_features* feat)
     return GRF_OK;
 }
 
-// out[g, i, :] /= den[g, i] (0 where the denominator is 0), one thread per 16 bytes of a row
-template <int D>
-__global__ void __launch_bounds__(256)
-divide_rows_kernel(int64_t rows, const float* __restrict__ den, __nv_bfloat16* __restrict__ out)
-{
-    constexpr int CPR = D / 8;
-    const int64_t x = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (x >= rows * CPR) return;
-    const float dn = den[x / CPR];
-    const float inv = dn != 0.0f ? 1.0f / dn : 0.0f;
-    uint4 v = reinterpret_cast<uint4*>(out)[x];
-    uint32_t* w = reinterpret_cast<uint32_t*>(&v);
-#pragma unroll
-    for (int e = 0; e < 4; ++e) {
-        const __nv_bfloat162 h = __floats2bfloat162_rn(__uint_as_float(w[e] << 16) * inv, __uint_as_float(w[e] & 0xffff0000u) * inv);
-        w[e] = *reinterpret_cast<const uint32_t*>(&h);
-    }
-    reinterpret_cast<uint4*>(out)[x] = v;
-}
-
 template <int M, int D>
 static int launch_tc(grf_ctx* ctx, const grf_features* feat, int32_t G, int32_t N,
                      const void* phiQ, const void* records, void* out, float* den_out)
@@ -655,36 +634,21 @@ static int launch_tc(grf_ctx* ctx, const grf_features* feat, int32_t G, int32_t 
         GRF_TRY(grf_buf_reserve(&ctx->den_scratch, sizeof(float) * (size_t)G * N));
         den = (float*)ctx->den_scratch.ptr;
     }
-    // The denominators need only the records, not the products: they are computed on a side stream while the
-    // gather-and-contract kernel runs (it leaves most of the load/store bandwidth idle), and a short kernel
-    // divides the rows afterwards.
-    if (!ctx->aux_stream) {
-        GRF_CUDA_TRY(cudaStreamCreateWithFlags(&ctx->aux_stream, cudaStreamNonBlocking));
-        GRF_CUDA_TRY(cudaEventCreateWithFlags(&ctx->aux_fork, cudaEventDisableTiming));
-        GRF_CUDA_TRY(cudaEventCreateWithFlags(&ctx->aux_join, cudaEventDisableTiming));
-    }
-    GRF_CUDA_TRY(cudaEventRecord(ctx->aux_fork, ctx->stream));
-    GRF_CUDA_TRY(cudaStreamWaitEvent(ctx->aux_stream, ctx->aux_fork, 0));
+    // (Running the denominators on a side stream beside the gather kernel was measured: both draw on the same
+    // L2 bandwidth, the pair ends 0.1 ms earlier at most, and the rows then need a second pass to be divided.)
     {
-        grf_launch_scope scope(ctx, 6, 1, ctx->aux_stream);
-        row_denominators_kernel<M, D><<<dim3(grf_ceil_div(N, 8), G), 256, 0, ctx->aux_stream>>>(
+        grf_launch_scope scope(ctx, 6);
+        row_denominators_kernel<M, D><<<dim3(grf_ceil_div(N, 8), G), 256, 0, ctx->stream>>>(
             N, phi.cols, (const int32_t*)phi.rowptr.ptr, (const int32_t*)phi.col.ptr, (const float*)phi.val.ptr,
             (const __nv_bfloat16*)phiQ, (const unsigned char*)records, den);
     }
-    GRF_CUDA_TRY(cudaEventRecord(ctx->aux_join, ctx->aux_stream));
     const dim3 grid(feat->plan_blocks, G);
     {
         grf_launch_scope scope(ctx, 5);
         gather_contract_tc_kernel<M, D><<<grid, TC_THREADS, Sh::SMEM, ctx->stream>>>(
             N, phi.cols, (const int32_t*)feat->plan_off.ptr, (const int32_t*)feat->plan_cnt.ptr,
             (const int32_t*)feat->plan_col.ptr, (const uint2*)feat->plan_coef.ptr, (const __nv_bfloat16*)phiQ,
-            (const unsigned char*)records, (__nv_bfloat16*)out, (const float*)nullptr, ctx->error_word);
-    }
-    GRF_CUDA_TRY(cudaStreamWaitEvent(ctx->stream, ctx->aux_join, 0));
-    {
-        grf_launch_scope scope(ctx, 6);
-        const int64_t pieces = (int64_t)G * N * (D / 8);
-        divide_rows_kernel<D><<<(unsigned)grf_ceil_div(pieces, 256), 256, 0, ctx->stream>>>((int64_t)G * N, den, (__nv_bfloat16*)out);
+            (const unsigned char*)records, (__nv_bfloat16*)out, den, ctx->error_word);
     }
     return cudaGetLastError() == cudaSuccess ? GRF_OK : GRF_ERR_CUDA;
 }

@@ -43,9 +43,6 @@ struct grf_ctx {
     // host-buffer path
     grf_buf h_rowptr, h_col, h_w, h_q, h_k, h_v, h_out, h_ws;
     grf_features* h_feat = nullptr;
-    // side stream of the attention: the denominators are computed beside the gather-and-contract kernel
-    cudaStream_t aux_stream = nullptr;
-    cudaEvent_t aux_fork = nullptr, aux_join = nullptr;
     // host-buffer path: phi(Q), phi(K), V are uploaded on one stream and the outputs downloaded on another, in
     // parts of a few problems each, beside the sampler and the attention of the other parts
     static constexpr int HOST_PARTS = 2;
@@ -67,8 +64,7 @@ struct grf_launch_scope {
     int cls;
     int n;
     cudaEvent_t beg = nullptr, end = nullptr;
-    cudaStream_t stream;
-    grf_launch_scope(grf_ctx* c, int cls_, int n_launches = 1, cudaStream_t on = nullptr);   // on = nullptr: the context's stream
+    grf_launch_scope(grf_ctx* c, int cls_, int n_launches = 1);
     ~grf_launch_scope();
 };
 
