@@ -5,15 +5,16 @@
 //     D[128 x d] += A_l[128 x m] * S_l[m x d],      A_l[i, a] = Phi_il * phi(q_i)_a   (0 where Phi_il = 0)
 // is m/16 tcgen05.mma instructions (M = 128, N = d, K = 16) accumulating in tensor memory: the sum over l
 // of Eq. 12 becomes the K dimension of one long matrix product, evaluated in a fixed order.
-//   - the record of node l (S_l in operand layout, then z_l) arrives by one contiguous bulk async copy into
-//     a ring of shared-memory slots; records further ahead are prefetched into L2;
-//   - A_l lives in tensor memory: each of the 128 "row" threads owns one query (= one TMEM lane), walks its
-//     own CSR row of Phi in step with the union list and stores its scaled phi(q) (or zeros) with tcgen05.st;
-//     so the MMA reads only S_l from shared memory;
-//   - two warps issue the MMAs for alternate groups of union entries into two accumulators (one issuing
-//     thread cannot keep the tensor pipe busy with N = d this small); one tcgen05.commit per group frees both
-//     the A slots and the record slots of that group; the epilogue adds the two accumulators, divides by the
-//     denominators (accumulated by the row threads from z_l) and writes the block's outputs;
+//   - the state tile of node l (S_l in operand layout, the head of its record) arrives by one contiguous bulk
+//     async copy into a ring of shared-memory slots, four tiles per landing barrier; the loader reads the node
+//     indices one group ahead of the copies;
+//   - A_l lives in tensor memory: each of the 128 "row" threads owns one query (= one TMEM lane), reads its
+//     coefficients Phi_il from the plan's dense table and stores its scaled phi(q) (zeros for most rows) with
+//     tcgen05.st, so the MMA reads only S_l from shared memory; three groups of A operands are in flight;
+//   - one warp issues the MMAs: its loop is warp-uniform and an elected lane issues (the same instruction
+//     issued from a single-lane branch costs about three times as much); one tcgen05.commit per group frees
+//     both the A slots and the record slots of that group; the epilogue divides by the denominators (a
+//     separate kernel, below) and writes the block's outputs;
 //   - every mbarrier wait is bounded: a wait that outlasts its limit raises an error word and the CTA drains
 //     its copies and MMAs, frees its tensor memory and exits.
 // Nodes that no query of the block touches are never loaded; a tile is loaded once per block, not once
@@ -34,10 +35,6 @@ __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
 __device__ __forceinline__ void mbar_arrive(uint32_t bar)
 {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes)
-{
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
 }
 __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
 {
@@ -63,12 +60,6 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
             else if (now - t0 > WAIT_CYCLES) { *abort_flag = 1; return false; }
         }
     }
-}
-
-__device__ __forceinline__ void bulk_copy_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar)
-{
-    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
 }
 
 // Shared-memory operand descriptor: unswizzled, 8-row core matrices of 128 contiguous bytes;
