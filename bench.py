@@ -120,6 +120,7 @@ def algorithmic_bytes(w, N, nnz_phi, nnz_psi, E):
     G, m, d = w.G, w.m, w.d
     S = G * N * m * d * es
     z = G * N * m * 4
+    zb = G * N * m * 2 if w.dtype == "bf16" else 0          # bf16 copy of z in the records
     csr = lambda nnz: nnz * 8 + (N + 1) * 4
     return {
         # graph read once; merged rows written once
@@ -128,11 +129,11 @@ def algorithmic_bytes(w, N, nnz_phi, nnz_psi, E):
         "compact": 2 * (nnz_phi + nnz_psi) * 8,
         "regroup": 3 * csr(nnz_psi),
         # phi(K), V, Psi^T read once; S and z written once
-        "build_states": G * N * (m + d) * es + csr(nnz_psi) + S + z,
+        "build_states": G * N * (m + d) * es + csr(nnz_psi) + S + z + zb,
         # S, z, phi(Q), Phi read once; out written once
         "gather_contract": S + z + G * N * m * es + csr(nnz_phi) + G * N * d * es,
         # z and Phi read once, denominators written once
-        "row_denominators": z + csr(nnz_phi) + G * N * m * es + G * N * 4,
+        "row_denominators": (zb if zb else z) + csr(nnz_phi) + G * N * m * es + G * N * 4,
         # Phi read twice (union lists, coefficient table)
         "block_plan": 2 * csr(nnz_phi),
     }
