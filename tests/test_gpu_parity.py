@@ -154,6 +154,41 @@ def test_attention_shapes_random_features(lib, m, d, dtype):
     feat.free()
 
 
+@pytest.mark.parametrize("m,d", [(16, 64), (32, 64), (64, 64), (32, 32)])
+def test_state_kernels_key_count_edges(lib, m, d):
+    """Nodes with 0, 1, 15 ... 200 keys: empty items, items that end on and next to the 16-key steps and the
+    64-key item boundary, nodes of several items; more than 64 nodes, so that two CTAs share the work."""
+    api, B, ctx = lib
+    rng = np.random.default_rng(7 * m + d)
+    N, G = 256, 2
+    lengths = [0, 1, 15, 16, 17, 63, 64, 65, 127, 128, 129, 200] * 6      # R = 72 nodes
+    R = len(lengths)
+    cols_of_node = [np.sort(rng.choice(N, size=c, replace=False)) for c in lengths]
+    rows = [[] for _ in range(N)]
+    for l, js in enumerate(cols_of_node):
+        for j in js:
+            rows[j].append(l)
+    rowptr = np.zeros(N + 1, np.int32); col = []; val = []
+    for j in range(N):
+        col += rows[j]; val += list(rng.uniform(0.1, 1.0, len(rows[j]))); rowptr[j + 1] = len(col)
+    Psi = oracle.CSR(rowptr, np.array(col, np.int32), np.array(val, np.float32), None, (N, R))
+    prow = [0]; pcol = []; pval = []
+    for _ in range(N):
+        c = np.sort(rng.choice(R, size=rng.integers(1, 8), replace=False))
+        pcol += list(c); pval += list(rng.uniform(0.1, 1.0, len(c))); prow.append(len(pcol))
+    Phi = oracle.CSR(np.array(prow, np.int32), np.array(pcol, np.int32), np.array(pval, np.float32), None, (N, R))
+    feat = api.features_from_csr(ctx, N, R, (Phi.rowptr, Phi.col, Phi.val), (Psi.rowptr, Psi.col, Psi.val))
+    PsiT = oracle.transpose(Psi)
+    assert list(np.diff(PsiT.rowptr)) == lengths
+    q, k, v = tensors.qkv(G, N, m, d, "bf16", 11)
+    ref = oracle.attn_sparse(tensors.widen(q), tensors.widen(k), tensors.widen(v), Phi, PsiT)
+    out, den = api.masked_linear_attn(ctx, feat, q.cuda(), k.cuda(), v.cuda(), want_den=True)
+    B.grf_ctx_check(ctx.handle)
+    helpers.assert_attn_close(out.float().cpu().numpy(), ref, helpers.TOL["bf16"], den.cpu().numpy(), f"key edges m{m} d{d}",
+                              min_ok=0.5)
+    feat.free()
+
+
 def test_identity_features_return_values(lib):
     api, B, ctx = lib
     N, G, m, d = 300, 2, 32, 64
