@@ -399,9 +399,11 @@ gather_contract_tc_kernel(int32_t N, int32_t R, const int32_t* __restrict__ plan
 // (problem, query); m/2 lanes take one node's z_l (its bf16 copy in the record, two components per lane), so a
 // warp handles 64/m nodes side by side.
 
+constexpr int DEN_GH = 4;   // problems per warp of the denominators kernel: they share the row's indices and coefficients
+
 template <int M, int D>
 __global__ void __launch_bounds__(256)
-row_denominators_kernel(int32_t N, int32_t R, const int32_t* __restrict__ rowptr, const int32_t* __restrict__ col,
+row_denominators_kernel(int32_t G, int32_t N, int32_t R, const int32_t* __restrict__ rowptr, const int32_t* __restrict__ col,
                         const float* __restrict__ val, const __nv_bfloat16* __restrict__ phiQ,
                         const unsigned char* __restrict__ records, float* __restrict__ den)
 {
@@ -412,12 +414,15 @@ row_denominators_kernel(int32_t N, int32_t R, const int32_t* __restrict__ rowptr
     const int lane = threadIdx.x & 31;
     const int sub = lane / LPL, pl = lane % LPL;
     const int32_t i = blockIdx.x * 8 + (threadIdx.x >> 5);
-    const int32_t g = blockIdx.y;
+    const int32_t g0 = blockIdx.y * DEN_GH;
     if (i >= N) return;
-    const unsigned char* zbase = records + (size_t)g * R * REC + (size_t)M * D * 2 + (size_t)M * 4;   // the bf16 copy of z
-    float z0[NT], z1[NT];
+    const size_t gstride = (size_t)R * REC;                 // from one problem's records to the next one's
+    const unsigned char* zbase = records + (size_t)g0 * gstride + (size_t)M * D * 2 + (size_t)M * 4;   // the bf16 copy of z
+    float z0[DEN_GH][NT], z1[DEN_GH][NT];
 #pragma unroll
-    for (int t = 0; t < NT; ++t) { z0[t] = 0.0f; z1[t] = 0.0f; }
+    for (int h = 0; h < DEN_GH; ++h)
+#pragma unroll
+        for (int t = 0; t < NT; ++t) { z0[h][t] = 0.0f; z1[h][t] = 0.0f; }
     const int32_t beg = rowptr[i], end = rowptr[i + 1];
     for (int32_t p0 = beg; p0 < end; p0 += 32) {
         const int32_t n = min(32, end - p0);
@@ -428,27 +433,38 @@ row_denominators_kernel(int32_t N, int32_t R, const int32_t* __restrict__ rowptr
             const int32_t l = __shfl_sync(0xffffffffu, c_mine, jj & 31);
             const float phi = __shfl_sync(0xffffffffu, v_mine, jj & 31);
             if (jj < n) {
-                const uint32_t* zl = reinterpret_cast<const uint32_t*>(zbase + (size_t)l * REC);
+                const uint32_t* zl = reinterpret_cast<const uint32_t*>(zbase + (size_t)l * REC) + pl;
+                uint32_t w[DEN_GH][NT];
 #pragma unroll
-                for (int t = 0; t < NT; ++t) {
-                    const uint32_t w = __ldg(zl + pl + LPL * t);
-                    z0[t] = fmaf(phi, __uint_as_float(w << 16), z0[t]);
-                    z1[t] = fmaf(phi, __uint_as_float(w & 0xffff0000u), z1[t]);
-                }
+                for (int h = 0; h < DEN_GH; ++h)
+#pragma unroll
+                    for (int t = 0; t < NT; ++t)
+                        w[h][t] = g0 + h < G ? __ldg(reinterpret_cast<const uint32_t*>(reinterpret_cast<const unsigned char*>(zl) + (size_t)h * gstride) + LPL * t) : 0u;
+#pragma unroll
+                for (int h = 0; h < DEN_GH; ++h)
+#pragma unroll
+                    for (int t = 0; t < NT; ++t) {
+                        z0[h][t] = fmaf(phi, __uint_as_float(w[h][t] << 16), z0[h][t]);
+                        z1[h][t] = fmaf(phi, __uint_as_float(w[h][t] & 0xffff0000u), z1[h][t]);
+                    }
             }
         }
     }
-    const uint32_t* q = reinterpret_cast<const uint32_t*>(phiQ + ((size_t)g * N + i) * M);
-    float d = 0.0f;
 #pragma unroll
-    for (int t = 0; t < NT; ++t) {
-        const uint32_t w = __ldg(q + pl + LPL * t);
-        d = fmaf(__uint_as_float(w << 16), z0[t], d);
-        d = fmaf(__uint_as_float(w & 0xffff0000u), z1[t], d);
+    for (int h = 0; h < DEN_GH; ++h) {
+        if (g0 + h >= G) break;
+        const uint32_t* q = reinterpret_cast<const uint32_t*>(phiQ + ((size_t)(g0 + h) * N + i) * M);
+        float d = 0.0f;
+#pragma unroll
+        for (int t = 0; t < NT; ++t) {
+            const uint32_t w = __ldg(q + pl + LPL * t);
+            d = fmaf(__uint_as_float(w << 16), z0[h][t], d);
+            d = fmaf(__uint_as_float(w & 0xffff0000u), z1[h][t], d);
+        }
+#pragma unroll
+        for (int off = 1; off < 32; off <<= 1) d += __shfl_xor_sync(0xffffffffu, d, off);
+        if (lane == 0) den[(size_t)(g0 + h) * N + i] = d;
     }
-#pragma unroll
-    for (int off = 1; off < 32; off <<= 1) d += __shfl_xor_sync(0xffffffffu, d, off);
-    if (lane == 0) den[(size_t)g * N + i] = d;
 }
 
 // ---------------------------------------------------------------------------------------------------
@@ -629,8 +645,8 @@ static int launch_tc(grf_ctx* ctx, const grf_features* feat, int32_t G, int32_t 
     // L2 bandwidth, the pair ends 0.1 ms earlier at most, and the rows then need a second pass to be divided.)
     {
         grf_launch_scope scope(ctx, 6);
-        row_denominators_kernel<M, D><<<dim3(grf_ceil_div(N, 8), G), 256, 0, ctx->stream>>>(
-            N, phi.cols, (const int32_t*)phi.rowptr.ptr, (const int32_t*)phi.col.ptr, (const float*)phi.val.ptr,
+        row_denominators_kernel<M, D><<<dim3(grf_ceil_div(N, 8), grf_ceil_div(G, DEN_GH)), 256, 0, ctx->stream>>>(
+            G, N, phi.cols, (const int32_t*)phi.rowptr.ptr, (const int32_t*)phi.col.ptr, (const float*)phi.val.ptr,
             (const __nv_bfloat16*)phiQ, (const unsigned char*)records, den);
     }
     const dim3 grid(feat->plan_blocks, G);
