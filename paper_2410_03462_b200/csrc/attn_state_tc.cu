@@ -525,19 +525,12 @@ build_states_tma_kernel(int32_t R, int32_t N, const int32_t* __restrict__ t_rowp
             const int32_t nitems = wc > 0 ? (wc + ITEM_KEYS - 1) / ITEM_KEYS : 1;
             if (++wit >= nitems) { ++wn; wit = 0; wbeg = node_beg[min(wn, nn)]; wc = node_beg[min(wn + 1, nn)] - wbeg; }
         };
-        struct Idx { int32_t nkeys, j[4], jlo, jhi; float p0, p1; };
+        struct Idx { int32_t nkeys, jlo, jhi; float p0, p1; };    // lane x holds key x (jlo) and key x + 32 (jhi)
         auto read_idx = [&]() {
             Idx x; x.nkeys = 0; x.p0 = 0.0f; x.p1 = 0.0f; x.jlo = -1; x.jhi = -1;
-#pragma unroll
-            for (int e = 0; e < 4; ++e) x.j[e] = 0;
             if (wn < nn) {
                 x.nkeys = min(ITEM_KEYS, wc - wit * ITEM_KEYS);
                 const int32_t pos = wbeg + wit * ITEM_KEYS;
-                if (x.nkeys > 0) {
-#pragma unroll
-                    for (int e = 0; e < 4; ++e)      // beyond the item's keys: repeat its last key (it meets a zero row)
-                        x.j[e] = __ldg(t_col + pos + min(4 * y4 + e, x.nkeys - 1));
-                }
                 if (lane < x.nkeys) { x.jlo = __ldg(t_col + pos + lane); x.p0 = __ldg(t_val + pos + lane); }
                 if (lane + 32 < x.nkeys) { x.jhi = __ldg(t_col + pos + lane + 32); x.p1 = __ldg(t_val + pos + lane + 32); }
             }
@@ -555,9 +548,17 @@ build_states_tma_kernel(int32_t R, int32_t N, const int32_t* __restrict__ t_rowp
                 asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;"
                              ::"r"(landed(s)), "r"((uint32_t)rows * 128u) : "memory");
             __syncwarp();
+            // lane y (< 16) gathers the value rows of keys 4y .. 4y+3; the keys come from the lanes that hold them;
+            // beyond the item's keys its last key is repeated (the row meets a zero row of phi(k))
+            int32_t r4[4];
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                const int32_t key = min(4 * y4 + e, max(cur.nkeys - 1, 0));
+                const int32_t a = __shfl_sync(0xffffffffu, cur.jlo, key & 31), b = __shfl_sync(0xffffffffu, cur.jhi, key & 31);
+                r4[e] = row0 + max(key < 32 ? a : b, 0);
+            }
             if (lane < 16 && 4 * y4 < rows)
-                tma_gather4(st + (uint32_t)y4 * 512u, &map_v, row0 + cur.j[0], row0 + cur.j[1], row0 + cur.j[2],
-                            row0 + cur.j[3], landed(s));
+                tma_gather4(st + (uint32_t)y4 * 512u, &map_v, r4[0], r4[1], r4[2], r4[3], landed(s));
 #pragma unroll
             for (int y = 0; y < NIK; ++y) {
                 const int32_t j = __shfl_sync(0xffffffffu, y < NIK / 2 ? cur.jlo : cur.jhi, (KPK * y + lane / CK) & 31);
