@@ -199,9 +199,10 @@ def attn_sparse(phiQ, phiK, V, Phi: CSR, PsiT: CSR, with_abs: bool = True):
     return dict(num=num, den=den, out=out, num_abs=num_abs, den_abs=den_abs)
 
 
-def attn_bruteforce(phiQ, phiK, V, Mhat: np.ndarray, rows=None):
-    """Eqs. 1-2 with the low-rank kernel of Eq. 3: A = (phiQ phiK^T) * Mhat, out = D^-1 A V, in fp64.
-    `Mhat` is a dense N x N mask (e.g. Phi Psi^T).  `rows` optionally restricts the queries."""
+def attn_bruteforce(phiQ, phiK, V, Mhat: np.ndarray, rows=None, kernel: str = "linear"):
+    """Eqs. 1-2: A = S * Mhat, out = D^-1 A V, in fp64, with S = phiQ phiK^T (Eq. 3, kernel="linear") or
+    S = exp(Q K^T) (softmax attention, kernel="exp").  `Mhat` is a dense N x N mask (e.g. Phi Psi^T, or Phi
+    itself for asymmetric features).  `rows` optionally restricts the queries."""
     Q = np.asarray(phiQ, dtype=np.float64)
     K = np.asarray(phiK, dtype=np.float64)
     Vd = np.asarray(V, dtype=np.float64)
@@ -211,7 +212,8 @@ def attn_bruteforce(phiQ, phiK, V, Mhat: np.ndarray, rows=None):
     num = np.empty((G, len(rows), Vd.shape[2])); den = np.empty((G, len(rows)))
     num_abs = np.empty_like(num); den_abs = np.empty_like(den)
     for g in range(G):
-        A = (Q[g][rows] @ K[g].T) * Mr
+        S = Q[g][rows] @ K[g].T
+        A = (np.exp(S) if kernel == "exp" else S) * Mr
         num[g] = A @ Vd[g]
         den[g] = A.sum(axis=1)
         num_abs[g] = np.abs(A) @ np.abs(Vd[g])      # sums of the absolute values of the terms
@@ -231,4 +233,28 @@ def mask_rows(Phi: CSR, Psi: CSR, rows) -> np.ndarray:
             l = Phi.col[p]
             s, e = PsiT.rowptr[l], PsiT.rowptr[l + 1]
             np.add.at(out[r], PsiT.col[s:e], float(Phi.val[p]) * PsiT.val[s:e].astype(np.float64))
+    return out
+
+
+def attn_asym_walks(Q, K, V, traj, load, f, kernel: str = "linear"):
+    """Alg. 2 as printed (asymmetric features), in fp64, for ensemble 0 of `traj`/`load`: for every node i, every
+    walk out of i and every step t of it, the visited node j contributes A_ij * f_t * load_t to the output
+    feature (times v_j) and to the normalisation; the result is the quotient (the 1/n cancels)."""
+    Qd = np.asarray(Q, dtype=np.float64); Kd = np.asarray(K, dtype=np.float64); Vd = np.asarray(V, dtype=np.float64)
+    G, N, _ = Qd.shape
+    _, _, n, Lp1 = traj.shape
+    out = np.zeros((G, N, Vd.shape[2]))
+    for g in range(G):
+        for i in range(N):
+            feat = np.zeros(Vd.shape[2]); norm = 0.0
+            for k in range(n):
+                for t in range(Lp1):
+                    j = traj[0, i, k, t]
+                    if j < 0:
+                        break
+                    s = float(Qd[g, i] @ Kd[g, j])
+                    a = np.exp(s) if kernel == "exp" else s
+                    wgt = a * float(f[t]) * float(load[0, i, k, t])
+                    feat += wgt * Vd[g, j]; norm += wgt
+            out[g, i] = feat / norm if norm != 0.0 else 0.0
     return out

@@ -413,3 +413,38 @@ def test_asymmetric_route_equals_walk_accumulation():
                 a = float(qd[i] @ kd[j]) * float(f_phi[t]) * float(load[0, i, kk, t])
                 acc += a * vd[j]; s += a
         assert np.allclose(got["out"][0, i], acc / s, rtol=1e-5, atol=1e-7)
+
+
+# ----------------------------------------------------------------------------- asymmetric features (Alg. 2)
+
+def test_softmax_kernel_with_all_ones_mask_is_plain_softmax_attention():
+    """A = exp(QK^T) with the mask 1 everywhere is softmax attention: a library routine pins the exp branch."""
+    from scipy.special import softmax
+    rng = np.random.default_rng(3)
+    Q = rng.standard_normal((2, 9, 5)) * 0.5; K = rng.standard_normal((2, 9, 5)) * 0.5; V = rng.standard_normal((2, 9, 4))
+    got = oracle.attn_bruteforce(Q, K, V, np.ones((9, 9)), kernel="exp")["out"]
+    want = np.stack([softmax(Q[g] @ K[g].T, axis=1) @ V[g] for g in range(2)])
+    assert np.allclose(got, want, rtol=1e-12, atol=1e-14)
+
+
+def test_asymmetric_route_three_ways():
+    """Psi = I (f_psi = delta_0): the S/z route of Eq. 12, the dense definition with Mhat = Phi and the walk
+    loop of Alg. 2 (which never forms Phi) give the same attention, for both similarity kernels where they apply."""
+    w = configs.tiny()
+    g = w.graph()
+    f_phi = w.alpha.astype(np.float32)
+    f_psi = np.zeros(w.max_len + 1, np.float32); f_psi[0] = 1.0
+    Phi, Psi, PsiT, traj, load = oracle.sample(g.rowptr, g.col, g.w, 11, w.n_walks, w.p_halt, w.max_len, f_phi, f_psi)
+    assert Psi.nnz == g.N and np.array_equal(Psi.col, np.arange(g.N)) and np.all(Psi.val == 1.0)
+    rng = np.random.default_rng(5)
+    f32 = lambda x: x.astype(np.float32).astype(np.float64)      # values that the fp32 interface of the S/z route keeps
+    Q = f32(np.abs(rng.standard_normal((2, g.N, 6))) + 0.05); K = f32(np.abs(rng.standard_normal((2, g.N, 6))) + 0.05)
+    V = f32(rng.standard_normal((2, g.N, 3)))
+    dense = oracle.attn_bruteforce(Q, K, V, Phi.dense())["out"]
+    sz = oracle.attn_sparse(Q, K, V, Phi, PsiT)["out"]
+    walks = oracle.attn_asym_walks(Q, K, V, traj, load, f_phi)
+    assert np.allclose(dense, sz, rtol=1e-10, atol=1e-12)
+    assert np.allclose(dense, walks, rtol=1e-5, atol=1e-7)       # Phi's entries are fp32 sums of the walk terms
+    dense_e = oracle.attn_bruteforce(Q * 0.3, K * 0.3, V, Phi.dense(), kernel="exp")["out"]
+    walks_e = oracle.attn_asym_walks(Q * 0.3, K * 0.3, V, traj, load, f_phi, kernel="exp")
+    assert np.allclose(dense_e, walks_e, rtol=1e-5, atol=1e-7)
