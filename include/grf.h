@@ -36,6 +36,10 @@ extern "C" {
 #define GRF_DTYPE_F32  0
 #define GRF_DTYPE_BF16 1
 
+/* similarity A_ij of grf_masked_attn_asym */
+#define GRF_KERNEL_LINEAR  0   /* A_ij = phi(q_i) . phi(k_j): the caller passes phi(Q), phi(K) */
+#define GRF_KERNEL_SOFTMAX 1   /* A_ij = exp(q_i . k_j): the caller passes Q, K (scaled as it wishes) */
+
 #define GRF_MAX_WALK_LEN 255     /* largest max_len accepted by the sampler */
 
 typedef struct grf_ctx grf_ctx;            /* device id, stream, reusable scratch                         */
@@ -153,6 +157,23 @@ size_t grf_attn_workspace_bytes(int32_t G, int32_t R, int32_t m, int32_t d, int 
 int grf_masked_linear_attn(grf_ctx* ctx, const grf_features* feat, int32_t G, int32_t N, int32_t m, int32_t d,
                            int dtype, const void* phiQ, const void* phiK, const void* V,
                            void* out, float* den_out, void* workspace, size_t workspace_bytes);
+
+/*
+ * Masked attention with ASYMMETRIC graph random features (App. "Asymmetric graph random features", Alg. 2):
+ * when the key-side modulation is f^(2) = delta_0 the key features are the identity, the mask estimate is
+ * Phi itself, and
+ *   out_i = sum_l Phi_il A_il v_l / sum_l Phi_il A_il    over the non-zeros of row i of Phi,
+ * with A_il = phi(q_i) . phi(k_l) (GRF_KERNEL_LINEAR) or exp(q_i . k_l) (GRF_KERNEL_SOFTMAX); m + d
+ * multiply-adds per non-zero, no workspace.  Only feat's Phi is used (N x N; sample it with f_phi = alpha
+ * and f_psi = delta_0, or pass any CSR through grf_features_from_csr).  Q, K [G][N][m], V, out [G][N][d]:
+ * DEVICE, row-major, 16-byte aligned, dtype GRF_DTYPE_F32 or _BF16 (sums in fp32); m, d in
+ * {8, 16, 32, 64, 128}; G <= 65535.  den_out: optional DEVICE fp32 [G][N] receiving the denominators (with
+ * the softmax kernel relative to exp(largest score of the row), which cancels in out).  A row whose
+ * denominator is exactly 0 yields out = 0.  Summation order is fixed; asynchronous.
+ */
+int grf_masked_attn_asym(grf_ctx* ctx, const grf_features* feat, int32_t G, int32_t N, int32_t m, int32_t d,
+                         int dtype, int kernel, const void* Q, const void* K, const void* V, void* out,
+                         float* den_out);
 
 /*
  * The whole path of Alg. 1 from HOST buffers, for callers that keep nothing on the device:

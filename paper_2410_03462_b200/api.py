@@ -109,3 +109,14 @@ def masked_linear_attn(ctx: Context, feat: Features, phiQ, phiK, V, workspace=No
     B.grf_masked_linear_attn(ctx.handle, feat.handle, G, N, m, d, dt, phiQ, phiK, V, out, den, workspace,
                              workspace.numel())
     return (out, den) if want_den else out
+
+
+def masked_attn_asym(ctx: Context, feat: Features, Q, K, V, softmax=False, want_den=False):
+    """Alg. 2 (asymmetric features: the mask estimate is Phi).  Q, K [G,N,m], V [G,N,d] CUDA tensors."""
+    G, N, m = Q.shape
+    d = V.shape[2]
+    out = torch.empty_like(V)
+    den = torch.empty((G, N), dtype=torch.float32, device=V.device) if want_den else None
+    B.grf_masked_attn_asym(ctx.handle, feat.handle, G, N, m, d, B.dtype_code(Q),
+                           B.GRF_KERNEL_SOFTMAX if softmax else B.GRF_KERNEL_LINEAR, Q, K, V, out, den)
+    return (out, den) if want_den else out

@@ -16,6 +16,7 @@ GRF_OK = 0
 GRF_ERR_INVALID, GRF_ERR_TOO_LARGE, GRF_ERR_WORKSPACE, GRF_ERR_CUDA, GRF_ERR_NOMEM, GRF_ERR_BADGRAPH = -1, -2, -3, -4, -5, -6
 GRF_ERR_TIMEOUT = -7
 GRF_DTYPE_F32, GRF_DTYPE_BF16 = 0, 1
+GRF_KERNEL_LINEAR, GRF_KERNEL_SOFTMAX = 0, 1
 
 _LIB_PATH = _build.LIB
 if not os.path.exists(_LIB_PATH):
@@ -40,6 +41,7 @@ _SIGNATURES = {
     "grf_csr_transpose_noalloc": (_int, [_int, _vp, _i32, _i32, _i64, _vp, _vp, _vp, _vp, _vp, _vp]),
     "grf_attn_workspace_bytes": (_sz, [_i32, _i32, _i32, _i32, _int]),
     "grf_masked_linear_attn": (_int, [_vp, _vp, _i32, _i32, _i32, _i32, _int, _vp, _vp, _vp, _vp, _vp, _vp, _sz]),
+    "grf_masked_attn_asym": (_int, [_vp, _vp, _i32, _i32, _i32, _i32, _int, _int, _vp, _vp, _vp, _vp, _vp]),
     "grf_step_host": (_int, [_vp, _i32, _vp, _vp, _vp, _u64, _i32, _f32, _i32, _vp, _vp,
                              _i32, _i32, _i32, _int, _vp, _vp, _vp, _vp]),
     "grf_ctx_launch_count": (_i64, [_vp]),
@@ -202,6 +204,11 @@ def grf_masked_linear_attn(ctx, features, G, N, m, d, dtype, phiQ, phiK, V, out,
     _check(lib.grf_masked_linear_attn(ctx, features, G, N, m, d, dtype, _dev(phiQ), _dev(phiK), _dev(V),
                                       _dev(out), _dev(den_out), _dev(workspace), workspace_bytes),
            "grf_masked_linear_attn")
+
+
+def grf_masked_attn_asym(ctx, features, G, N, m, d, dtype, kernel, Q, K, V, out, den_out):
+    _check(lib.grf_masked_attn_asym(ctx, features, G, N, m, d, dtype, kernel, _dev(Q), _dev(K), _dev(V), _dev(out),
+                                    _dev(den_out)), "grf_masked_attn_asym")
 
 
 def grf_step_host(ctx, N, rowptr, col, w, seed, n_walks, p_halt, max_len, f_phi, f_psi, G, m, d, dtype,

@@ -189,6 +189,65 @@ def test_state_kernels_key_count_edges(lib, m, d):
     feat.free()
 
 
+@pytest.mark.parametrize("dtype", ["fp32", "bf16"])
+@pytest.mark.parametrize("softmax", [False, True])
+def test_asymmetric_attention_matches_oracle(lib, dtype, softmax):
+    """Alg. 2: features sampled with f_psi = delta_0; the fused kernel against the dense definition with
+    Mhat = Phi, and (linear kernel) against the general S/z path on the same feature object."""
+    api, B, ctx = lib
+    w = configs.point_cloud_4096(1024)
+    g = w.graph()
+    f_phi = w.alpha.astype(np.float32)
+    f_psi = np.zeros(w.max_len + 1, np.float32); f_psi[0] = 1.0
+    feat = api.sample(ctx, api.DeviceGraph(g), configs.WALK_SEED, w.n_walks, w.p_halt, w.max_len, f_phi, f_psi)
+    Phi, Psi, PsiT, _, _ = helpers.oracle_features(w, g, configs.WALK_SEED, f_phi, f_psi)
+    G = 3
+    q, k, v = tensors.qkv(G, g.N, w.m, w.d, dtype, configs.QKV_SEED)
+    if softmax:
+        q = (q.float() * 0.25).to(q.dtype); k = (k.float() * 0.25).to(k.dtype)
+    ref = oracle.attn_bruteforce(tensors.widen(q), tensors.widen(k), tensors.widen(v), Phi.dense(),
+                                 kernel="exp" if softmax else "linear")
+    out, den = api.masked_attn_asym(ctx, feat, q.cuda(), k.cuda(), v.cuda(), softmax=softmax, want_den=True)
+    B.grf_ctx_check(ctx.handle)
+    den_h = den.cpu().numpy()
+    if softmax:     # the kernel's denominators are relative to exp(row maximum): compare the quotient only
+        den_h = None
+    helpers.assert_attn_close(out.float().cpu().numpy(), ref, helpers.TOL[dtype], den_h, f"asym softmax={softmax} {dtype}")
+    if not softmax:
+        general = api.masked_linear_attn(ctx, feat, q.cuda(), k.cuda(), v.cuda())
+        B.grf_ctx_check(ctx.handle)
+        tol = 2e-2 if dtype == "bf16" else 1e-5
+        assert torch.allclose(out.float(), general.float(), rtol=tol, atol=tol)
+    # run-to-run identical
+    again = api.masked_attn_asym(ctx, feat, q.cuda(), k.cuda(), v.cuda(), softmax=softmax)
+    assert torch.equal(out, again)
+    feat.free()
+
+
+@pytest.mark.parametrize("m,d", [(8, 8), (16, 128), (128, 16), (64, 64), (32, 32)])
+def test_asymmetric_attention_shapes(lib, m, d):
+    api, B, ctx = lib
+    rng = np.random.default_rng(m + 7 * d)
+    N, G = 203, 2
+    rowptr = [0]; col = []; val = []
+    for i in range(N):
+        c = np.sort(rng.choice(N, size=rng.integers(0, 70), replace=False))      # empty rows and rows of 3 batches
+        col += list(c); val += list(rng.uniform(0.1, 1.0, len(c))); rowptr.append(len(col))
+    Phi = oracle.CSR(np.array(rowptr, np.int32), np.array(col, np.int32), np.array(val, np.float32), None, (N, N))
+    eye = (np.arange(N + 1, dtype=np.int32), np.arange(N, dtype=np.int32), np.ones(N, np.float32))
+    feat = api.features_from_csr(ctx, N, N, (Phi.rowptr, Phi.col, Phi.val), eye)
+    for dtype in ("fp32", "bf16"):
+        q, k, v = tensors.qkv(G, N, m, d, dtype, 3)
+        for softmax in (False, True):
+            qq, kk = (q, k) if not softmax else ((q.float() * 0.2).to(q.dtype), (k.float() * 0.2).to(k.dtype))
+            ref = oracle.attn_bruteforce(tensors.widen(qq), tensors.widen(kk), tensors.widen(v), Phi.dense(),
+                                         kernel="exp" if softmax else "linear")
+            out = api.masked_attn_asym(ctx, feat, qq.cuda(), kk.cuda(), v.cuda(), softmax=softmax)
+            B.grf_ctx_check(ctx.handle)
+            helpers.assert_attn_close(out.float().cpu().numpy(), ref, helpers.TOL[dtype], None, f"asym m{m} d{d} {dtype} softmax={softmax}")
+    feat.free()
+
+
 def test_identity_features_return_values(lib):
     api, B, ctx = lib
     N, G, m, d = 300, 2, 32, 64
