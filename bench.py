@@ -172,11 +172,19 @@ def run_ours(args):
         w.name += f"-heads{args.heads}"
     g = w.graph()
     N, E = g.N, g.E
-    f = B.grf_deconvolve(w.alpha).astype(np.float32)
+    asym = args.route == "asym"
+    if asym:      # Alg. 2: f_phi = alpha, f_psi = delta_0 (no key-side walks contribute, Psi = I)
+        f = w.alpha.astype(np.float32)
+        f_psi = np.zeros(w.max_len + 1, np.float32); f_psi[0] = 1.0
+    else:
+        f = B.grf_deconvolve(w.alpha).astype(np.float32)
+        f_psi = None
     ctx = api.Context(local)
     dg = api.DeviceGraph(g, local)
     # every rank has its own batch of the same shape (weak scaling over independent problems)
     q, k, v = tensors.qkv(w.G, N, w.m, w.d, w.dtype, rank_seed(configs.QKV_SEED, rank))
+    if asym and args.softmax:     # keep the exponents moderate
+        q, k = (q.float() * 0.25).to(q.dtype), (k.float() * 0.25).to(k.dtype)
     qd, kd, vd = q.cuda(), k.cuda(), v.cuda()
     dt = B.dtype_code(qd)
     ws_bytes = B.grf_attn_workspace_bytes(w.G, N, w.m, w.d, dt)
@@ -185,10 +193,17 @@ def run_ours(args):
     flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
     feat = api.Features(ctx, None)
 
+    def attention():
+        if asym:
+            B.grf_masked_attn_asym(ctx.handle, feat.handle, w.G, N, w.m, w.d, dt,
+                                   B.GRF_KERNEL_SOFTMAX if args.softmax else B.GRF_KERNEL_LINEAR, qd, kd, vd, out, None)
+        else:
+            B.grf_masked_linear_attn(ctx.handle, feat.handle, w.G, N, w.m, w.d, dt, qd, kd, vd, out, None, ws, ws_bytes)
+
     def step(i):
         feat.handle = B.grf_sample(ctx.handle, N, dg.rowptr, dg.col, dg.w, configs.WALK_SEED + i, w.n_walks, w.p_halt,
-                                   w.max_len, f, None, feat.handle)
-        B.grf_masked_linear_attn(ctx.handle, feat.handle, w.G, N, w.m, w.d, dt, qd, kd, vd, out, None, ws, ws_bytes)
+                                   w.max_len, f, f_psi, feat.handle)
+        attention()
 
     sampler = ClockSampler(local) if rank == 0 else None
     B.grf_ctx_enable_timing(ctx.handle, True)      # per-kernel events exist before the timed region starts
@@ -214,9 +229,9 @@ def run_ours(args):
         flush.zero_()
         evs[i][0].record()
         feat.handle = B.grf_sample(ctx.handle, N, dg.rowptr, dg.col, dg.w, configs.WALK_SEED + 1000 + i, w.n_walks,
-                                   w.p_halt, w.max_len, f, None, feat.handle)
+                                   w.p_halt, w.max_len, f, f_psi, feat.handle)
         ev_mid[i].record()
-        B.grf_masked_linear_attn(ctx.handle, feat.handle, w.G, N, w.m, w.d, dt, qd, kd, vd, out, None, ws, ws_bytes)
+        attention()
         evs[i][1].record()
     barrier()
     wall = time.perf_counter() - t_wall0
@@ -241,15 +256,17 @@ def run_ours(args):
         B.grf_step_host(ctx.handle, N, rp_h, c_h, w_h, configs.WALK_SEED + 2000 + i, w.n_walks, w.p_halt, w.max_len,
                         f, None, w.G, w.m, w.d, dt, qh, kh, vh, oh)
 
-    host_step(0)
-    barrier()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record()
-    for i in range(e2e_steps):
-        host_step(1 + i)
-    e1.record()
-    barrier()
-    e2e_ms = e0.elapsed_time(e1) / e2e_steps
+    e2e_ms = float("nan")
+    if not asym:
+        host_step(0)
+        barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for i in range(e2e_steps):
+            host_step(1 + i)
+        e1.record()
+        barrier()
+        e2e_ms = e0.elapsed_time(e1) / e2e_steps
     h2d = (rp_h.numel() + c_h.numel() + w_h.numel()) * 4 + sum(t.numel() * t.element_size() for t in (qh, kh, vh))
     d2h = oh.numel() * oh.element_size()
 
@@ -271,6 +288,9 @@ def run_ours(args):
     if rank == 0:
         peak_gbs, peak_kind = peaks()
         alg = algorithmic_bytes(w, N, nnz_phi, nnz_psi, E)
+        if asym:   # Q, K, V, Phi read once, out written once; no states
+            es = 2 if w.dtype == "bf16" else 4
+            alg["gather_contract"] = w.G * N * (2 * w.m + 2 * w.d) * es + nnz_phi * 8 + (N + 1) * 4
         per_kernel = {}
         for name, (ms, n) in ktimes.items():
             per = ms / max(n, 1)
@@ -289,14 +309,17 @@ def run_ours(args):
                        "n_walks": w.n_walks, "p_halt": w.p_halt, "max_len": w.max_len,
                        "nnz_phi": nnz_phi, "nnz_psi": nnz_psi,
                        "l2": "256 MiB flush write between steps, outside the per-step events",
-                       "step": "grf_sample (both ensembles) + grf_masked_linear_attn, features resampled every step"},
+                       "step": ("grf_sample (f_psi = delta_0) + grf_masked_attn_asym (Alg. 2, %s similarity), features "
+                                "resampled every step" % ("softmax" if args.softmax else "linear")) if asym else
+                               "grf_sample (both ensembles) + grf_masked_linear_attn, features resampled every step"},
             "clocks": clocks,
             "gpu_launches": launches,
-            "e2e": {"value": tokens_per_step / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+            "e2e": None if asym else
+                   {"value": tokens_per_step / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
                     "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms, "entry_point": "grf_step_host"},
             "roofline": {"kernel": dom, "bound": "hbm", "achieved": achieved, "peak": peak_gbs, "unit": "GB/s",
                          "frac": achieved / peak_gbs, "peak_source": peak_kind,
-                         "traffic": NCU_TRAFFIC_BYTES.get(w.name, {}).get(dom),
+                         "traffic": None if asym else NCU_TRAFFIC_BYTES.get(w.name, {}).get(dom),
                          "algorithmic_bytes": alg[dom], "ms_per_launch": dom_ms},
             "phases": {"sample_ms": statistics.mean(sample_ms), "attn_ms": statistics.mean(attn_ms),
                        "sample_ms_min_med_max": [min(sample_ms), statistics.median(sample_ms), max(sample_ms)],
@@ -369,6 +392,10 @@ def main():
     ap.add_argument("--workload", default="pc32768")
     ap.add_argument("--cpu-heads", type=int, default=1, help="problems of the batch the CPU baseline really runs")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--route", choices=["sz", "asym"], default="sz",
+                    help="sz: Alg. 1 (per-node states, the default); asym: Alg. 2 (asymmetric features, Psi = I), "
+                         "a variant outside the headline metric, no end-to-end leg")
+    ap.add_argument("--softmax", action="store_true", help="with --route asym: A_ij = exp(q_i . k_j)")
     ap.add_argument("--heads", type=int, default=0, help="override the workload's head count (profiling of a smaller case)")
     args = ap.parse_args()
     if args.warmup < 3 and args.impl == "ours":
