@@ -5,8 +5,9 @@
 // over the nodes l that the walkers out of node i visited: m + d multiply-adds per non-zero of Phi, no
 // per-node states at all.
 //
-// One warp per (problem, query).  Non-zeros are taken 32 at a time: lane t computes the whole dot product of
-// the batch's t-th key row with the query (the query sits in shared memory and is read as a broadcast), then
+// One warp per query and two problems (they share the row's indices and mask values).  Non-zeros are taken
+// 32 at a time: lane t computes the whole dot product of the batch's t-th key row with the query (the query
+// sits in shared memory and is read as a broadcast), then
 // the lanes spread over the d output columns and the batch's value rows are added one after the other, each
 // read as one coalesced row.  The exponentials are taken relative to a running maximum of the scores, which
 // cancels in the quotient; sums are carried in fp32 in a fixed order, so results are run-to-run identical.
@@ -45,33 +46,40 @@ template <> struct Row<__nv_bfloat16> {
 };
 
 constexpr int ASYM_WARPS = 8;
+constexpr int ASYM_GH = 2;      // problems per warp: they share the row's indices and mask values
 
 template <typename T, int M, int D, bool SOFTMAX>
 __global__ void __launch_bounds__(ASYM_WARPS * 32)
-asym_attention_kernel(int32_t N, const int32_t* __restrict__ rowptr, const int32_t* __restrict__ col,
+asym_attention_kernel(int32_t G, int32_t N, const int32_t* __restrict__ rowptr, const int32_t* __restrict__ col,
                       const float* __restrict__ val, const T* __restrict__ Q, const T* __restrict__ K,
                       const T* __restrict__ V, T* __restrict__ out, float* __restrict__ den_out)
 {
     constexpr int CH = Row<T>::CH;
     constexpr int EPL = D >= 32 ? D / 32 : 1;        // output columns per lane
-    __shared__ float qs[ASYM_WARPS][M];
+    constexpr int GH = ASYM_GH;
+    __shared__ float qs[ASYM_WARPS][GH][M];
 
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int32_t i = blockIdx.x * ASYM_WARPS + warp;
-    const int32_t g = blockIdx.y;
+    const int32_t g0 = blockIdx.y * GH;
     if (i >= N) return;
-    const T* qrow = Q + ((size_t)g * N + i) * M;
-    for (int a = lane; a < M; a += 32) qs[warp][a] = Row<T>::get(qrow + a);
+#pragma unroll
+    for (int h = 0; h < GH; ++h) {
+        const int32_t g = min(g0 + h, G - 1);        // a problem beyond the batch repeats the last one and is not written
+        const T* qrow = Q + ((size_t)g * N + i) * M;
+        for (int a = lane; a < M; a += 32) qs[warp][h][a] = Row<T>::get(qrow + a);
+    }
     __syncwarp();
-    const T* Kg = K + (size_t)g * N * M;
-    const T* Vg = V + (size_t)g * N * D;
     const bool col_lane = lane * EPL < D;            // lanes that own output columns
 
-    float acc[EPL];
+    float acc[GH][EPL];
+    float den[GH], run_max[GH];                      // this lane's share of the denominators; softmax: running maxima
 #pragma unroll
-    for (int e = 0; e < EPL; ++e) acc[e] = 0.0f;
-    float den = 0.0f;                                // this lane's share of the denominator
-    float run_max = -INFINITY;                       // softmax only: maximum of the scores seen so far
+    for (int h = 0; h < GH; ++h) {
+        den[h] = 0.0f; run_max[h] = -INFINITY;
+#pragma unroll
+        for (int e = 0; e < EPL; ++e) acc[h][e] = 0.0f;
+    }
 
     const int32_t beg = rowptr[i], end = rowptr[i + 1];
     for (int32_t p0 = beg; p0 < end; p0 += 32) {
@@ -79,82 +87,95 @@ asym_attention_kernel(int32_t N, const int32_t* __restrict__ rowptr, const int32
         const bool valid = lane < n;
         const int32_t l = valid ? __ldg(col + p0 + lane) : 0;
         const float phi = valid ? __ldg(val + p0 + lane) : 0.0f;
-        // score of this lane's key: the whole dot product in one lane
-        float s = 0.0f;
-        if (valid) {
-            const T* krow = Kg + (size_t)l * M;
+        float w[GH];
 #pragma unroll
-            for (int c = 0; c < M / CH; ++c) {
-                float v[CH];
-                Row<T>::load(krow + c * CH, v);
+        for (int h = 0; h < GH; ++h) {
+            const int32_t g = min(g0 + h, G - 1);
+            // score of this lane's key: the whole dot product in one lane
+            float s = 0.0f;
+            if (valid) {
+                const T* krow = K + ((size_t)g * N + l) * M;
 #pragma unroll
-                for (int e = 0; e < CH; ++e) s = fmaf(v[e], qs[warp][c * CH + e], s);
+                for (int c = 0; c < M / CH; ++c) {
+                    float v[CH];
+                    Row<T>::load(krow + c * CH, v);
+#pragma unroll
+                    for (int e = 0; e < CH; ++e) s = fmaf(v[e], qs[warp][h][c * CH + e], s);
+                }
             }
-        }
-        float w;
-        if (SOFTMAX) {
-            float bmax = valid ? s : -INFINITY;
+            if (SOFTMAX) {
+                float bmax = valid ? s : -INFINITY;
 #pragma unroll
-            for (int off = 1; off < 32; off <<= 1) bmax = fmaxf(bmax, __shfl_xor_sync(0xffffffffu, bmax, off));
-            const float new_max = fmaxf(run_max, bmax);
-            const float rescale = __expf(run_max - new_max);     // 0 on the first batch (run_max = -inf)
+                for (int off = 1; off < 32; off <<= 1) bmax = fmaxf(bmax, __shfl_xor_sync(0xffffffffu, bmax, off));
+                const float new_max = fmaxf(run_max[h], bmax);
+                const float rescale = __expf(run_max[h] - new_max);     // 0 on the first batch (run_max = -inf)
 #pragma unroll
-            for (int e = 0; e < EPL; ++e) acc[e] *= rescale;
-            den *= rescale;
-            run_max = new_max;
-            w = valid ? phi * __expf(s - new_max) : 0.0f;
-        } else {
-            w = phi * s;
+                for (int e = 0; e < EPL; ++e) acc[h][e] *= rescale;
+                den[h] *= rescale;
+                run_max[h] = new_max;
+                w[h] = valid ? phi * __expf(s - new_max) : 0.0f;
+            } else {
+                w[h] = phi * s;
+            }
+            den[h] += w[h];
         }
-        den += w;
         // the batch's value rows, one after the other, lanes across the output columns
         for (int32_t t = 0; t < n; ++t) {
-            const float wt = __shfl_sync(0xffffffffu, w, t);
             const int32_t lt = __shfl_sync(0xffffffffu, l, t);
-            if (col_lane) {
-                const T* vrow = Vg + (size_t)lt * D + lane * EPL;
-                if constexpr (sizeof(T) == 2 && EPL == 2) {
-                    const uint32_t x = __ldg(reinterpret_cast<const uint32_t*>(vrow));
-                    acc[0] = fmaf(wt, __uint_as_float(x << 16), acc[0]);
-                    acc[1] = fmaf(wt, __uint_as_float(x & 0xffff0000u), acc[1]);
-                } else if constexpr (sizeof(T) == 2 && EPL == 4) {
-                    const uint2 x = __ldg(reinterpret_cast<const uint2*>(vrow));
-                    acc[0] = fmaf(wt, __uint_as_float(x.x << 16), acc[0]);
-                    acc[1] = fmaf(wt, __uint_as_float(x.x & 0xffff0000u), acc[1]);
-                    acc[2] = fmaf(wt, __uint_as_float(x.y << 16), acc[2]);
-                    acc[3] = fmaf(wt, __uint_as_float(x.y & 0xffff0000u), acc[3]);
-                } else {
 #pragma unroll
-                    for (int e = 0; e < EPL; ++e) acc[e] = fmaf(wt, Row<T>::get(vrow + e), acc[e]);
+            for (int h = 0; h < GH; ++h) {
+                const float wt = __shfl_sync(0xffffffffu, w[h], t);
+                const int32_t g = min(g0 + h, G - 1);
+                if (col_lane) {
+                    const T* vrow = V + ((size_t)g * N + lt) * D + lane * EPL;
+                    if constexpr (sizeof(T) == 2 && EPL == 2) {
+                        const uint32_t x = __ldg(reinterpret_cast<const uint32_t*>(vrow));
+                        acc[h][0] = fmaf(wt, __uint_as_float(x << 16), acc[h][0]);
+                        acc[h][1] = fmaf(wt, __uint_as_float(x & 0xffff0000u), acc[h][1]);
+                    } else if constexpr (sizeof(T) == 2 && EPL == 4) {
+                        const uint2 x = __ldg(reinterpret_cast<const uint2*>(vrow));
+                        acc[h][0] = fmaf(wt, __uint_as_float(x.x << 16), acc[h][0]);
+                        acc[h][1] = fmaf(wt, __uint_as_float(x.x & 0xffff0000u), acc[h][1]);
+                        acc[h][2] = fmaf(wt, __uint_as_float(x.y << 16), acc[h][2]);
+                        acc[h][3] = fmaf(wt, __uint_as_float(x.y & 0xffff0000u), acc[h][3]);
+                    } else {
+#pragma unroll
+                        for (int e = 0; e < EPL; ++e) acc[h][e] = fmaf(wt, Row<T>::get(vrow + e), acc[h][e]);
+                    }
                 }
             }
         }
     }
 #pragma unroll
-    for (int off = 1; off < 32; off <<= 1) den += __shfl_xor_sync(0xffffffffu, den, off);
-    const float inv = den != 0.0f ? 1.0f / den : 0.0f;
-    if (col_lane) {
-        T* orow = out + ((size_t)g * N + i) * D + lane * EPL;
+    for (int h = 0; h < GH; ++h) {
+        float dn = den[h];
 #pragma unroll
-        for (int e = 0; e < EPL; ++e) Row<T>::put(orow + e, acc[e] * inv);
+        for (int off = 1; off < 32; off <<= 1) dn += __shfl_xor_sync(0xffffffffu, dn, off);
+        if (g0 + h >= G) break;
+        const float inv = dn != 0.0f ? 1.0f / dn : 0.0f;
+        if (col_lane) {
+            T* orow = out + ((size_t)(g0 + h) * N + i) * D + lane * EPL;
+#pragma unroll
+            for (int e = 0; e < EPL; ++e) Row<T>::put(orow + e, acc[h][e] * inv);
+        }
+        // with the softmax kernel the reported denominator is relative to exp(max score of the row)
+        if (lane == 0 && den_out) den_out[(size_t)(g0 + h) * N + i] = dn;
     }
-    // with the softmax kernel the reported denominator is relative to exp(max score of the row)
-    if (lane == 0 && den_out) den_out[(size_t)g * N + i] = den;
 }
 
 template <typename T, int M, int D>
 int launch_md(grf_ctx* ctx, const grf_csr_dev& phi, int32_t G, int32_t N, int kernel, const void* Q, const void* K,
               const void* V, void* out, float* den_out)
 {
-    const dim3 grid(grf_ceil_div(N, ASYM_WARPS), G);
+    const dim3 grid(grf_ceil_div(N, ASYM_WARPS), grf_ceil_div(G, ASYM_GH));
     grf_launch_scope scope(ctx, 5);
     if (kernel == GRF_KERNEL_SOFTMAX)
         asym_attention_kernel<T, M, D, true><<<grid, ASYM_WARPS * 32, 0, ctx->stream>>>(
-            N, (const int32_t*)phi.rowptr.ptr, (const int32_t*)phi.col.ptr, (const float*)phi.val.ptr, (const T*)Q,
+            G, N, (const int32_t*)phi.rowptr.ptr, (const int32_t*)phi.col.ptr, (const float*)phi.val.ptr, (const T*)Q,
             (const T*)K, (const T*)V, (T*)out, den_out);
     else
         asym_attention_kernel<T, M, D, false><<<grid, ASYM_WARPS * 32, 0, ctx->stream>>>(
-            N, (const int32_t*)phi.rowptr.ptr, (const int32_t*)phi.col.ptr, (const float*)phi.val.ptr, (const T*)Q,
+            G, N, (const int32_t*)phi.rowptr.ptr, (const int32_t*)phi.col.ptr, (const float*)phi.val.ptr, (const T*)Q,
             (const T*)K, (const T*)V, (T*)out, den_out);
     return GRF_OK;
 }
@@ -194,7 +215,7 @@ extern "C" int grf_masked_attn_asym(grf_ctx* ctx, const grf_features* feat, int3
                                     float* den_out)
 {
     if (!ctx || !feat || !Q || !K || !V || !out) return GRF_ERR_INVALID;
-    if (G <= 0 || G > 65535 || N <= 0) return GRF_ERR_INVALID;
+    if (G <= 0 || G > 65535 * ASYM_GH || N <= 0) return GRF_ERR_INVALID;
     if (kernel != GRF_KERNEL_LINEAR && kernel != GRF_KERNEL_SOFTMAX) return GRF_ERR_INVALID;
     if (dtype != GRF_DTYPE_F32 && dtype != GRF_DTYPE_BF16) return GRF_ERR_INVALID;
     if (feat->phi.rows != N || feat->phi.cols != N) return GRF_ERR_INVALID;       // the mask estimate is Phi: N x N
