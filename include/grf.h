@@ -152,7 +152,9 @@ size_t grf_attn_workspace_bytes(int32_t G, int32_t R, int32_t m, int32_t d, int 
  * GRF_DTYPE_F32 or _BF16 (bf16: S is stored in bf16, sums are carried in fp32).  den_out: optional
  * DEVICE fp32 [G][N] receiving the denominators.  A row whose denominator is exactly 0 yields out = 0.
  * m, d in {8, 16, 32, 64, 128}.  workspace: DEVICE, 256-byte aligned.  Summation order is fixed, so
- * results are run-to-run identical.  Asynchronous.
+ * results are run-to-run identical.  Asynchronous, except that the first bf16 call after the features were
+ * created or resampled prepares a per-block plan of Phi inside the feature object, which waits for the stream
+ * once (so a feature object must not be used by two threads at the same time).
  */
 int grf_masked_linear_attn(grf_ctx* ctx, const grf_features* feat, int32_t G, int32_t N, int32_t m, int32_t d,
                            int dtype, const void* phiQ, const void* phiK, const void* V,

@@ -239,7 +239,7 @@ extern "C" int grf_features_from_csr(grf_ctx* ctx, int32_t N, int32_t R,
     rc = grf_transpose_launch(ctx, N, R, nnz_psi, (const int32_t*)f->psi.rowptr.ptr, (const int32_t*)f->psi.col.ptr,
                               (const float*)f->psi.val.ptr, (int32_t*)f->psit.rowptr.ptr,
                               (int32_t*)f->psit.col.ptr, (float*)f->psit.val.ptr);
-    if (rc == GRF_OK) rc = grf_build_block_plan(ctx, f);
+    if (rc == GRF_OK) { f->plan_stale = true; f->plan_ready = false; }   // built at the first attention that needs it
     if (rc == GRF_OK && cudaGetLastError() != cudaSuccess) rc = GRF_ERR_CUDA;
     if (rc != GRF_OK) { grf_features_free(f); return rc; }
     *out = f;

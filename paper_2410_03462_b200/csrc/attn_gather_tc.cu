@@ -664,7 +664,14 @@ static int launch_tc(grf_ctx* ctx, const grf_features* feat, int32_t G, int32_t 
 int grf_gather_contract_tc(grf_ctx* ctx, const grf_features* feat, int32_t G, int32_t N, int32_t m, int32_t d,
                            const void* phiQ, const void* records, void* out, float* den_out)
 {
-    if (!feat->plan_ready || G > 65535) return 1;
+    if (G > 65535) return 1;
+    if (feat->plan_stale) {
+        // the plan is a cache inside the feature object, built on first use (the asymmetric route never needs it)
+        grf_features* f = const_cast<grf_features*>(feat);
+        GRF_TRY(grf_build_block_plan(ctx, f));
+        f->plan_stale = false;
+    }
+    if (!feat->plan_ready) return 1;
 #define GRF_TC_CASE(MM, DD) \
     if (m == MM && d == DD) return launch_tc<MM, DD>(ctx, feat, G, N, phiQ, records, out, den_out);
     GRF_TC_CASE(16, 16) GRF_TC_CASE(16, 32) GRF_TC_CASE(16, 64) GRF_TC_CASE(16, 128)

@@ -84,6 +84,7 @@ struct grf_features {
     grf_buf plan_coef;              // dense bf16 coefficients [quad of union entries][row of the block][4]
     int32_t plan_blocks = 0;
     bool plan_ready = false;
+    bool plan_stale = true;         // Phi changed since the plan was built: the gather kernel's launcher rebuilds it
 };
 
 int grf_buf_reserve(grf_buf* b, size_t bytes);          // grows (contents not preserved)

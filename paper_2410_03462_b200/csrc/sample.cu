@@ -348,7 +348,9 @@ static int sample_into(grf_ctx* ctx, grf_features* feat, const grf_walk_params& 
                                  (const int32_t*)feat->psi.col.ptr, (const float*)feat->psi.val.ptr,
                                  (int32_t*)feat->psit.rowptr.ptr, (int32_t*)feat->psit.col.ptr,
                                  (float*)feat->psit.val.ptr));
-    return grf_build_block_plan(ctx, feat);
+    feat->plan_stale = true;       // the block plan of Phi is built by the first attention call that needs it
+    feat->plan_ready = false;
+    return GRF_OK;
 }
 
 extern "C" int grf_sample(grf_ctx* ctx, int32_t N, const int32_t* rowptr, const int32_t* col, const float* w,
