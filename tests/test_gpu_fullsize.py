@@ -50,6 +50,38 @@ def test_bench_workload_sampler_and_sampled_attention_rows():
     ctx.close()
 
 
+def test_bench_workload_asymmetric_route_sampled_rows():
+    """Alg. 2 at the bench size (f_psi = delta_0, so the mask estimate is Phi): sampled query rows of both
+    similarities against the brute force of Eqs. 1-2 on the dense rows of Phi."""
+    from paper_2410_03462_b200 import api, binding as B
+    w = configs.point_cloud_32768()
+    g = w.graph()
+    ctx = api.Context(0)
+    f_phi = w.alpha.astype(np.float32)
+    f_psi = np.zeros(w.max_len + 1, np.float32); f_psi[0] = 1.0
+    feat = api.sample(ctx, api.DeviceGraph(g), configs.WALK_SEED, w.n_walks, w.p_halt, w.max_len, f_phi, f_psi)
+    Phi, Psi, PsiT, _, _ = helpers.oracle_features(w, g, configs.WALK_SEED, f_phi, f_psi)
+    assert Psi.nnz == g.N
+    rng = np.random.default_rng(6)
+    rows = np.unique(np.concatenate([[0, 7, 8, g.N - 1], rng.integers(0, g.N, 60)]))
+    Mrows = np.zeros((len(rows), g.N))
+    for r, i in enumerate(rows):
+        s, e = Phi.rowptr[i], Phi.rowptr[i + 1]
+        Mrows[r, Phi.col[s:e]] = Phi.val[s:e]
+    q, k, v = tensors.qkv(w.G, g.N, w.m, w.d, w.dtype, configs.QKV_SEED)
+    for softmax in (False, True):
+        qq, kk = (q, k) if not softmax else ((q.float() * 0.25).to(q.dtype), (k.float() * 0.25).to(k.dtype))
+        ref = oracle.attn_bruteforce(tensors.widen(qq), tensors.widen(kk), tensors.widen(v), Mrows_full(Mrows, rows, g.N),
+                                     rows=rows, kernel="exp" if softmax else "linear")
+        out = api.masked_attn_asym(ctx, feat, qq.cuda(), kk.cuda(), v.cuda(), softmax=softmax)
+        B.grf_ctx_check(ctx.handle)
+        helpers.assert_attn_close(out[:, rows].float().cpu().numpy(), ref, helpers.TOL["bf16"], None,
+                                  f"full size asymmetric softmax={softmax}")
+        assert torch.isfinite(out.float()).all()
+    feat.free()
+    ctx.close()
+
+
 def Mrows_full(Mrows, rows, N):
     """attn_bruteforce indexes the mask by absolute row: place the sampled rows into an N x N frame lazily."""
     class _Rows:
