@@ -167,7 +167,7 @@ constexpr int TC_THREADS = 192;
 
 template <int M, int D>
 __global__ void __launch_bounds__(TC_THREADS)
-gather_contract_tc_kernel(int32_t N, int32_t R, const int32_t* __restrict__ plan_off,
+gather_contract_tc_kernel(int32_t G, int32_t nblocks, int32_t N, int32_t R, const int32_t* __restrict__ plan_off,
                           const int32_t* __restrict__ plan_cnt, const int32_t* __restrict__ plan_col,
                           const uint2* __restrict__ plan_coef,
                           const __nv_bfloat16* __restrict__ phiQ, const unsigned char* __restrict__ records,
@@ -182,7 +182,23 @@ gather_contract_tc_kernel(int32_t N, int32_t R, const int32_t* __restrict__ plan
     __shared__ int abort_flag;
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int32_t blk = blockIdx.x, g = blockIdx.y;
+    // Launch order.  The blocks' union sizes differ by up to a factor of three and the CTAs that start last
+    // decide when the kernel ends, so the last quarter of the problems is taken block by block in order of
+    // decreasing union size (all of these problems for a block together); the first three quarters keep the
+    // order of the rows, in which neighbouring blocks run together and share their tiles in L2.
+    int32_t blk, g;
+    {
+        const int32_t tail_g = G / 4, head_g = G - tail_g;
+        const uint32_t idx = blockIdx.x;
+        if (idx < (uint32_t)head_g * (uint32_t)nblocks) {
+            g = (int32_t)(idx / (uint32_t)nblocks);
+            blk = (int32_t)(idx % (uint32_t)nblocks);
+        } else {
+            const uint32_t j = idx - (uint32_t)head_g * (uint32_t)nblocks;
+            g = head_g + (int32_t)(j % (uint32_t)tail_g);
+            blk = plan_cnt[nblocks + (int32_t)(j / (uint32_t)tail_g)];
+        }
+    }
     const uint32_t b_base = (smem_u32(smem_dyn) + 1023u) & ~1023u;
     const unsigned char* b_generic = smem_dyn + (b_base - smem_u32(smem_dyn));
     const uint32_t bar_base = smem_u32(bars);
@@ -585,6 +601,20 @@ block_coef_kernel(int32_t N, int32_t R, const int32_t* __restrict__ rowptr, cons
         }
 }
 
+// order[r] = the block with the r-th largest union (ties: lower index first), stored behind the counts
+__global__ void __launch_bounds__(256) block_order_kernel(int32_t nblocks, int32_t* __restrict__ plan_cnt)
+{
+    const int32_t i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= nblocks) return;
+    const int32_t c = plan_cnt[i];
+    int32_t rank = 0;
+    for (int32_t j = 0; j < nblocks; ++j) {
+        const int32_t cj = plan_cnt[j];
+        rank += (cj > c || (cj == c && j < i)) ? 1 : 0;
+    }
+    plan_cnt[nblocks + rank] = i;
+}
+
 }  // namespace
 
 int grf_build_block_plan(grf_ctx* ctx, grf_features* feat)
@@ -596,7 +626,7 @@ int grf_build_block_plan(grf_ctx* ctx, grf_features* feat)
     if (words * 8 > 200 * 1024 || phi.nnz <= 0) return GRF_OK;   // no plan: the ALU kernel serves this object
     const int32_t nblocks = grf_ceil_div(N, BQ);
     GRF_TRY(grf_buf_reserve(&feat->plan_off, sizeof(int32_t) * (size_t)nblocks));
-    GRF_TRY(grf_buf_reserve(&feat->plan_cnt, sizeof(int32_t) * (size_t)nblocks));
+    GRF_TRY(grf_buf_reserve(&feat->plan_cnt, sizeof(int32_t) * 2 * (size_t)nblocks));   // counts, then blocks by decreasing count
     GRF_TRY(grf_buf_reserve(&feat->plan_col, phi.col.bytes + sizeof(int32_t) * 3 * (size_t)nblocks));
     GRF_TRY(grf_buf_reserve(&feat->plan_total, sizeof(int32_t)));
     GRF_CUDA_TRY(cudaMemsetAsync(feat->plan_total.ptr, 0, sizeof(int32_t), ctx->stream));
@@ -606,6 +636,10 @@ int grf_build_block_plan(grf_ctx* ctx, grf_features* feat)
         block_plan_kernel<<<nblocks, 256, words * 4, ctx->stream>>>(
             N, R, (const int32_t*)phi.rowptr.ptr, (const int32_t*)phi.col.ptr, (int32_t*)feat->plan_off.ptr,
             (int32_t*)feat->plan_cnt.ptr, (int32_t*)feat->plan_col.ptr, (int32_t*)feat->plan_total.ptr);
+    }
+    {
+        grf_launch_scope scope(ctx, 7);
+        block_order_kernel<<<grf_ceil_div(nblocks, 256), 256, 0, ctx->stream>>>(nblocks, (int32_t*)feat->plan_cnt.ptr);
     }
     GRF_CUDA_TRY(cudaGetLastError());
     // the table's size is known only now
@@ -649,11 +683,11 @@ static int launch_tc(grf_ctx* ctx, const grf_features* feat, int32_t G, int32_t 
             G, N, phi.cols, (const int32_t*)phi.rowptr.ptr, (const int32_t*)phi.col.ptr, (const float*)phi.val.ptr,
             (const __nv_bfloat16*)phiQ, (const unsigned char*)records, den);
     }
-    const dim3 grid(feat->plan_blocks, G);
+    const dim3 grid((unsigned)feat->plan_blocks * (unsigned)G);
     {
         grf_launch_scope scope(ctx, 5);
         gather_contract_tc_kernel<M, D><<<grid, TC_THREADS, Sh::SMEM, ctx->stream>>>(
-            N, phi.cols, (const int32_t*)feat->plan_off.ptr, (const int32_t*)feat->plan_cnt.ptr,
+            G, feat->plan_blocks, N, phi.cols, (const int32_t*)feat->plan_off.ptr, (const int32_t*)feat->plan_cnt.ptr,
             (const int32_t*)feat->plan_col.ptr, (const uint2*)feat->plan_coef.ptr, (const __nv_bfloat16*)phiQ,
             (const unsigned char*)records, (__nv_bfloat16*)out, den, ctx->error_word);
     }
