@@ -34,10 +34,10 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0}
 # heads, so the figures are scaled by 4).  Set an entry to None when its kernel changes after the capture.
 NCU_TRAFFIC_BYTES = {
     "pointcloud-gmm16-N32768": {
-        "gather_contract": 4 * (1.140300e9 + 10.290944e6),
-        "build_states": 4 * (0.063216e9 + 226.042880e6),
-        "row_denominators": 4 * (0.037776e9 + 0.012032e6),
-        "walk_merge": 0.005128e9 + 7.008000e6,
+        "gather_contract": 4 * (1.133120e9 + 12.062208e6),
+        "build_states": 4 * (0.062991e9 + 226.052096e6),
+        "row_denominators": 4 * (0.037775e9 + 0.042496e6),
+        "walk_merge": 0.005105e9 + 6.034688e6,
     }
 }
 
