@@ -411,8 +411,8 @@ int launch_state_tc(grf_ctx* ctx, const grf_csr_dev& psit, int32_t G, int32_t N,
 // rows of a 2-D tensor per instruction, row indices given in registers), so the gather does not pass through
 // the load/store units.  A gathered v_j row is 128 bytes: 64 rows stacked at a 128-byte pitch, written with
 // the 128-byte swizzle, ARE the MN-major swizzled operand (8 keys x 128 bytes per swizzle atom).  The second
-// atom along M (rows 64..127: the ones row that yields z_l, then zeros) is one constant region shared by all
-// stages, reached through the descriptor's leading-dimension offset.  The copy engine sustains about one
+// atom along M (rows 64..127: the ones row that yields z_l, then zeros) is one constant 2 KB region shared by
+// all stages and K steps, reached through the descriptor's leading-dimension offset.  The copy engine sustains about one
 // four-row gather per 15 cycles per SM whatever the rows' length, so the shorter phi(k_j) rows do not go
 // through it as well: they travel as asynchronous 16-byte copies through the load/store units (which would
 // otherwise idle) into the padded unswizzled layout of the kernel above, and are scaled in place by Psi_jl.
@@ -427,7 +427,8 @@ template <int M> struct TmaShape {
     static constexpr int NS = 4;                                // one stage per producer warp
     static constexpr int ACC_COLS = M < 32 ? 32 : M;
     static constexpr int TMEM_COLS = 2 * ACC_COLS < 32 ? 32 : 2 * ACC_COLS;
-    static constexpr size_t SMEM = (size_t)NS * STAGE + A_BYTES + 1024;
+    static constexpr int CONST_BYTES = 2048;                    // the constant second atom of A: one K step (16 keys)
+    static constexpr size_t SMEM = (size_t)NS * STAGE + CONST_BYTES + 1024;
     static_assert(STAGE % 1024 == 0, "stages must keep the swizzle phase");
 };
 
@@ -492,10 +493,10 @@ build_states_tma_kernel(int32_t R, int32_t N, const int32_t* __restrict__ t_rowp
     if (tid <= NODES_PER_CTA) node_beg[tid] = t_rowptr[min(l0 + tid, R)];
     // stages start as zeros (pad rows are multiplied before they are ever written); the constant atom is zero
     // except for bf16 1.0 in element 0 of logical piece 0 of every key row, which the swizzle puts at piece r % 8
-    for (int x = tid; x < (NS * Sh::STAGE + Sh::A_BYTES) / 16; x += ST_THREADS)
+    for (int x = tid; x < (NS * Sh::STAGE + Sh::CONST_BYTES) / 16; x += ST_THREADS)
         *reinterpret_cast<uint4*>(stage_generic + (size_t)x * 16) = make_uint4(0u, 0u, 0u, 0u);
     __syncthreads();
-    for (int r = tid; r < ITEM_KEYS; r += ST_THREADS)
+    for (int r = tid; r < 16; r += ST_THREADS)
         *reinterpret_cast<unsigned short*>(stage_generic + (size_t)NS * Sh::STAGE + (size_t)r * 128 + (size_t)(r % 8) * 16) = 0x3F80u;
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
@@ -627,7 +628,8 @@ build_states_tma_kernel(int32_t R, int32_t N, const int32_t* __restrict__ t_rowp
                 const uint32_t b_op = a_op + Sh::A_BYTES;
                 for (int32_t ks = 0; ks < ksteps; ++ks) {
                     // A: two atoms along M (gathered rows, then the constant atom), 8-key groups 1024 bytes apart
-                    const uint64_t ad = swizzled_desc(a_op + (uint32_t)ks * 2048u, const_base - a_op, 1024u, 2);
+                    // (every K step points its second atom at the same constant 2 KB)
+                    const uint64_t ad = swizzled_desc(a_op + (uint32_t)ks * 2048u, const_base - (a_op + (uint32_t)ks * 2048u), 1024u, 2);
                     const uint64_t bd = operand_desc(b_op + (uint32_t)ks * Sh::B_KSTEP, Sh::B_LBO, Sh::B_SBO);
                     mma_bf16_ss(acc, ad, bd, idesc, (it > 0 || ks > 0) ? 1u : 0u);
                 }
