@@ -13,7 +13,8 @@ Two layers:
 Pins (tests/test_oracle_*.py): Philox known answers; closed-form f for alpha_k = 2^-k;
 (I - W/2)^-1; deterministic walks on a perfect matching; expected deposits per walk;
 the L1 bound of Thm 3.2's proof; unbiasedness of Phi Psi^T; Lemma 3.3; brute force vs
-S/z route; identity and all-ones features reducing to plain V / unmasked linear attention.
+S/z route; identity and all-ones features reducing to plain V / unmasked linear attention; the exp similarity
+with an all-ones mask against scipy's softmax; Alg. 2's loop over walks against the dense definition with Mhat = Phi.
 The order of equal columns inside a transposed row and the (walk, t) summation order are
 fixed by this oracle's specification, not by the paper: parity unpinned by the paper for
 those two orderings (they change no value beyond fp32 rounding order).
