@@ -281,6 +281,8 @@ extern "C" int grf_masked_linear_attn(grf_ctx* ctx, const grf_features* feat, in
     if (chunk > G) chunk = G;
     if (chunk > 65535) chunk = 65535;
     const size_t es = elem_size(dtype);
+    // the plan's build waits for the stream once: do it before the attention kernels are queued, not between them
+    if (dtype == GRF_DTYPE_BF16 && ctx->use_tensor_cores) GRF_TRY(grf_ensure_block_plan(ctx, feat));
     for (int64_t g0 = 0; g0 < G; g0 += chunk) {
         const int32_t gc = (int32_t)((G - g0) < chunk ? (G - g0) : chunk);
         // chunk layout: records [gc][R], contiguous

@@ -694,17 +694,22 @@ static int launch_tc(grf_ctx* ctx, const grf_features* feat, int32_t G, int32_t 
     return cudaGetLastError() == cudaSuccess ? GRF_OK : GRF_ERR_CUDA;
 }
 
+// The plan is a cache inside the feature object, built on first use (the asymmetric route never needs it).
+int grf_ensure_block_plan(grf_ctx* ctx, const grf_features* feat)
+{
+    if (!feat->plan_stale) return GRF_OK;
+    grf_features* f = const_cast<grf_features*>(feat);
+    GRF_TRY(grf_build_block_plan(ctx, f));
+    f->plan_stale = false;
+    return GRF_OK;
+}
+
 // Returns GRF_OK after launching, or 1 when this shape/object has no tensor-core path (caller falls back).
 int grf_gather_contract_tc(grf_ctx* ctx, const grf_features* feat, int32_t G, int32_t N, int32_t m, int32_t d,
                            const void* phiQ, const void* records, void* out, float* den_out)
 {
     if (G > 65535) return 1;
-    if (feat->plan_stale) {
-        // the plan is a cache inside the feature object, built on first use (the asymmetric route never needs it)
-        grf_features* f = const_cast<grf_features*>(feat);
-        GRF_TRY(grf_build_block_plan(ctx, f));
-        f->plan_stale = false;
-    }
+    GRF_TRY(grf_ensure_block_plan(ctx, feat));
     if (!feat->plan_ready) return 1;
 #define GRF_TC_CASE(MM, DD) \
     if (m == MM && d == DD) return launch_tc<MM, DD>(ctx, feat, G, N, phiQ, records, out, den_out);

@@ -124,6 +124,7 @@ int grf_gather_contract_alu(grf_ctx* ctx, const grf_csr_dev& phi, int32_t G, int
                             int dtype, const void* phiQ, const void* records, void* out, float* den_out);
 // attn_gather_tc.cu
 int grf_build_block_plan(grf_ctx* ctx, grf_features* feat);
+int grf_ensure_block_plan(grf_ctx* ctx, const grf_features* feat);   // builds it if Phi changed since the last build
 int grf_gather_contract_tc(grf_ctx* ctx, const grf_features* feat, int32_t G, int32_t N, int32_t m, int32_t d,
                            const void* phiQ, const void* records, void* out, float* den_out);
 
