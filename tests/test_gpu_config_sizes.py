@@ -1,0 +1,154 @@
+"""GPU parity at the stated sizes of the workloads (the smaller cuts live in test_gpu_parity.py):
+
+  * point cloud N = 4096 with all 8 heads against the full O(N^2) brute force of Eqs. 1-2;
+  * ViT grid with all 64 x 12 = 768 problems in one call (the launch geometry of the full batch), the oracle on
+    the first, a middle and the last problem;
+  * 8-regular graphs of the scaling sweep at N = 2^14, 2^17 and 2^18 on sampled query rows, each row's mask
+    computed by the oracle as sum_l Phi_il Psi^T_l (records far larger than L2; at 2^18 the object is served by
+    the kernels that run when neighbouring rows share too few nodes for a block plan).
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from tests import helpers
+from tests.test_gpu_fullsize import Mrows_full
+from workloads import configs, tensors
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def lib():
+    from paper_2410_03462_b200 import api, binding
+    ctx = api.Context(0)
+    yield api, binding, ctx
+    ctx.close()
+
+
+def _both_gather_kernels(lib, feat, q, k, v, check):
+    api, B, ctx = lib
+    qd, kd, vd = q.cuda(), k.cuda(), v.cuda()
+    for tensor_cores in (True, False):
+        B.grf_ctx_use_tensor_cores(ctx.handle, tensor_cores)
+        out, den = api.masked_linear_attn(ctx, feat, qd, kd, vd, want_den=True)
+        B.grf_ctx_check(ctx.handle)
+        check(out, den, f"tensor_cores={tensor_cores}")
+    B.grf_ctx_use_tensor_cores(ctx.handle, True)
+
+
+def test_point_cloud_4096_all_heads_against_full_bruteforce(lib):
+    api, B, ctx = lib
+    w = configs.point_cloud_4096()
+    g = w.graph()
+    assert g.N == 4096 and w.G == 8
+    f = oracle.deconvolve(w.alpha).astype(np.float32)
+    feat = api.sample(ctx, api.DeviceGraph(g), configs.WALK_SEED, w.n_walks, w.p_halt, w.max_len, f)
+    Phi, Psi, PsiT, _, _ = helpers.oracle_features(w, g, configs.WALK_SEED, f)
+    helpers.assert_csr_equal(feat.to_host(0), Phi, "Phi", val_rtol=0)
+    helpers.assert_csr_equal(feat.to_host(2), PsiT, "Psi^T", val_rtol=0)
+    q, k, v = tensors.qkv(w.G, g.N, w.m, w.d, w.dtype, configs.QKV_SEED)
+    Mhat = Phi.dense() @ Psi.dense().T                       # Eq. 2's mask, dense, fp64
+    ref = oracle.attn_bruteforce(tensors.widen(q), tensors.widen(k), tensors.widen(v), Mhat)
+
+    def check(out, den, what):
+        helpers.assert_attn_close(out.float().cpu().numpy(), ref, helpers.TOL["bf16"], den.cpu().numpy(),
+                                  f"{w.name} {what}", same_sign=True)
+
+    _both_gather_kernels(lib, feat, q, k, v, check)
+    feat.free()
+
+
+def test_vit_grid_full_batch_of_768_problems(lib):
+    api, B, ctx = lib
+    w = configs.vit_grid()
+    g = w.graph()
+    assert w.G == 768 and g.N == 196
+    f = oracle.deconvolve(w.alpha).astype(np.float32)
+    feat = api.sample(ctx, api.DeviceGraph(g), configs.WALK_SEED, w.n_walks, w.p_halt, w.max_len, f)
+    Phi, Psi, PsiT, _, _ = helpers.oracle_features(w, g, configs.WALK_SEED, f)
+    helpers.assert_csr_equal(feat.to_host(0), Phi, "Phi", val_rtol=0)
+    q, k, v = tensors.qkv(w.G, g.N, w.m, w.d, w.dtype, configs.QKV_SEED)
+    probs = [0, 383, 767]
+    ref = oracle.attn_sparse(tensors.widen(q[probs]), tensors.widen(k[probs]), tensors.widen(v[probs]), Phi, PsiT)
+    # the S/z route of the oracle against the dense definition on one of them (the alpha of this workload give
+    # mixed-sign f, so the mask has entries of both signs)
+    bf = oracle.attn_bruteforce(tensors.widen(q[767:]), tensors.widen(k[767:]), tensors.widen(v[767:]),
+                                Phi.dense() @ Psi.dense().T)
+    assert np.allclose(bf["num"][0], ref["num"][2], rtol=1e-9, atol=1e-9)
+    assert np.allclose(bf["den"][0], ref["den"][2], rtol=1e-9, atol=1e-9)
+
+    def check(out, den, what):
+        excluded = helpers.assert_attn_close(out[probs].float().cpu().numpy(), ref, helpers.TOL["bf16"],
+                                             den[probs].cpu().numpy(), f"{w.name} G=768 {what}")
+        assert excluded < 0.05
+        assert torch.isfinite(out.float()).all()
+
+    _both_gather_kernels(lib, feat, q, k, v, check)
+    # all problems see the same features: two problems given identical inputs must give identical outputs
+    q2, k2, v2 = q.clone(), k.clone(), v.clone()
+    q2[500], k2[500], v2[500] = q[3], k[3], v[3]
+    out = api.masked_linear_attn(ctx, feat, q2.cuda(), k2.cuda(), v2.cuda())
+    assert torch.equal(out[500], out[3])
+    feat.free()
+
+
+@pytest.mark.parametrize("log2N", [14, 17, 18])
+def test_regular_graph_sweep_points_on_sampled_rows(lib, log2N):
+    api, B, ctx = lib
+    w = configs.sweep(log2N)
+    g = w.graph()
+    f = oracle.deconvolve(w.alpha).astype(np.float32)
+    feat = api.sample(ctx, api.DeviceGraph(g), configs.WALK_SEED, w.n_walks, w.p_halt, w.max_len, f)
+    Phi, Psi, PsiT, _, _ = helpers.oracle_features(w, g, configs.WALK_SEED, f)
+    for which, want in ((0, Phi), (1, Psi), (2, PsiT)):
+        rp, c, val = feat.to_host(which)
+        assert np.array_equal(rp, want.rowptr) and np.array_equal(c, want.col)
+        assert np.array_equal(val.view(np.uint32), want.val.view(np.uint32))
+    q, k, v = tensors.qkv(w.G, g.N, w.m, w.d, w.dtype, configs.QKV_SEED)
+    rng = np.random.default_rng(log2N)
+    rows = np.unique(np.concatenate([[0, 127, 128, g.N - 129, g.N - 1], rng.integers(0, g.N, 72)]))
+    assert len(rows) >= 64
+    Mrows = oracle.mask_rows(Phi, Psi, rows)
+    ref = oracle.attn_bruteforce(tensors.widen(q), tensors.widen(k), tensors.widen(v), Mrows_full(Mrows, rows, g.N),
+                                 rows=rows)
+
+    def check(out, den, what):
+        helpers.assert_attn_close(out[:, rows].float().cpu().numpy(), ref, helpers.TOL["bf16"],
+                                  den[:, rows].cpu().numpy(), f"{w.name} {what}", same_sign=True)
+        assert torch.isfinite(out.float()).all() and (den > 0).all()
+
+    _both_gather_kernels(lib, feat, q, k, v, check)
+    feat.free()
+
+
+def test_wide_feature_space_few_nonzeros(lib):
+    """R = 900 000 feature columns with a few thousand non-zeros: a column bitmap of this width does not fit a
+    CTA's shared memory, so the object has no block plan and the plain gather kernel serves both settings."""
+    api, B, ctx = lib
+    rng = np.random.default_rng(99)
+    N, R, G, m, d = 300, 900_000, 1, 16, 16
+
+    def rand_csr(per_row):
+        rowptr = [0]; col = []; val = []
+        for r in range(N):
+            c = np.sort(rng.choice(R // 1000, size=rng.integers(0, per_row + 1), replace=False)) * 1000 + rng.integers(0, 2)
+            col += list(c); val += list(rng.uniform(0.1, 1.0, len(c))); rowptr.append(len(col))
+        return oracle.CSR(np.array(rowptr, np.int32), np.array(col, np.int32), np.array(val, np.float32), None, (N, R))
+
+    Phi, Psi = rand_csr(40), rand_csr(40)
+    feat = api.features_from_csr(ctx, N, R, (Phi.rowptr, Phi.col, Phi.val), (Psi.rowptr, Psi.col, Psi.val))
+    helpers.assert_csr_equal(feat.to_host(2), oracle.transpose(Psi), "Psi^T", val_rtol=0)
+    q, k, v = tensors.qkv(G, N, m, d, "bf16", 8)
+    rows = np.arange(N)
+    Mrows = oracle.mask_rows(Phi, Psi, rows)
+    assert (Mrows != 0).sum() > N           # the two matrices do share columns
+    ref = oracle.attn_bruteforce(tensors.widen(q), tensors.widen(k), tensors.widen(v), Mrows)
+
+    def check(out, den, what):
+        helpers.assert_attn_close(out.float().cpu().numpy(), ref, helpers.TOL["bf16"], den.cpu().numpy(),
+                                  f"wide R {what}", same_sign=True)
+
+    _both_gather_kernels(lib, feat, q, k, v, check)
+    feat.free()

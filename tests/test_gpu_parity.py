@@ -64,7 +64,7 @@ def test_features_structure_bit_exact_values_close(lib, name):
     feat.free()
 
 
-def _attn_case(lib, w, g, G, f_phi=None, f_psi=None, ws_bytes=None):
+def _attn_case(lib, w, g, G, f_phi=None, f_psi=None, ws_bytes=None, same_sign=False):
     api, B, ctx = lib
     if f_phi is None:
         f_phi = oracle.deconvolve(w.alpha).astype(np.float32)
@@ -79,7 +79,7 @@ def _attn_case(lib, w, g, G, f_phi=None, f_psi=None, ws_bytes=None):
                                           workspace_bytes=ws_bytes)
         B.grf_ctx_check(ctx.handle)
         helpers.assert_attn_close(out.float().cpu().numpy(), ref, helpers.TOL[w.dtype], den.cpu().numpy(),
-                                  f"{w.name} tensor_cores={tensor_cores}")
+                                  f"{w.name} tensor_cores={tensor_cores}", same_sign=same_sign)
         outs.append(out)
     B.grf_ctx_use_tensor_cores(ctx.handle, True)
     feat.free()
@@ -88,7 +88,7 @@ def _attn_case(lib, w, g, G, f_phi=None, f_psi=None, ws_bytes=None):
 
 def test_attention_tiny_fp32(lib):
     w = configs.tiny()
-    _attn_case(lib, w, w.graph(), 1)
+    _attn_case(lib, w, w.graph(), 1, same_sign=True)
 
 
 def test_attention_vit_bf16(lib):
@@ -98,12 +98,12 @@ def test_attention_vit_bf16(lib):
 
 def test_attention_point_cloud_bf16(lib):
     w = configs.point_cloud_4096(2048)
-    _attn_case(lib, w, w.graph(), 2)
+    _attn_case(lib, w, w.graph(), 2, same_sign=True)
 
 
 def test_attention_regular_graph_bf16(lib):
     w = configs.sweep(11)
-    _attn_case(lib, w, w.graph(), 2)
+    _attn_case(lib, w, w.graph(), 2, same_sign=True)
 
 
 def test_attention_asymmetric_features(lib):
@@ -133,12 +133,16 @@ def test_attention_shapes_random_features(lib, m, d, dtype):
 
     def rand_csr(rows, cols, per_row):
         rowptr = [0]; col = []; val = []
-        for _ in range(rows):
-            c = np.sort(rng.choice(cols, size=rng.integers(1, per_row + 1), replace=False))
+        for r in range(rows):
+            # rows 0, 5, 130 and the last one (one in every query block, the ragged one included) and about one in
+            # ten of the others have no entry at all: Eq. 12 with an empty sum, out = 0
+            n = 0 if r in (0, 5, 130, rows - 1) else rng.integers(0, per_row + 1) * (rng.random() > 0.1)
+            c = np.sort(rng.choice(cols, size=n, replace=False))
             col += list(c); val += list(rng.standard_normal(len(c))); rowptr.append(len(col))
         return oracle.CSR(np.array(rowptr, np.int32), np.array(col, np.int32), np.array(val, np.float32), None, (rows, cols))
 
     Phi, Psi = rand_csr(N, R, 9), rand_csr(N, R, 12)
+    assert (np.diff(Phi.rowptr) == 0).sum() >= 4
     feat = api.features_from_csr(ctx, N, R, (Phi.rowptr, Phi.col, Phi.val), (Psi.rowptr, Psi.col, Psi.val))
     PsiT = oracle.transpose(Psi)
     helpers.assert_csr_equal(feat.to_host(2), PsiT, "Psi^T", val_rtol=0)
@@ -149,7 +153,7 @@ def test_attention_shapes_random_features(lib, m, d, dtype):
         out, den = api.masked_linear_attn(ctx, feat, q.cuda(), k.cuda(), v.cuda(), want_den=True)
         B.grf_ctx_check(ctx.handle)
         helpers.assert_attn_close(out.float().cpu().numpy(), ref, helpers.TOL[dtype], den.cpu().numpy(),
-                                  f"m{m} d{d} tensor_cores={tensor_cores}", min_ok=0.5)
+                                  f"m{m} d{d} tensor_cores={tensor_cores}")
     B.grf_ctx_use_tensor_cores(ctx.handle, True)
     feat.free()
 
@@ -185,7 +189,7 @@ def test_state_kernels_key_count_edges(lib, m, d):
     out, den = api.masked_linear_attn(ctx, feat, q.cuda(), k.cuda(), v.cuda(), want_den=True)
     B.grf_ctx_check(ctx.handle)
     helpers.assert_attn_close(out.float().cpu().numpy(), ref, helpers.TOL["bf16"], den.cpu().numpy(), f"key edges m{m} d{d}",
-                              min_ok=0.5)
+                              same_sign=True)
     feat.free()
 
 

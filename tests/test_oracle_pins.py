@@ -364,6 +364,61 @@ def test_sparse_route_equals_bruteforce_on_tiny_workload():
     assert np.allclose(oracle.mask_rows(Phi, Psi, rows), (Phi.dense() @ Psi.dense().T)[rows], atol=1e-15)
 
 
+def _abs_inputs_reference(q, k, v, Phi, Psi):
+    """The tolerance scale by its definition, computed densely: the sums of the absolute values of the terms of
+    num and den are what Eqs. 1-2 give for |phi(q)|, |phi(k)|, |v| under the mask |Phi| |Psi|^T (every term of the
+    S/z route is a product Phi_il q_a Psi_jl k_ja v_jb, so its absolute value factorises)."""
+    Mabs = np.abs(Phi.dense()) @ np.abs(Psi.dense()).T
+    return oracle.attn_bruteforce(np.abs(q), np.abs(k), np.abs(v), Mabs)
+
+
+def test_tolerance_scale_nonnegative_features_equals_dense_definition():
+    """num_abs / den_abs of the S/z route set the bound of every GPU comparison.  For non-negative features and
+    phi(Q), phi(K) >= 0 every A_ij >= 0, so they must equal |A| |V| and sum_j |A_ij| of the dense definition."""
+    w = configs.tiny()
+    g = w.graph()
+    f = oracle.deconvolve(w.alpha).astype(np.float32)
+    Phi, Psi, PsiT, _, _ = oracle.sample(g.rowptr, g.col, g.w, 42, w.n_walks, w.p_halt, w.max_len, f)
+    rng = np.random.default_rng(13)
+    cases = [(Phi, Psi, 64, 16, 16, 1)]
+    cases.append((_rand_csr(rng, 29, 11, 4, signed=False), _rand_csr(rng, 29, 11, 5, signed=False), 29, 5, 3, 2))
+    for P, S, N, m, d, G in cases:
+        assert (P.val >= 0).all() and (S.val >= 0).all()
+        q, k, v = _qkv(rng, G, N, m, d)
+        bf = oracle.attn_bruteforce(q, k, v, P.dense() @ S.dense().T)
+        sr = oracle.attn_sparse(q, k, v, P, oracle.transpose(S))
+        assert np.allclose(sr["num_abs"], bf["num_abs"], rtol=1e-11, atol=1e-300)
+        assert np.allclose(sr["den_abs"], bf["den_abs"], rtol=1e-11, atol=1e-300)
+        assert np.allclose(sr["den_abs"], sr["den"], rtol=1e-11, atol=1e-300)      # same-sign terms: no cancellation
+        # and the definition itself: a term counted twice or squared would show here
+        ab = _abs_inputs_reference(q, k, v, P, S)
+        assert np.allclose(sr["num_abs"], ab["num"], rtol=1e-11, atol=1e-300)
+        assert np.allclose(sr["den_abs"], ab["den"], rtol=1e-11, atol=1e-300)
+
+
+def test_tolerance_scale_signed_features():
+    """Signed rectangular features and signed phi: the scale equals the dense evaluation on absolute values
+    exactly, and is never below the dense route's own |A| |V| (terms that cancel inside Mhat_ij count separately
+    in the S/z route)."""
+    rng = np.random.default_rng(14)
+    G, N, R, m, d = 2, 31, 13, 4, 5
+    q = rng.standard_normal((G, N, m)).astype(np.float32)
+    k = rng.standard_normal((G, N, m)).astype(np.float32)
+    v = rng.standard_normal((G, N, d)).astype(np.float32)
+    Phi = _rand_csr(rng, N, R, 6, signed=True)
+    Psi = _rand_csr(rng, N, R, 5, signed=True)
+    sr = oracle.attn_sparse(q, k, v, Phi, oracle.transpose(Psi))
+    ab = _abs_inputs_reference(q, k, v, Phi, Psi)
+    # the S/z route sums |Phi_il q_a| * |Psi_jl k_ja v_jb| per feature component a; the dense evaluation on absolute
+    # values sums (|q|.|k|) |Mhat|_ij |v_jb|: the same terms, regrouped
+    assert np.allclose(sr["num_abs"], ab["num"], rtol=1e-11, atol=1e-300)
+    assert np.allclose(sr["den_abs"], ab["den"], rtol=1e-11, atol=1e-300)
+    bf = oracle.attn_bruteforce(q, k, v, Phi.dense() @ Psi.dense().T)
+    assert (sr["num_abs"] >= bf["num_abs"] * (1 - 1e-12)).all()
+    assert (sr["den_abs"] >= bf["den_abs"] * (1 - 1e-12)).all()
+    assert (sr["num_abs"] > bf["num_abs"] * (1 + 1e-6)).any()        # and cancellation does occur in this case
+
+
 def test_identity_features_return_values():
     """Phi = Psi = I: Mhat = I, so out_i = v_i wherever phi(q_i).phi(k_i) != 0."""
     rng = np.random.default_rng(4)
