@@ -134,8 +134,10 @@ def walks(rowptr, col, w, seed: int, n_walks: int, p_halt: float, max_len: int):
     return traj, load
 
 
-def features_from_walks(traj, load, e: int, f) -> CSR:
-    """Eq. 10 for ensemble e with modulation f (fp32 [L+1])."""
+def features_from_walks(traj, load, e: int, f, keep_zero: bool = False) -> CSR:
+    """Eq. 10 for ensemble e with modulation f (fp32 [L+1]).  Called again on the same walks with another f it is
+    the re-modulation of Alg. 1's learnable (f_i) without re-walking.  keep_zero=True keeps the entries of prefixes
+    whose coefficient is exactly 0 (as zeros), which makes the index structure independent of f."""
     _, N, n, Lp1 = traj.shape
     f = np.ascontiguousarray(f, dtype=np.float32)
     assert f.shape[0] == Lp1
@@ -146,7 +148,7 @@ def features_from_walks(traj, load, e: int, f) -> CSR:
     val64 = np.empty(cap, dtype=np.float64)
     nnz = _load().oracle_features(ctypes.c_int32(N), ctypes.c_int32(n), ctypes.c_int32(Lp1 - 1),
                                   ctypes.c_int32(e), _p(traj), _p(load), _p(f),
-                                  _p(rowptr), _p(col), _p(val), _p(val64))
+                                  _p(rowptr), _p(col), _p(val), _p(val64), ctypes.c_int32(int(keep_zero)))
     if nnz < 0:
         raise MemoryError
     return CSR(rowptr, col[:nnz].copy(), val[:nnz].copy(), val64[:nnz].copy(), (N, N))
@@ -162,14 +164,42 @@ def transpose(a: CSR) -> CSR:
     return CSR(t_rowptr, t_col, t_val, None, (cols, rows))
 
 
-def sample(rowptr, col, w, seed, n_walks, p_halt, max_len, f_phi, f_psi=None):
+def sample(rowptr, col, w, seed, n_walks, p_halt, max_len, f_phi, f_psi=None, keep_zero: bool = False):
     """Alg. 1 steps 1-2 for two independent ensembles: returns (Phi, Psi, Psi^T, traj, load)."""
     traj, load = walks(rowptr, col, w, seed, n_walks, p_halt, max_len)
     if f_psi is None:
         f_psi = f_phi
-    Phi = features_from_walks(traj, load, 0, f_phi)
-    Psi = features_from_walks(traj, load, 1, f_psi)
+    Phi = features_from_walks(traj, load, 0, f_phi, keep_zero)
+    Psi = features_from_walks(traj, load, 1, f_psi, keep_zero)
     return Phi, Psi, transpose(Psi), traj, load
+
+
+# ----------------------------------------------------------------------------- FLOP counts (Sec. 4, "Time complexity")
+
+def flops_masked_linear(Phi: CSR, PsiT: CSR, m: int, d: int) -> int:
+    """Floating-point operations of GRF-masked linear attention evaluated as Eq. 12, counted term by term for one
+    problem: every non-zero Psi_jl costs one product with each of the m components of phi(k_j) and then one
+    multiply-add into each of the d+1 columns of [S_l | z_l]; every non-zero Phi_il likewise against phi(q_i) and
+    [S_l | z_l]; a multiply-add counts as 2; the N*d final divisions are added."""
+    total = 0
+    for l in range(PsiT.shape[0]):
+        for _ in range(PsiT.rowptr[l], PsiT.rowptr[l + 1]):
+            total += m + 2 * m * (d + 1)
+    for i in range(Phi.shape[0]):
+        for _ in range(Phi.rowptr[i], Phi.rowptr[i + 1]):
+            total += m + 2 * m * (d + 1)
+    return total + Phi.shape[0] * d
+
+
+def flops_unmasked_linear(N: int, m: int, d: int) -> int:
+    """Eq. 3 evaluated right to left: phi(K)^T [V | 1] (2 N m (d+1)), then phi(Q) times it (2 N m (d+1)), N d divisions."""
+    return 4 * N * m * (d + 1) + N * d
+
+
+def flops_softmax(N: int, m: int, d: int) -> int:
+    """Unmasked softmax attention with query/key width m: scores 2 N^2 m, exponentials N^2, row sums N^2,
+    weighted values 2 N^2 d, N d divisions."""
+    return N * N * (2 * m + 2 + 2 * d) + N * d
 
 
 # ----------------------------------------------------------------------------- attention
@@ -235,6 +265,37 @@ def mask_rows(Phi: CSR, Psi: CSR, rows) -> np.ndarray:
             s, e = PsiT.rowptr[l], PsiT.rowptr[l + 1]
             np.add.at(out[r], PsiT.col[s:e], float(Phi.val[p]) * PsiT.val[s:e].astype(np.float64))
     return out
+
+
+def materialise(Phi: CSR, Psi: CSR) -> CSR:
+    """The mask estimate itself, Mhat = Phi Psi^T (Sec. 3.3: Mhat_ij = phi_hat(v_i)^T phi_hat(v_j)), as a sparse
+    matrix: row i is sum_l Phi_il * (row l of Psi^T), accumulated in fp64 with l ascending; an entry exists iff
+    some l has Phi_il and Psi_jl both stored (even if the products cancel).  `val` holds the fp32 rounding."""
+    PsiT = transpose(Psi)
+    N, Nk = Phi.shape[0], Psi.shape[0]
+    rowptr = np.zeros(N + 1, dtype=np.int64)
+    cols, vals = [], []
+    acc = np.zeros(Nk)
+    hit = np.zeros(Nk, dtype=bool)
+    for i in range(N):
+        touched = []
+        for p in range(Phi.rowptr[i], Phi.rowptr[i + 1]):
+            l = Phi.col[p]
+            s, e = PsiT.rowptr[l], PsiT.rowptr[l + 1]
+            js = PsiT.col[s:e]
+            acc[js] += float(Phi.val[p]) * PsiT.val[s:e].astype(np.float64)   # the j of one row l are distinct
+            hit[js] = True
+            touched.append(js)
+        if touched:
+            js = np.unique(np.concatenate(touched))
+            cols.append(js.astype(np.int32)); vals.append(acc[js].copy())
+            acc[js] = 0.0; hit[js] = False
+            rowptr[i + 1] = rowptr[i] + len(js)
+        else:
+            rowptr[i + 1] = rowptr[i]
+    col = np.concatenate(cols) if cols else np.zeros(0, np.int32)
+    val64 = np.concatenate(vals) if vals else np.zeros(0)
+    return CSR(rowptr.astype(np.int32), col, val64.astype(np.float32), val64, (N, Nk))
 
 
 def attn_asym_walks(Q, K, V, traj, load, f, kernel: str = "linear"):

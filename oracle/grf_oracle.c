@@ -11,7 +11,9 @@
  *                          traversed edge weights (Eq. 9) over its probability
  *                          p(omega) = prod_hops (1 - p_halt)/deg (simple random walk with
  *                          geometric length, Thm 3.2's setting), modulated by f_len.
- *   oracle_features        Eq. 10: phi_hat(v_i)_q = (1/n) sum_walks sum_prefixes ending at q.
+ *   oracle_features        Eq. 10: phi_hat(v_i)_q = (1/n) sum_walks sum_prefixes ending at q.  Because it works from
+ *                          stored walks, calling it again with other coefficients f IS re-modulation without
+ *                          re-walking (the "learnable mask parameters (f_i)" of Alg. 1 change, the walks do not).
  *   oracle_transpose       regrouping of a CSR matrix by column (no arithmetic).
  *   oracle_attn_sparse     Eq. 12 / Alg. 1 step 5 evaluated through the per-node states
  *                          S_l = sum_j Psi_jl phi(k_j) v_j^T, z_l = sum_j Psi_jl phi(k_j).
@@ -129,10 +131,14 @@ static int cmp_deposit(const void* a, const void* b)
  * rowptr_out [N+1]; col_out/val_out/val64_out sized for N*n*(L+1) entries.  Returns nnz.
  * val   = fp32 sum, in ascending (walk, t) order, of (f_t * load) * (1/n), each product in fp32
  * val64 = the same sum carried in fp64 (terms widened from the fp32 loads)
+ * keep_zero != 0: prefixes whose coefficient f_t is exactly 0 are deposited as well (their terms are zeros),
+ * so that the index structure is the set of visited nodes whatever f is: the structure a feature object
+ * must have if its coefficients are to be changed later without new walks.
  */
 int64_t oracle_features(int32_t N, int32_t n, int32_t L, int32_t e,
                         const int32_t* traj, const float* load, const float* f,
-                        int32_t* rowptr_out, int32_t* col_out, float* val_out, double* val64_out)
+                        int32_t* rowptr_out, int32_t* col_out, float* val_out, double* val64_out,
+                        int32_t keep_zero)
 {
     const int64_t stride = (int64_t)L + 1;
     const float inv_n = 1.0f / (float)n;
@@ -146,7 +152,7 @@ int64_t oracle_features(int32_t N, int32_t n, int32_t L, int32_t e,
             const int32_t* tr = traj + (((int64_t)e * N + i) * n + k) * stride;
             const float* ld = load + (((int64_t)e * N + i) * n + k) * stride;
             for (int32_t t = 0; t <= L && tr[t] >= 0; ++t) {
-                if (f[t] == 0.0f) continue;
+                if (f[t] == 0.0f && !keep_zero) continue;
                 float dep = f[t] * ld[t];
                 dep = dep * inv_n;
                 buf[cnt].col = tr[t];

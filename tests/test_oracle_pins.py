@@ -503,3 +503,102 @@ def test_asymmetric_route_three_ways():
     dense_e = oracle.attn_bruteforce(Q * 0.3, K * 0.3, V, Phi.dense(), kernel="exp")["out"]
     walks_e = oracle.attn_asym_walks(Q * 0.3, K * 0.3, V, traj, load, f_phi, kernel="exp")
     assert np.allclose(dense_e, walks_e, rtol=1e-5, atol=1e-7)
+
+
+# ------------------------------------------------------------------ re-modulation, FLOP counts, the mask itself
+
+def test_keep_zero_structure_is_the_visited_set_and_values_agree_on_the_plain_support():
+    """With keep_zero the index structure must not depend on f (it is the set of visited nodes), the values on the
+    support of the plain assembly must be bit-identical to it, and the extra entries are exact zeros."""
+    w = configs.tiny(); g = w.graph()
+    traj, load = oracle.walks(g.rowptr, g.col, g.w, 5, w.n_walks, w.p_halt, w.max_len)
+    f = oracle.deconvolve(w.alpha).astype(np.float32)
+    f[2] = 0.0; f[5] = 0.0
+    plain = oracle.features_from_walks(traj, load, 0, f)
+    kept = oracle.features_from_walks(traj, load, 0, f, keep_zero=True)
+    ones = oracle.features_from_walks(traj, load, 0, np.ones_like(f), keep_zero=True)
+    assert np.array_equal(kept.rowptr, ones.rowptr) and np.array_equal(kept.col, ones.col)
+    # the visited set, straight from the trajectories
+    for i in range(g.N):
+        visited = np.unique(traj[0, i][traj[0, i] >= 0])
+        assert np.array_equal(kept.col[kept.rowptr[i]:kept.rowptr[i + 1]], visited)
+    assert kept.nnz > plain.nnz
+    D = {(i, int(c)): v for i in range(g.N) for c, v in zip(kept.col[kept.rowptr[i]:kept.rowptr[i + 1]],
+                                                             kept.val[kept.rowptr[i]:kept.rowptr[i + 1]])}
+    on_plain = set()
+    for i in range(g.N):
+        for c, v in zip(plain.col[plain.rowptr[i]:plain.rowptr[i + 1]], plain.val[plain.rowptr[i]:plain.rowptr[i + 1]]):
+            assert D[(i, int(c))].tobytes() == v.tobytes() or (D[(i, int(c))] == 0 and v == 0)
+            on_plain.add((i, int(c)))
+    assert all(v == 0 for key, v in D.items() if key not in on_plain)
+    # no zero coefficient: the two assemblies are the same matrix
+    f2 = oracle.deconvolve(w.alpha).astype(np.float32)
+    a = oracle.features_from_walks(traj, load, 1, f2); b = oracle.features_from_walks(traj, load, 1, f2, keep_zero=True)
+    assert np.array_equal(a.col, b.col) and a.val.tobytes() == b.val.tobytes()
+
+
+def test_remodulation_is_linear_in_f():
+    """Eq. 10 is linear in the coefficients: features(f) = sum_t f_t * features(e_t) (fp64 shadows, same walks)."""
+    w = configs.tiny(); g = w.graph()
+    traj, load = oracle.walks(g.rowptr, g.col, g.w, 11, w.n_walks, w.p_halt, w.max_len)
+    rng = np.random.default_rng(3)
+    f = rng.standard_normal(w.max_len + 1).astype(np.float32)
+    full = oracle.features_from_walks(traj, load, 0, f, keep_zero=True)
+    acc = np.zeros(full.nnz)
+    for t in range(w.max_len + 1):
+        e_t = np.zeros(w.max_len + 1, np.float32); e_t[t] = 1.0
+        part = oracle.features_from_walks(traj, load, 0, e_t, keep_zero=True)
+        assert np.array_equal(part.col, full.col)
+        acc += float(f[t]) * part.val64
+    assert np.allclose(acc, full.val64, rtol=1e-12, atol=1e-15)
+
+
+def test_flop_counts_closed_forms_and_linear_growth():
+    """Sec. 4 "Time complexity": 1-D grids, n = 4, p_halt = 0.5, m = d = 8, mean over 10 seeds.  The term-by-term
+    count equals nnz * (m + 2m(d+1)) per matrix, stays below the bound from the expected number of deposits, grows
+    linearly in N, and the softmax count grows quadratically."""
+    m = d = 8; n = 4; p = 0.5; L = 8
+    f = oracle.deconvolve(0.5 ** np.arange(L + 1)).astype(np.float32)
+    means = {}
+    for N in (64, 128, 256):
+        g = graphs.path_graph(N, 0.5)
+        counts = []
+        for seed in range(10):
+            Phi, Psi, PsiT, _, _ = oracle.sample(g.rowptr, g.col, g.w, seed, n, p, L, f)
+            c = oracle.flops_masked_linear(Phi, PsiT, m, d)
+            assert c == (Phi.nnz + PsiT.nnz) * (m + 2 * m * (d + 1)) + N * d
+            counts.append(c)
+        means[N] = np.mean(counts)
+        deposits = n * (1 - (1 - p) ** (L + 1)) / p          # expected deposits per row bound the row's non-zeros
+        assert means[N] <= 2 * N * deposits * (m + 2 * m * (d + 1)) + N * d
+        assert means[N] > oracle.flops_unmasked_linear(N, m, d)          # "a constant multiplicative cost"
+    assert abs(means[128] / means[64] - 2) < 0.1 and abs(means[256] / means[128] - 2) < 0.1
+    assert oracle.flops_unmasked_linear(128, m, d) == 4 * 128 * m * (d + 1) + 128 * d
+    r = oracle.flops_softmax(256, m, d) / oracle.flops_softmax(128, m, d)
+    assert 3.9 < r < 4.0
+
+
+def test_materialised_mask_equals_dense_product():
+    w = configs.tiny(); g = w.graph()
+    f = oracle.deconvolve(w.alpha).astype(np.float32)
+    Phi, Psi, PsiT, _, _ = oracle.sample(g.rowptr, g.col, g.w, 9, w.n_walks, w.p_halt, w.max_len, f)
+    M = oracle.materialise(Phi, Psi)
+    dense = Phi.dense() @ Psi.dense().T
+    as64 = lambda X: sp.csr_matrix((X.val64, X.col, X.rowptr), shape=X.shape).toarray()
+    assert np.allclose(as64(M), dense, rtol=0, atol=1e-15)
+    assert np.allclose(M.dense(), dense, rtol=1e-7, atol=0)          # val is the fp32 rounding of val64
+    ref = (sp.csr_matrix((np.ones(Phi.nnz), Phi.col, Phi.rowptr), shape=Phi.shape) @
+           sp.csr_matrix((np.ones(Psi.nnz), Psi.col, Psi.rowptr), shape=Psi.shape).T).tocsr()
+    ref.sort_indices()
+    assert np.array_equal(M.rowptr, ref.indptr) and np.array_equal(M.col, ref.indices)      # structural support
+    rows = [0, 7, 63]
+    assert np.allclose(oracle.mask_rows(Phi, Psi, rows), dense[rows], rtol=0, atol=1e-15)
+    # rectangular, signed
+    rng = np.random.default_rng(2)
+    A = sp.random(20, 13, 0.3, random_state=1, data_rvs=rng.standard_normal, format="csr"); A.sort_indices()
+    Bm = sp.random(17, 13, 0.3, random_state=2, data_rvs=rng.standard_normal, format="csr"); Bm.sort_indices()
+    a = oracle.CSR(A.indptr.astype(np.int32), A.indices.astype(np.int32), A.data.astype(np.float32), None, A.shape)
+    b = oracle.CSR(Bm.indptr.astype(np.int32), Bm.indices.astype(np.int32), Bm.data.astype(np.float32), None, Bm.shape)
+    M2 = oracle.materialise(a, b)
+    assert M2.shape == (20, 17)
+    assert np.allclose(as64(M2), a.dense() @ b.dense().T, rtol=0, atol=1e-12)
