@@ -80,6 +80,37 @@ int grf_sample(grf_ctx* ctx, int32_t N, const int32_t* rowptr, const int32_t* co
                uint64_t seed, int32_t n_walks, float p_halt, int32_t max_len,
                const float* f_phi, const float* f_psi, grf_features** inout);
 
+/*
+ * Re-modulation without re-walking (Alg. 1: the modulation coefficients (f_i) are learnable, the walks are not;
+ * Sec. 4: walks "can be pre-computed and frozen").
+ *
+ * grf_ctx_keep_walks(ctx, 1): from now on grf_sample also keeps, inside the feature object, the deposits behind
+ * every entry: for each prefix of each walk that ends at the entry's node, its length t and its load (Eq. 9's
+ * weight over its probability).  In this mode a prefix deposits whatever its coefficient, so the index structure
+ * of Phi and Psi is the set of visited nodes and does not depend on f; an entry all of whose coefficients are 0
+ * holds the value 0.  Entries that plain sampling would also create get bit-identical values.  Extra device
+ * memory: 5 bytes per deposit plus 4 per entry.
+ *
+ * grf_remodulate: gives a feature object sampled in that mode new coefficients (HOST arrays of max_len + 1
+ * values, max_len as sampled; f_psi == NULL means f_phi).  Values become sum (f_t * load) * (1 / n_walks) over the
+ * entry's deposits, same operations and order as the sampler's: the result is bit-identical to sampling again
+ * with the same seed and the new coefficients, without any walk being taken.  Psi^T is regrouped.  Asynchronous.
+ * GRF_ERR_INVALID if the object holds no deposits or max_len differs.
+ */
+int grf_ctx_keep_walks(grf_ctx* ctx, int enable);
+int grf_remodulate(grf_ctx* ctx, grf_features* feat, int32_t max_len, const float* f_phi, const float* f_psi);
+
+/*
+ * Floating-point operation counts of one attention problem (Sec. 4 "Time complexity", the figure of FLOPs against
+ * the number of nodes), from the feature object's non-zero counts; HOST outputs, any may be NULL:
+ *   masked          Eq. 12: every non-zero of Psi and of Phi costs m products with phi(k_j) / phi(q_i) and m(d+1)
+ *                   multiply-adds (2 operations each) into / against [S_l | z_l]; plus N*d divisions;
+ *   unmasked_linear Eq. 3 right to left: 4 N m (d+1) + N d;
+ *   softmax         N^2 (2m + 2 + 2d) + N d  (scores, exponentials, row sums, weighted values).
+ */
+int grf_attn_flops(const grf_features* feat, int32_t m, int32_t d, int64_t* masked, int64_t* unmasked_linear,
+                   int64_t* softmax);
+
 /* The walks themselves, for checking (Sec. 3.3): traj and load are DEVICE arrays
  * [2][N][n_walks][max_len+1]; traj holds the node at step t or -1 after the walk ended, load the
  * importance weight of that prefix (0 after the end).  Same arguments and limits as grf_sample. */

@@ -31,6 +31,9 @@ _SIGNATURES = {
     "grf_ctx_destroy": (_int, [_vp]),
     "grf_deconvolve": (_int, [_vp, _i32, _vp]),
     "grf_sample": (_int, [_vp, _i32, _vp, _vp, _vp, _u64, _i32, _f32, _i32, _vp, _vp, ctypes.POINTER(_vp)]),
+    "grf_ctx_keep_walks": (_int, [_vp, _int]),
+    "grf_remodulate": (_int, [_vp, _vp, _i32, _vp, _vp]),
+    "grf_attn_flops": (_int, [_vp, _i32, _i32, ctypes.POINTER(_i64), ctypes.POINTER(_i64), ctypes.POINTER(_i64)]),
     "grf_debug_walks": (_int, [_vp, _i32, _vp, _vp, _vp, _u64, _i32, _f32, _i32, _vp, _vp]),
     "grf_features_from_csr": (_int, [_vp, _i32, _i32, _vp, _vp, _vp, _vp, _vp, _vp, ctypes.POINTER(_vp)]),
     "grf_features_view": (_int, [_vp, _int, ctypes.POINTER(_i32), ctypes.POINTER(_i32), ctypes.POINTER(_i64),
@@ -152,6 +155,25 @@ def grf_sample(ctx, N, rowptr, col, w, seed, n_walks, p_halt, max_len, f_phi, f_
     _check(lib.grf_sample(ctx, N, _dev(rowptr), _dev(col), _dev(w), seed, n_walks, p_halt, max_len,
                           p_phi, p_psi, ctypes.byref(h)), "grf_sample")
     return h.value
+
+
+def grf_ctx_keep_walks(ctx: int, enable: bool):
+    _check(lib.grf_ctx_keep_walks(ctx, int(enable)), "grf_ctx_keep_walks")
+
+
+def grf_remodulate(ctx, features, max_len, f_phi, f_psi=None):
+    p_phi, k1 = _host(f_phi, np.float32)
+    p_psi, k2 = _host(f_psi, np.float32)
+    if k1 is None or k1.shape[0] != max_len + 1 or (k2 is not None and k2.shape[0] != max_len + 1):
+        raise ValueError("modulation arrays must hold max_len + 1 coefficients")
+    _check(lib.grf_remodulate(ctx, features, max_len, p_phi, p_psi), "grf_remodulate")
+
+
+def grf_attn_flops(features, m, d):
+    """(masked, unmasked_linear, softmax) operation counts of one problem."""
+    a, b, c = _i64(), _i64(), _i64()
+    _check(lib.grf_attn_flops(features, m, d, ctypes.byref(a), ctypes.byref(b), ctypes.byref(c)), "grf_attn_flops")
+    return a.value, b.value, c.value
 
 
 def grf_debug_walks(ctx, N, rowptr, col, w, seed, n_walks, p_halt, max_len, traj, load):

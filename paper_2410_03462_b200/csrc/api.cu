@@ -60,6 +60,7 @@ extern "C" int grf_ctx_destroy(grf_ctx* ctx)
     cudaSetDevice(ctx->device);
     cudaStreamSynchronize(ctx->stream);
     grf_buf* bufs[] = {&ctx->stage_col, &ctx->stage_val, &ctx->counts, &ctx->rowptr2, &ctx->scan_blocks,
+                       &ctx->stage_dep_start, &ctx->stage_dep_t, &ctx->stage_dep_load, &ctx->dep_counts, &ctx->dep_rowptr2,
                        &ctx->t_cursor, &ctx->t_tmp_col, &ctx->t_tmp_val, &ctx->den_scratch, &ctx->h_rowptr, &ctx->h_col, &ctx->h_w,
                        &ctx->h_q, &ctx->h_k, &ctx->h_v, &ctx->h_out, &ctx->h_ws};
     for (grf_buf* b : bufs) grf_buf_release(b);
@@ -160,6 +161,18 @@ extern "C" int grf_deconvolve(const double* alpha, int32_t len, double* f_out)
     return GRF_OK;
 }
 
+extern "C" int grf_attn_flops(const grf_features* feat, int32_t m, int32_t d, int64_t* masked,
+                              int64_t* unmasked_linear, int64_t* softmax)
+{
+    if (!feat || m <= 0 || d <= 0) return GRF_ERR_INVALID;
+    const int64_t N = feat->phi.rows;
+    const int64_t per_nonzero = (int64_t)m + 2 * (int64_t)m * (d + 1);     // scale phi(.), then multiply-add into [S_l | z_l]
+    if (masked) *masked = (feat->phi.nnz + feat->psit.nnz) * per_nonzero + N * d;
+    if (unmasked_linear) *unmasked_linear = 4 * N * m * (d + 1) + N * d;
+    if (softmax) *softmax = N * N * (2 * (int64_t)m + 2 + 2 * (int64_t)d) + N * d;
+    return GRF_OK;
+}
+
 static void csr_release(grf_csr_dev* m)
 {
     grf_buf_release(&m->rowptr); grf_buf_release(&m->col); grf_buf_release(&m->val);
@@ -172,6 +185,9 @@ extern "C" int grf_features_free(grf_features* feat)
     csr_release(&feat->phi); csr_release(&feat->psi); csr_release(&feat->psit);
     grf_buf_release(&feat->plan_off); grf_buf_release(&feat->plan_cnt);
     grf_buf_release(&feat->plan_col); grf_buf_release(&feat->plan_total); grf_buf_release(&feat->plan_coef);
+    for (int e = 0; e < 2; ++e) {
+        grf_buf_release(&feat->kept.dep_ptr[e]); grf_buf_release(&feat->kept.dep_t[e]); grf_buf_release(&feat->kept.dep_load[e]);
+    }
     delete feat;
     return GRF_OK;
 }

@@ -37,6 +37,9 @@ struct grf_ctx {
     grf_buf counts;                 // per-row nonzero counts (both matrices)
     grf_buf rowptr2;                // scanned counts, [2][N+1]
     grf_buf scan_blocks;            // block totals of the two-level scan
+    // sampler scratch when the walks' deposits are kept (grf_ctx_keep_walks)
+    bool keep_walks = false;
+    grf_buf stage_dep_start, stage_dep_t, stage_dep_load, dep_counts, dep_rowptr2;
     // transpose scratch
     grf_buf t_cursor, t_tmp_col, t_tmp_val;
     grf_buf den_scratch;            // denominators of the tensor-core gather path when the caller wants none
@@ -76,9 +79,20 @@ struct grf_csr_dev {
 
 #define GRF_PLAN_BLOCK 128   // queries per block of the tensor-core gather kernel
 
+// The deposits behind every entry of Phi (index 0) and Psi (index 1), kept when the sampler was asked to: entry p
+// of the matrix owns deposits dep_ptr[p] .. dep_ptr[p+1]-1, each a (step t, load of the prefix) pair, in the
+// order in which the sampler adds them.
+struct grf_kept_walks {
+    bool valid = false;
+    int32_t n_walks = 0, max_len = 0;
+    int64_t deposits[2] = {0, 0};
+    grf_buf dep_ptr[2], dep_t[2], dep_load[2];
+};
+
 struct grf_features {
     int device = 0;
     grf_csr_dev phi, psi, psit;
+    grf_kept_walks kept;
     // block plan of Phi: per block of GRF_PLAN_BLOCK rows, the sorted distinct columns
     grf_buf plan_off, plan_cnt, plan_col, plan_total;
     grf_buf plan_coef;              // dense bf16 coefficients [quad of union entries][row of the block][4]

@@ -98,11 +98,18 @@ __device__ __forceinline__ void sort_in_registers(uint32_t* keys, int lane)
     for (int r = 0; r < E; ++r) keys[lane * E + r] = v[r];
 }
 
+// KEEP: the row's deposits themselves are kept as well (for grf_remodulate): every prefix deposits whatever its
+// coefficient, the sorted list of (step, load) pairs of the row goes to a staging area of stride P.cap, and every
+// merged entry records where its deposits begin in that list.  The values are computed by the same operations in
+// the same order as without KEEP.
+template <bool KEEP>
 __global__ void __launch_bounds__(256)
 walk_merge_kernel(const __grid_constant__ grf_walk_params P,
                   const int32_t* __restrict__ rowptr, const int32_t* __restrict__ col, const float* __restrict__ w,
                   int32_t stage_stride, int32_t* __restrict__ stage_col, float* __restrict__ stage_val,
-                  int32_t* __restrict__ counts)
+                  int32_t* __restrict__ counts,
+                  int32_t* __restrict__ stage_dep_start, unsigned char* __restrict__ stage_dep_t,
+                  float* __restrict__ stage_dep_load, int32_t* __restrict__ dep_counts)
 {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     const int lane = threadIdx.x & 31;
@@ -128,12 +135,12 @@ walk_merge_kernel(const __grid_constant__ grf_walk_params P,
         wk.words[0] = wk.words[1] = wk.words[2] = wk.words[3] = 0;
         for (int32_t t = 0;; ++t) {
             const float ft = P.f[e][t];
-            const bool dep = wk.alive && ft != 0.0f;
+            const bool dep = wk.alive && (KEEP || ft != 0.0f);
             const uint32_t dm = __ballot_sync(0xffffffffu, dep);
             if (dep) {
                 const int32_t seq = k * Lp1 + t;
                 keys[cnt + __popc(dm & lt_mask)] = ((uint32_t)wk.v << P.seq_bits) | (uint32_t)seq;
-                vals[seq] = __fmul_rn(__fmul_rn(ft, wk.load), P.inv_n);
+                vals[seq] = KEEP ? wk.load : __fmul_rn(__fmul_rn(ft, wk.load), P.inv_n);
             }
             cnt += __popc(dm);
             if (t == P.max_len) break;
@@ -174,6 +181,13 @@ walk_merge_kernel(const __grid_constant__ grf_walk_params P,
     const uint32_t seq_mask = (1u << P.seq_bits) - 1u;
     int32_t r = 0;
     const size_t out_base = (size_t)row * stage_stride;
+    const size_t dep_base = (size_t)row * P.cap;
+    // value of the deposit with sequence number seq = walk * (max_len + 1) + t
+    auto term = [&](uint32_t seq) {
+        if (!KEEP) return vals[seq];
+        const int32_t t = (int32_t)seq % Lp1;
+        return __fmul_rn(__fmul_rn(P.f[e][t], vals[seq]), P.inv_n);
+    };
     for (int32_t base = 0; base < cnt; base += 32) {
         const int32_t p = base + lane;
         const bool valid = p < cnt;
@@ -181,20 +195,77 @@ walk_merge_kernel(const __grid_constant__ grf_walk_params P,
         const uint32_t c = key >> P.seq_bits;
         const bool head = valid && (p == 0 || (keys[p - 1] >> P.seq_bits) != c);
         const uint32_t hm = __ballot_sync(0xffffffffu, head);
+        if (KEEP && valid) {
+            stage_dep_t[dep_base + p] = (unsigned char)((int32_t)(key & seq_mask) % Lp1);
+            stage_dep_load[dep_base + p] = vals[key & seq_mask];
+        }
         if (head) {
-            float s = vals[key & seq_mask];
+            float s = term(key & seq_mask);
             for (int32_t q = p + 1; q < cnt; ++q) {
                 const uint32_t kq = keys[q];
                 if ((kq >> P.seq_bits) != c) break;
-                s = __fadd_rn(s, vals[kq & seq_mask]);
+                s = __fadd_rn(s, term(kq & seq_mask));
             }
             const int32_t rank = r + __popc(hm & lt_mask);
             stage_col[out_base + rank] = (int32_t)c;
             stage_val[out_base + rank] = s;
+            if (KEEP) stage_dep_start[out_base + rank] = p;
         }
         r += __popc(hm);
     }
-    if (lane == 0) counts[row] = r;
+    if (lane == 0) {
+        counts[row] = r;
+        if (KEEP) dep_counts[row] = cnt;
+    }
+}
+
+// Kept deposits: moves every row's sorted (step, load) list from the staging area to its place and turns the
+// entries' in-row start positions into absolute offsets (dep_ptr has one more element than the matrix has entries).
+__global__ void __launch_bounds__(256)
+compact_deposits_kernel(int32_t N, int32_t stage_stride, int32_t cap,
+                        const int32_t* __restrict__ stage_dep_start, const unsigned char* __restrict__ stage_dep_t,
+                        const float* __restrict__ stage_dep_load,
+                        const int32_t* __restrict__ rowptr_phi, const int32_t* __restrict__ rowptr_psi,
+                        const int32_t* __restrict__ dep_rowptr2,
+                        int32_t* __restrict__ ptr_phi, unsigned char* __restrict__ t_phi, float* __restrict__ load_phi,
+                        int32_t* __restrict__ ptr_psi, unsigned char* __restrict__ t_psi, float* __restrict__ load_psi)
+{
+    const int lane = threadIdx.x & 31;
+    const int32_t row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    if (row >= 2 * N) return;
+    const int32_t e = row >= N ? 1 : 0;
+    const int32_t i = row - e * N;
+    const int32_t* rp = e ? rowptr_psi : rowptr_phi;
+    const int32_t* drp = dep_rowptr2 + (size_t)e * (N + 1);
+    int32_t* optr = e ? ptr_psi : ptr_phi;
+    unsigned char* ot = e ? t_psi : t_phi;
+    float* ol = e ? load_psi : load_phi;
+    const int32_t beg = rp[i], len = rp[i + 1] - beg;
+    const int32_t dbeg = drp[i], dlen = drp[i + 1] - dbeg;
+    for (int32_t x = lane; x < len; x += 32) optr[beg + x] = dbeg + stage_dep_start[(size_t)row * stage_stride + x];
+    for (int32_t x = lane; x < dlen; x += 32) {
+        ot[dbeg + x] = stage_dep_t[(size_t)row * cap + x];
+        ol[dbeg + x] = stage_dep_load[(size_t)row * cap + x];
+    }
+    if (i == N - 1 && lane == 0) optr[rp[N]] = drp[N];
+}
+
+// Re-modulation (Alg. 1 step 2 with new "learnable mask parameters (f_i)"): every entry's value is rebuilt from its
+// kept deposits as sum (f_t * load) * (1/n), the products and the sum taken in the sampler's operations and order.
+struct grf_remod_params { float f[2][GRF_MAX_WALK_LEN + 1]; float inv_n; };
+__global__ void __launch_bounds__(256)
+remodulate_kernel(const __grid_constant__ grf_remod_params P, int32_t e, int64_t nnz, const int32_t* __restrict__ dep_ptr,
+                  const unsigned char* __restrict__ dep_t, const float* __restrict__ dep_load, float* __restrict__ val)
+{
+    const int64_t p = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (p >= nnz) return;
+    const int32_t beg = dep_ptr[p], end = dep_ptr[p + 1];
+    float s = 0.0f;
+    for (int32_t q = beg; q < end; ++q) {
+        const float term = __fmul_rn(__fmul_rn(P.f[e][dep_t[q]], dep_load[q]), P.inv_n);
+        s = q == beg ? term : __fadd_rn(s, term);
+    }
+    val[p] = s;
 }
 
 // Copies each merged row from the fixed-stride staging area to its place in the CSR arrays.
@@ -297,24 +368,48 @@ static int sample_into(grf_ctx* ctx, grf_features* feat, const grf_walk_params& 
     GRF_TRY(grf_csr_reserve(&feat->phi, N, N, 0));
     GRF_TRY(grf_csr_reserve(&feat->psi, N, N, 0));
 
+    const bool keep = ctx->keep_walks;
+    feat->kept.valid = false;
+    if (keep) {
+        GRF_TRY(grf_buf_reserve(&ctx->stage_dep_start, rows2 * stride * sizeof(int32_t)));
+        GRF_TRY(grf_buf_reserve(&ctx->stage_dep_t, rows2 * (size_t)P.cap));
+        GRF_TRY(grf_buf_reserve(&ctx->stage_dep_load, rows2 * (size_t)P.cap * sizeof(float)));
+        GRF_TRY(grf_buf_reserve(&ctx->dep_counts, rows2 * sizeof(int32_t)));
+        GRF_TRY(grf_buf_reserve(&ctx->dep_rowptr2, 2 * ((size_t)N + 1) * sizeof(int32_t)));
+    }
+
     const size_t per_warp = walk_smem_per_warp(P);
     int warps = (int)((200u * 1024u) / per_warp);
     if (warps > 8) warps = 8;
     if (warps < 1) warps = 1;
     const size_t smem = per_warp * warps;
     static_assert(sizeof(grf_walk_params) <= 4096, "kernel parameter block too large");
-    GRF_CUDA_TRY(cudaFuncSetAttribute(walk_merge_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    GRF_CUDA_TRY(cudaFuncSetAttribute(walk_merge_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    GRF_CUDA_TRY(cudaFuncSetAttribute(walk_merge_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     {
         grf_launch_scope scope(ctx, 0);
-        walk_merge_kernel<<<grf_ceil_div(rows2, warps), warps * 32, smem, ctx->stream>>>(
-            P, rowptr, col, w, stride, (int32_t*)ctx->stage_col.ptr, (float*)ctx->stage_val.ptr,
-            (int32_t*)ctx->counts.ptr);
+        if (keep)
+            walk_merge_kernel<true><<<grf_ceil_div(rows2, warps), warps * 32, smem, ctx->stream>>>(
+                P, rowptr, col, w, stride, (int32_t*)ctx->stage_col.ptr, (float*)ctx->stage_val.ptr,
+                (int32_t*)ctx->counts.ptr, (int32_t*)ctx->stage_dep_start.ptr, (unsigned char*)ctx->stage_dep_t.ptr,
+                (float*)ctx->stage_dep_load.ptr, (int32_t*)ctx->dep_counts.ptr);
+        else
+            walk_merge_kernel<false><<<grf_ceil_div(rows2, warps), warps * 32, smem, ctx->stream>>>(
+                P, rowptr, col, w, stride, (int32_t*)ctx->stage_col.ptr, (float*)ctx->stage_val.ptr,
+                (int32_t*)ctx->counts.ptr, nullptr, nullptr, nullptr, nullptr);
     }
     GRF_CUDA_TRY(cudaGetLastError());
 
     // counts -> row pointers of Phi (segment 0) and Psi (segment 1)
     int32_t* scan_out = (int32_t*)ctx->rowptr2.ptr;
     GRF_TRY(grf_exclusive_scan(ctx, (const int32_t*)ctx->counts.ptr, scan_out, N, 2));
+    int32_t* dep_scan = (int32_t*)ctx->dep_rowptr2.ptr;
+    if (keep) {
+        GRF_TRY(grf_exclusive_scan(ctx, (const int32_t*)ctx->dep_counts.ptr, dep_scan, N, 2));
+        GRF_CUDA_TRY(cudaMemcpyAsync(ctx->pinned + 2, dep_scan + N, sizeof(int32_t), cudaMemcpyDeviceToHost, ctx->stream));
+        GRF_CUDA_TRY(cudaMemcpyAsync(ctx->pinned + 3, dep_scan + 2 * N + 1, sizeof(int32_t), cudaMemcpyDeviceToHost,
+                                     ctx->stream));
+    }
     GRF_CUDA_TRY(cudaMemcpyAsync(feat->phi.rowptr.ptr, scan_out, ((size_t)N + 1) * sizeof(int32_t),
                                  cudaMemcpyDeviceToDevice, ctx->stream));
     GRF_CUDA_TRY(cudaMemcpyAsync(feat->psi.rowptr.ptr, scan_out + N + 1, ((size_t)N + 1) * sizeof(int32_t),
@@ -343,6 +438,29 @@ static int sample_into(grf_ctx* ctx, grf_features* feat, const grf_walk_params& 
             (int32_t*)feat->psi.col.ptr, (float*)feat->psi.val.ptr);
     }
     GRF_CUDA_TRY(cudaGetLastError());
+    if (keep) {
+        grf_kept_walks& K = feat->kept;
+        const int64_t nnz_e[2] = {nnz_phi, nnz_psi};
+        for (int e = 0; e < 2; ++e) {
+            K.deposits[e] = ctx->pinned[2 + e];
+            const size_t dcap = (size_t)K.deposits[e] + (size_t)K.deposits[e] / 8 + 64;
+            if (K.dep_ptr[e].bytes < ((size_t)nnz_e[e] + 1) * 4)
+                GRF_TRY(grf_buf_reserve(&K.dep_ptr[e], ((size_t)nnz_e[e] + (size_t)nnz_e[e] / 8 + 65) * 4));
+            if (K.dep_t[e].bytes < (size_t)K.deposits[e]) GRF_TRY(grf_buf_reserve(&K.dep_t[e], dcap));
+            if (K.dep_load[e].bytes < (size_t)K.deposits[e] * 4) GRF_TRY(grf_buf_reserve(&K.dep_load[e], dcap * 4));
+        }
+        {
+            grf_launch_scope scope(ctx, 2);
+            compact_deposits_kernel<<<grf_ceil_div(rows2, 8), 256, 0, ctx->stream>>>(
+                N, stride, P.cap, (const int32_t*)ctx->stage_dep_start.ptr, (const unsigned char*)ctx->stage_dep_t.ptr,
+                (const float*)ctx->stage_dep_load.ptr, (const int32_t*)feat->phi.rowptr.ptr,
+                (const int32_t*)feat->psi.rowptr.ptr, dep_scan,
+                (int32_t*)K.dep_ptr[0].ptr, (unsigned char*)K.dep_t[0].ptr, (float*)K.dep_load[0].ptr,
+                (int32_t*)K.dep_ptr[1].ptr, (unsigned char*)K.dep_t[1].ptr, (float*)K.dep_load[1].ptr);
+        }
+        GRF_CUDA_TRY(cudaGetLastError());
+        K.n_walks = P.n_walks; K.max_len = P.max_len; K.valid = true;
+    }
 
     GRF_TRY(grf_transpose_launch(ctx, N, N, nnz_psi, (const int32_t*)feat->psi.rowptr.ptr,
                                  (const int32_t*)feat->psi.col.ptr, (const float*)feat->psi.val.ptr,
@@ -391,5 +509,44 @@ extern "C" int grf_debug_walks(grf_ctx* ctx, int32_t N, const int32_t* rowptr, c
         debug_walks_kernel<<<grf_ceil_div(total, 256), 256, 0, ctx->stream>>>(P, rowptr, col, w, traj, load);
     }
     GRF_CUDA_TRY(cudaGetLastError());
+    return GRF_OK;
+}
+
+extern "C" int grf_ctx_keep_walks(grf_ctx* ctx, int enable)
+{
+    if (!ctx) return GRF_ERR_INVALID;
+    ctx->keep_walks = enable != 0;
+    return GRF_OK;
+}
+
+extern "C" int grf_remodulate(grf_ctx* ctx, grf_features* feat, int32_t max_len, const float* f_phi, const float* f_psi)
+{
+    if (!ctx || !feat || !f_phi) return GRF_ERR_INVALID;
+    grf_kept_walks& K = feat->kept;
+    if (!K.valid || max_len != K.max_len) return GRF_ERR_INVALID;
+    GRF_CUDA_TRY(cudaSetDevice(ctx->device));
+    if (!f_psi) f_psi = f_phi;
+    grf_remod_params P;
+    for (int t = 0; t <= GRF_MAX_WALK_LEN; ++t) {
+        P.f[0][t] = t <= max_len ? f_phi[t] : 0.0f;
+        P.f[1][t] = t <= max_len ? f_psi[t] : 0.0f;
+    }
+    P.inv_n = 1.0f / (float)K.n_walks;
+    grf_csr_dev* mats[2] = {&feat->phi, &feat->psi};
+    for (int e = 0; e < 2; ++e) {
+        if (mats[e]->nnz == 0) continue;
+        grf_launch_scope scope(ctx, 2);
+        remodulate_kernel<<<grf_ceil_div(mats[e]->nnz, 256), 256, 0, ctx->stream>>>(
+            P, e, mats[e]->nnz, (const int32_t*)K.dep_ptr[e].ptr, (const unsigned char*)K.dep_t[e].ptr,
+            (const float*)K.dep_load[e].ptr, (float*)mats[e]->val.ptr);
+    }
+    GRF_CUDA_TRY(cudaGetLastError());
+    // Psi^T carries copies of Psi's values: regroup again (same structure, new values)
+    GRF_TRY(grf_transpose_launch(ctx, feat->psi.rows, feat->psi.cols, feat->psi.nnz, (const int32_t*)feat->psi.rowptr.ptr,
+                                 (const int32_t*)feat->psi.col.ptr, (const float*)feat->psi.val.ptr,
+                                 (int32_t*)feat->psit.rowptr.ptr, (int32_t*)feat->psit.col.ptr,
+                                 (float*)feat->psit.val.ptr));
+    feat->plan_stale = true;       // the coefficient table of the tensor-core gather holds Phi's old values
+    feat->plan_ready = false;
     return GRF_OK;
 }
