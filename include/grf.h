@@ -183,9 +183,9 @@ size_t grf_attn_workspace_bytes(int32_t G, int32_t R, int32_t m, int32_t d, int 
  * GRF_DTYPE_F32 or _BF16 (bf16: S is stored in bf16, sums are carried in fp32).  den_out: optional
  * DEVICE fp32 [G][N] receiving the denominators.  A row whose denominator is exactly 0 yields out = 0.
  * m, d in {8, 16, 32, 64, 128}.  workspace: DEVICE, 256-byte aligned.  Summation order is fixed, so
- * results are run-to-run identical.  Asynchronous, except that the first bf16 call after the features were
- * created or resampled prepares a per-block plan of Phi inside the feature object, which waits for the stream
- * once (so a feature object must not be used by two threads at the same time).
+ * results are run-to-run identical.  Asynchronous, except that the first bf16 call with m and d multiples of 16
+ * after the features were created, resampled or re-modulated prepares a per-block plan of Phi inside the feature
+ * object, which waits for the stream once (so a feature object must not be used by two threads at the same time).
  */
 int grf_masked_linear_attn(grf_ctx* ctx, const grf_features* feat, int32_t G, int32_t N, int32_t m, int32_t d,
                            int dtype, const void* phiQ, const void* phiK, const void* V,
@@ -207,6 +207,32 @@ int grf_masked_linear_attn(grf_ctx* ctx, const grf_features* feat, int32_t G, in
 int grf_masked_attn_asym(grf_ctx* ctx, const grf_features* feat, int32_t G, int32_t N, int32_t m, int32_t d,
                          int dtype, int kernel, const void* Q, const void* K, const void* V, void* out,
                          float* den_out);
+
+/*
+ * Masked attention with the mask estimate materialised (Eqs. 1-2 with Mhat = Phi Psi^T, Sec. 3.3: Mhat_ij =
+ * phi_hat(v_i)^T phi_hat(v_j)): the same outputs as grf_masked_linear_attn, computed over the non-zeros of Mhat
+ * instead of through the per-node states of Eq. 12.  It pays where consecutive node ids are neighbours in the
+ * graph (grids, spatially sorted point clouds): the rows of a block of 128 queries then reach few keys between them.
+ *
+ * grf_features_materialise: forms Mhat once for a feature object (N x N; Phi and Psi may be N x R) as dense bf16
+ * blocks, one per 128 consecutive rows, over the sorted list of keys the block reaches (sums in fp32, fixed order).
+ * Needs the block plan of Phi (built here if absent).  Waits for the stream twice.  The mask is dropped when the
+ * object is resampled or re-modulated.  GRF_ERR_TOO_LARGE when N > 294912 or the blocks would exceed 8 GiB (no
+ * locality: use grf_masked_linear_attn).
+ * grf_mask_stats: HOST outputs (any may be NULL): number of blocks, key entries summed over the blocks (padded
+ * to multiples of 64), device bytes held.  GRF_ERR_INVALID when the object holds no mask.
+ * grf_mask_rows: writes n dense rows of Mhat, out[x][j] = Mhat[rows[x]][j], fp32, to DEVICE out [n][N];
+ * rows: DEVICE int32 [n].  Asynchronous.
+ * grf_masked_attn_mhat: out_i = sum_j Mhat_ij (phi(q_i).phi(k_j)) v_j / sum_j Mhat_ij (phi(q_i).phi(k_j)) for G
+ * problems; arguments as grf_masked_linear_attn, no workspace.  dtype GRF_DTYPE_BF16, d = 64, m in {16, 32, 64}
+ * (other shapes: GRF_ERR_INVALID); scores are fp32, the masked scores are rounded to bf16 before they multiply V and
+ * before they are added into the denominator.  Summation order is fixed.  Asynchronous.
+ */
+int grf_features_materialise(grf_ctx* ctx, grf_features* feat);
+int grf_mask_stats(const grf_features* feat, int32_t* blocks, int64_t* key_entries, int64_t* bytes);
+int grf_mask_rows(grf_ctx* ctx, const grf_features* feat, int32_t n, const int32_t* rows, float* out);
+int grf_masked_attn_mhat(grf_ctx* ctx, const grf_features* feat, int32_t G, int32_t N, int32_t m, int32_t d,
+                         int dtype, const void* phiQ, const void* phiK, const void* V, void* out, float* den_out);
 
 /*
  * The whole path of Alg. 1 from HOST buffers, for callers that keep nothing on the device:

@@ -120,3 +120,13 @@ def masked_attn_asym(ctx: Context, feat: Features, Q, K, V, softmax=False, want_
     B.grf_masked_attn_asym(ctx.handle, feat.handle, G, N, m, d, B.dtype_code(Q),
                            B.GRF_KERNEL_SOFTMAX if softmax else B.GRF_KERNEL_LINEAR, Q, K, V, out, den)
     return (out, den) if want_den else out
+
+
+def masked_attn_mhat(ctx: Context, feat: Features, phiQ, phiK, V, want_den=False):
+    """Eqs. 1-2 over the materialised mask (call B.grf_features_materialise first).  bf16, d = 64."""
+    G, N, m = phiQ.shape
+    d = V.shape[2]
+    out = torch.empty_like(V)
+    den = torch.empty((G, N), dtype=torch.float32, device=V.device) if want_den else None
+    B.grf_masked_attn_mhat(ctx.handle, feat.handle, G, N, m, d, B.dtype_code(phiQ), phiQ, phiK, V, out, den)
+    return (out, den) if want_den else out

@@ -45,6 +45,10 @@ _SIGNATURES = {
     "grf_attn_workspace_bytes": (_sz, [_i32, _i32, _i32, _i32, _int]),
     "grf_masked_linear_attn": (_int, [_vp, _vp, _i32, _i32, _i32, _i32, _int, _vp, _vp, _vp, _vp, _vp, _vp, _sz]),
     "grf_masked_attn_asym": (_int, [_vp, _vp, _i32, _i32, _i32, _i32, _int, _int, _vp, _vp, _vp, _vp, _vp]),
+    "grf_features_materialise": (_int, [_vp, _vp]),
+    "grf_mask_stats": (_int, [_vp, ctypes.POINTER(_i32), ctypes.POINTER(_i64), ctypes.POINTER(_i64)]),
+    "grf_mask_rows": (_int, [_vp, _vp, _i32, _vp, _vp]),
+    "grf_masked_attn_mhat": (_int, [_vp, _vp, _i32, _i32, _i32, _i32, _int, _vp, _vp, _vp, _vp, _vp]),
     "grf_step_host": (_int, [_vp, _i32, _vp, _vp, _vp, _u64, _i32, _f32, _i32, _vp, _vp,
                              _i32, _i32, _i32, _int, _vp, _vp, _vp, _vp]),
     "grf_ctx_launch_count": (_i64, [_vp]),
@@ -231,6 +235,26 @@ def grf_masked_linear_attn(ctx, features, G, N, m, d, dtype, phiQ, phiK, V, out,
 def grf_masked_attn_asym(ctx, features, G, N, m, d, dtype, kernel, Q, K, V, out, den_out):
     _check(lib.grf_masked_attn_asym(ctx, features, G, N, m, d, dtype, kernel, _dev(Q), _dev(K), _dev(V), _dev(out),
                                     _dev(den_out)), "grf_masked_attn_asym")
+
+
+def grf_features_materialise(ctx, features):
+    _check(lib.grf_features_materialise(ctx, features), "grf_features_materialise")
+
+
+def grf_mask_stats(features):
+    """(blocks, key entries over all blocks, device bytes)."""
+    b, e, n = _i32(), _i64(), _i64()
+    _check(lib.grf_mask_stats(features, ctypes.byref(b), ctypes.byref(e), ctypes.byref(n)), "grf_mask_stats")
+    return b.value, e.value, n.value
+
+
+def grf_mask_rows(ctx, features, n, rows, out):
+    _check(lib.grf_mask_rows(ctx, features, n, _dev(rows), _dev(out)), "grf_mask_rows")
+
+
+def grf_masked_attn_mhat(ctx, features, G, N, m, d, dtype, phiQ, phiK, V, out, den_out):
+    _check(lib.grf_masked_attn_mhat(ctx, features, G, N, m, d, dtype, _dev(phiQ), _dev(phiK), _dev(V), _dev(out),
+                                    _dev(den_out)), "grf_masked_attn_mhat")
 
 
 def grf_step_host(ctx, N, rowptr, col, w, seed, n_walks, p_halt, max_len, f_phi, f_psi, G, m, d, dtype,

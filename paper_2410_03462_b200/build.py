@@ -10,7 +10,7 @@ CSRC = os.path.join(HERE, "csrc")
 INCLUDE = os.path.join(os.path.dirname(HERE), "include")
 LIB = os.path.join(HERE, "libgrf.so")
 SOURCES = ["api.cu", "sample.cu", "scan.cu", "transpose.cu", "attn_state.cu", "attn_gather.cu", "attn_gather_tc.cu",
-           "attn_state_tc.cu", "attn_asym.cu"]
+           "attn_state_tc.cu", "attn_asym.cu", "tensor_map.cu", "attn_mhat.cu"]
 
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-std=c++17", "-lineinfo",

@@ -185,6 +185,7 @@ extern "C" int grf_features_free(grf_features* feat)
     csr_release(&feat->phi); csr_release(&feat->psi); csr_release(&feat->psit);
     grf_buf_release(&feat->plan_off); grf_buf_release(&feat->plan_cnt);
     grf_buf_release(&feat->plan_col); grf_buf_release(&feat->plan_total); grf_buf_release(&feat->plan_coef);
+    grf_mask_release(feat);
     for (int e = 0; e < 2; ++e) {
         grf_buf_release(&feat->kept.dep_ptr[e]); grf_buf_release(&feat->kept.dep_t[e]); grf_buf_release(&feat->kept.dep_load[e]);
     }
@@ -298,7 +299,9 @@ extern "C" int grf_masked_linear_attn(grf_ctx* ctx, const grf_features* feat, in
     if (chunk > 65535) chunk = 65535;
     const size_t es = elem_size(dtype);
     // the plan's build waits for the stream once: do it before the attention kernels are queued, not between them
-    if (dtype == GRF_DTYPE_BF16 && ctx->use_tensor_cores) GRF_TRY(grf_ensure_block_plan(ctx, feat));
+    // (only for shapes the tensor-core gather covers: other shapes never read the plan)
+    if (dtype == GRF_DTYPE_BF16 && ctx->use_tensor_cores && m % 16 == 0 && d % 16 == 0)
+        GRF_TRY(grf_ensure_block_plan(ctx, feat));
     for (int64_t g0 = 0; g0 < G; g0 += chunk) {
         const int32_t gc = (int32_t)((G - g0) < chunk ? (G - g0) : chunk);
         // chunk layout: records [gc][R], contiguous

@@ -215,7 +215,7 @@ extern "C" int grf_masked_attn_asym(grf_ctx* ctx, const grf_features* feat, int3
                                     float* den_out)
 {
     if (!ctx || !feat || !Q || !K || !V || !out) return GRF_ERR_INVALID;
-    if (G <= 0 || G > 65535 * ASYM_GH || N <= 0) return GRF_ERR_INVALID;
+    if (G <= 0 || G > 65535 || N <= 0) return GRF_ERR_INVALID;
     if (kernel != GRF_KERNEL_LINEAR && kernel != GRF_KERNEL_SOFTMAX) return GRF_ERR_INVALID;
     if (dtype != GRF_DTYPE_F32 && dtype != GRF_DTYPE_BF16) return GRF_ERR_INVALID;
     if (feat->phi.rows != N || feat->phi.cols != N) return GRF_ERR_INVALID;       // the mask estimate is Phi: N x N

@@ -19,132 +19,12 @@
 //     its copies and MMAs, frees its tensor memory and exits.
 // Nodes that no query of the block touches are never loaded; a tile is loaded once per block, not once
 // per query, which is where the method's "constant multiplicative cost" is paid down.
-#include "grf_internal.cuh"
+#include "tc_common.cuh"
 
 namespace {
 
 constexpr int BQ = GRF_PLAN_BLOCK;  // queries per CTA = MMA M
-constexpr long long WAIT_CYCLES = 4000000000ll;   // a wait that lasts longer than this (about 2 s) gives up
-
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
-{
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar)
-{
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
-{
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-    return ok != 0;
-}
-// Bounded wait: false when another thread of the CTA has given up or when this wait lasted too long
-// (then it raises the CTA's abort flag itself).
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag)
-{
-    long long t0 = 0;
-    for (uint32_t it = 0;; ++it) {
-        if (mbar_try_wait(bar, parity)) return true;
-        if ((it & 63u) == 63u) {
-            if (*abort_flag) return false;
-            const long long now = clock64();
-            if (t0 == 0) t0 = now;
-            else if (now - t0 > WAIT_CYCLES) { *abort_flag = 1; return false; }
-        }
-    }
-}
-
-// Shared-memory operand descriptor: unswizzled, 8-row core matrices of 128 contiguous bytes;
-// lbo = byte distance between the two 16-byte K chunks of one instruction, sbo = between 8-row groups.
-__device__ __forceinline__ uint64_t operand_desc(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes)
-{
-    uint64_t d = (uint64_t)((saddr & 0x3FFFFu) >> 4);
-    d |= (uint64_t)(lbo_bytes >> 4) << 16;
-    d |= (uint64_t)(sbo_bytes >> 4) << 32;
-    d |= (uint64_t)1 << 46;  // descriptor version of this architecture
-    return d;
-}
-
-// Instruction descriptor: bf16 x bf16 -> fp32, both operands K-major, M = 128, N = n.
-__host__ __device__ constexpr uint32_t instr_desc_bf16(int n)
-{
-    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
-}
-
-// The issuing helpers below are called by ALL lanes of a converged warp with the same arguments; elect.sync
-// picks the lane that issues.  (Issued from a branch that only one lane takes, the same instruction costs
-// its thread about three times as many cycles: the operands of these instructions are warp-uniform.)
-__device__ __forceinline__ void mma_commit(uint32_t bar)
-{
-    asm volatile(
-        "{\n\t.reg .pred q;\n\t"
-        "elect.sync _|q, 0xffffffff;\n\t"
-        "@q tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n\t}"
-        ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ void expect_tx_elected(uint32_t bar, uint32_t bytes)
-{
-    asm volatile(
-        "{\n\t.reg .pred q;\n\t"
-        "elect.sync _|q, 0xffffffff;\n\t"
-        "@q mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;\n\t}"
-        ::"r"(bar), "r"(bytes) : "memory");
-}
-// bulk copy of one record into its slot, by one elected lane
-__device__ __forceinline__ void load_record_elected(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar)
-{
-    asm volatile(
-        "{\n\t.reg .pred q;\n\t"
-        "elect.sync _|q, 0xffffffff;\n\t"
-        "@q cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];\n\t}"
-        ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
-}
-
-__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16])
-{
-    asm volatile(
-        "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
-        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
-          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
-        : "r"(taddr));
-    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-}
-
-__device__ __forceinline__ void tmem_st8(uint32_t taddr, const uint32_t (&r)[8])
-{
-    asm volatile("tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
-                 ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7])
-                 : "memory");
-}
-
-__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&r)[16])
-{
-    asm volatile(
-        "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};"
-        ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),
-          "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
-        : "memory");
-}
-
-// A operand in tensor memory (row i of the block = lane i, two bf16 per 32-bit column), B in shared memory
-__device__ __forceinline__ void mma_bf16_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t bdesc, uint32_t idesc,
-                                            uint32_t accumulate)
-{
-    asm volatile(
-        "{\n\t.reg .pred p, q;\n\t"
-        "setp.ne.b32 p, %4, 0;\n\t"
-        "elect.sync _|q, 0xffffffff;\n\t"
-        "@q tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
-        ::"r"(d_tmem), "r"(a_tmem), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
-}
+using namespace grf_tc;
 
 constexpr int pow2_at_least(int x) { return x <= 32 ? 32 : (x <= 64 ? 64 : (x <= 128 ? 128 : (x <= 256 ? 256 : 512))); }
 
@@ -351,7 +231,7 @@ gather_contract_tc_kernel(int32_t G, int32_t nblocks, int32_t N, int32_t R, cons
             for (int j = 0; j < GU; ++j) {
                 const int32_t u = gi * GU + j;
                 if (u < uend)
-                    load_record_elected(b_base + (uint32_t)(u % NREC) * Sh::TILE_BYTES, recs + (size_t)l_cur[j] * Sh::REC_BYTES,
+                    bulk_load_elected(b_base + (uint32_t)(u % NREC) * Sh::TILE_BYTES, recs + (size_t)l_cur[j] * Sh::REC_BYTES,
                                         Sh::TILE_BYTES, rec_full(gi % NBC));
             }
             issued = uend;
@@ -370,7 +250,7 @@ gather_contract_tc_kernel(int32_t G, int32_t nblocks, int32_t N, int32_t R, cons
         // ------------------------------------------------------------ MMA issuer: all groups, in list order
         // The whole warp runs the loop in step (every exit is voted on), so that the issuing helpers meet a
         // converged warp.
-        constexpr uint32_t idesc = instr_desc_bf16(D);
+        constexpr uint32_t idesc = instr_desc(D, false, false);
         const uint32_t acc = tmem_base;
         bool ok = true;
         bool first = true;

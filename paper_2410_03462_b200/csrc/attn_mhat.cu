@@ -1,0 +1,600 @@
+// Masked attention with the mask estimate materialised (Eqs. 1-2 with Mhat = Phi Psi^T, Sec. 3.3), bf16 storage.
+//
+// Instead of going through the per-node states of Eq. 12, the sparse product Mhat = Phi Psi^T is formed once per
+// feature object and the attention is evaluated from its definition,
+//     out_i = sum_j Mhat_ij (phi(q_i) . phi(k_j)) v_j / sum_j Mhat_ij (phi(q_i) . phi(k_j)),
+// over the non-zeros of Mhat only.  On graphs whose node numbering keeps neighbours together, the rows of a block
+// of 128 consecutive queries reach a few thousand keys between them and about a quarter of that block of Mhat is
+// non-zero: dense enough for the tensor cores.  Per block the mask is stored densely (bf16) over the block's key
+// list, and one CTA per (block, problem) runs a two-product pipeline over tiles of 64 keys:
+//     S = phi(Q_blk) phi(K_tile)^T   (tcgen05, accumulator in tensor memory)
+//     P = S * Mhat_tile              (row threads: tensor memory -> registers -> tensor memory, bf16)
+//     O += P V_tile                  (tcgen05, P read from tensor memory)
+// and the row sums of P give the denominators.  Key and value rows are gathered by key index: value rows by the
+// tensor-map copy engine (tile::gather4) into the 128-byte-swizzled operand layout, key-feature rows by 16-byte
+// asynchronous copies into the unswizzled K-major layout.
+//
+// Building the mask (once per feature object): the key list of a block is the union of the rows of Psi^T over the
+// block's node list (the block plan of Phi); the values are accumulated row by row, one warp per row, in ascending
+// order of the node l, each lane owning distinct keys, so the sums are reproducible without atomics.
+#include "tc_common.cuh"
+
+namespace {
+
+using namespace grf_tc;
+
+constexpr int BQ = GRF_PLAN_BLOCK;      // queries per block
+constexpr int KT = GRF_MASK_TILE;       // keys per tile
+
+// ---------------------------------------------------------------------------------------------------
+// Key lists: one CTA per block of rows.  Two passes: pass 0 counts (the counts, padded to whole tiles, are then
+// scanned into offsets), pass 1 writes the sorted lists.
+
+__global__ void __launch_bounds__(256)
+mask_keys_kernel(int32_t Nk, const int32_t* __restrict__ plan_off, const int32_t* __restrict__ plan_cnt,
+                 const int32_t* __restrict__ plan_col, const int32_t* __restrict__ t_rowptr,
+                 const int32_t* __restrict__ t_col, int pass, const int32_t* __restrict__ mk_off,
+                 int32_t* __restrict__ mk_cnt, int32_t* __restrict__ mk_key)
+{
+    extern __shared__ uint32_t bitmap[];        // one bit per key
+    __shared__ int32_t warp_sums[8];
+    __shared__ int32_t block_total;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int32_t blk = blockIdx.x;
+    const int32_t words = (Nk + 31) >> 5;
+    for (int32_t x = tid; x < words; x += 256) bitmap[x] = 0u;
+    __syncthreads();
+    const int32_t* ulist = plan_col + plan_off[blk];
+    const int32_t ucnt = plan_cnt[blk];
+    for (int32_t u = warp; u < ucnt; u += 8) {
+        const int32_t l = ulist[u];
+        for (int32_t p = t_rowptr[l] + lane; p < t_rowptr[l + 1]; p += 32) {
+            const int32_t j = t_col[p];
+            atomicOr(&bitmap[j >> 5], 1u << (j & 31));
+        }
+    }
+    __syncthreads();
+    // each thread owns a contiguous range of words so that the list comes out sorted
+    const int32_t per = (words + 255) / 256;
+    const int32_t w0 = min(words, tid * per), w1 = min(words, w0 + per);
+    int32_t mine = 0;
+    for (int32_t x = w0; x < w1; ++x) mine += __popc(bitmap[x]);
+    int32_t inc = mine;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const int32_t y = __shfl_up_sync(0xffffffffu, inc, o);
+        if (lane >= o) inc += y;
+    }
+    if (lane == 31) warp_sums[warp] = inc;
+    __syncthreads();
+    int32_t before = inc - mine;
+    for (int w = 0; w < warp; ++w) before += warp_sums[w];
+    if (tid == 255) {
+        block_total = before + mine;
+        if (pass == 0) mk_cnt[blk] = (block_total + KT - 1) / KT * KT;
+    }
+    if (pass == 0) return;
+    __syncthreads();
+    const int32_t base_off = mk_off[blk];
+    int32_t o = base_off + before;
+    for (int32_t x = w0; x < w1; ++x) {
+        uint32_t bits = bitmap[x];
+        while (bits) {
+            const int b = __ffs(bits) - 1;
+            bits &= bits - 1;
+            mk_key[o++] = (x << 5) + b;
+        }
+    }
+    __syncthreads();
+    // padding: the last key again (its mask values are zeros)
+    const int32_t padded = (block_total + KT - 1) / KT * KT;
+    if (block_total > 0)
+        for (int32_t e = block_total + tid; e < padded; e += 256) mk_key[base_off + e] = mk_key[base_off + block_total - 1];
+}
+
+// order[r] = the block with the r-th largest key list (ties: lower index first), stored behind the counts
+__global__ void __launch_bounds__(256) mask_order_kernel(int32_t nblocks, int32_t* __restrict__ mk_cnt)
+{
+    const int32_t i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= nblocks) return;
+    const int32_t c = mk_cnt[i];
+    int32_t rank = 0;
+    for (int32_t j = 0; j < nblocks; ++j) {
+        const int32_t cj = mk_cnt[j];
+        rank += (cj > c || (cj == c && j < i)) ? 1 : 0;
+    }
+    mk_cnt[nblocks + rank] = i;
+}
+
+// ---------------------------------------------------------------------------------------------------
+// Mask values: Mhat_ij = sum_l Phi_il Psi_jl for the rows i of one block and the keys j of its list.
+// One CTA per block, one warp per row at a time.  The warp keeps the row's accumulators (fp32, one per key of a
+// segment of the list) in shared memory; for every non-zero Phi_il, taken in ascending l, its lanes add
+// Phi_il * Psi_jl at the position of key j, found from a bitmap of the block's keys and the number of set bits
+// before each bitmap word.  Keys of one l are distinct, so no two lanes meet at one position, and the warp is
+// synchronised between two l: the order of every sum is fixed.  Lists longer than a segment take further passes.
+
+constexpr int MASK_SEG = 4096;          // accumulators per warp
+constexpr int MASK_WARPS = 8;
+
+__global__ void __launch_bounds__(MASK_WARPS * 32)
+mask_values_kernel(int32_t N, int32_t Nk, const int32_t* __restrict__ phi_rowptr, const int32_t* __restrict__ phi_col,
+                   const float* __restrict__ phi_val, const int32_t* __restrict__ t_rowptr,
+                   const int32_t* __restrict__ t_col, const float* __restrict__ t_val,
+                   const int32_t* __restrict__ mk_off, const int32_t* __restrict__ mk_cnt,
+                   const int32_t* __restrict__ mk_key, __nv_bfloat16* __restrict__ mk_val)
+{
+    extern __shared__ uint32_t smem_mask[];     // bitmap, set bits before each word, accumulators
+    __shared__ int32_t warp_sums[MASK_WARPS];
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int32_t blk = blockIdx.x;
+    const int32_t words = (Nk + 31) >> 5;
+    uint32_t* bitmap = smem_mask;
+    int32_t* before_word = reinterpret_cast<int32_t*>(smem_mask + words);
+    float* acc = reinterpret_cast<float*>(smem_mask + 2 * (size_t)words) + (size_t)warp * MASK_SEG;
+    const int32_t off = mk_off[blk], cnt = mk_cnt[blk];
+    for (int32_t x = tid; x < words; x += MASK_WARPS * 32) bitmap[x] = 0u;
+    __syncthreads();
+    for (int32_t e = tid; e < cnt; e += MASK_WARPS * 32) {
+        const int32_t j = mk_key[off + e];
+        atomicOr(&bitmap[j >> 5], 1u << (j & 31));
+    }
+    __syncthreads();
+    {
+        const int32_t per = (words + MASK_WARPS * 32 - 1) / (MASK_WARPS * 32);
+        const int32_t w0 = min(words, tid * per), w1 = min(words, w0 + per);
+        int32_t mine = 0;
+        for (int32_t x = w0; x < w1; ++x) mine += __popc(bitmap[x]);
+        int32_t inc = mine;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const int32_t y = __shfl_up_sync(0xffffffffu, inc, o);
+            if (lane >= o) inc += y;
+        }
+        if (lane == 31) warp_sums[warp] = inc;
+        __syncthreads();
+        int32_t run = inc - mine;
+        for (int w = 0; w < warp; ++w) run += warp_sums[w];
+        for (int32_t x = w0; x < w1; ++x) { before_word[x] = run; run += __popc(bitmap[x]); }
+    }
+    __syncthreads();
+    const int32_t r0 = blk * BQ;
+    for (int32_t seg0 = 0; seg0 < cnt; seg0 += MASK_SEG) {
+        const int32_t seglen = min(MASK_SEG, cnt - seg0);       // a multiple of the tile, hence of 8
+        for (int32_t rr = warp; rr < BQ; rr += MASK_WARPS) {
+            const int32_t r = r0 + rr;
+            for (int32_t x = lane; x < seglen; x += 32) acc[x] = 0.0f;
+            __syncwarp();
+            if (r < N) {
+                for (int32_t p = phi_rowptr[r]; p < phi_rowptr[r + 1]; ++p) {
+                    const int32_t l = __ldg(phi_col + p);
+                    const float phi = __ldg(phi_val + p);
+                    for (int32_t q = __ldg(t_rowptr + l) + lane; q < __ldg(t_rowptr + l + 1); q += 32) {
+                        const int32_t j = __ldg(t_col + q);
+                        const int32_t pos = before_word[j >> 5] + __popc(bitmap[j >> 5] & ((1u << (j & 31)) - 1u)) - seg0;
+                        if (pos >= 0 && pos < seglen) acc[pos] = fmaf(phi, __ldg(t_val + q), acc[pos]);
+                    }
+                    __syncwarp();
+                }
+            }
+            // the row's values of this segment, eight keys (16 bytes) per lane at a time
+            for (int32_t c8 = lane; c8 < seglen / 8; c8 += 32) {
+                uint32_t w[4];
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    const __nv_bfloat162 h = __floats2bfloat162_rn(acc[c8 * 8 + 2 * e], acc[c8 * 8 + 2 * e + 1]);
+                    w[e] = *reinterpret_cast<const uint32_t*>(&h);
+                }
+                uint4* dst = reinterpret_cast<uint4*>(mk_val + ((size_t)((off + seg0) / 8 + c8) * BQ + rr) * 8);
+                *dst = make_uint4(w[0], w[1], w[2], w[3]);
+            }
+            __syncwarp();
+        }
+    }
+}
+
+// Dense rows of the mask for checking and export: out[x][j] = Mhat[rows[x]][j] (zeros elsewhere), one CTA per row.
+__global__ void __launch_bounds__(256)
+mask_rows_kernel(int32_t Nk, const int32_t* __restrict__ rows, const int32_t* __restrict__ mk_off,
+                 const int32_t* __restrict__ mk_cnt, const int32_t* __restrict__ mk_key,
+                 const __nv_bfloat16* __restrict__ mk_val, float* __restrict__ out)
+{
+    const int32_t r = rows[blockIdx.x];
+    float* o = out + (size_t)blockIdx.x * Nk;
+    for (int32_t j = threadIdx.x; j < Nk; j += 256) o[j] = 0.0f;
+    __syncthreads();
+    const int32_t blk = r / BQ, rr = r % BQ;
+    const int32_t off = mk_off[blk], cnt = mk_cnt[blk];
+    // padding entries repeat the last key with the value 0: skip an entry whose predecessor has the same key
+    for (int32_t e = threadIdx.x; e < cnt; e += 256) {
+        const int32_t j = mk_key[off + e];
+        if (e > 0 && mk_key[off + e - 1] == j) continue;
+        o[j] = __bfloat162float(mk_val[((size_t)((off + e) / 8) * BQ + rr) * 8 + ((off + e) & 7)]);
+    }
+}
+
+// ---------------------------------------------------------------------------------------------------
+// The attention kernel.  warps 0-3: row threads (one query = one tensor-memory lane each); warp 4: producer
+// (gathers of key-feature and value rows); warp 5: MMA issuer.
+
+template <int M> struct MhShape {
+    static constexpr int D = 64;
+    static constexpr int NS = 4;                          // key/value stages in flight
+    static constexpr int V_BYTES = KT * 128;              // 64 gathered value rows, 128-byte swizzle
+    static constexpr int K_BYTES = KT * M * 2;            // [M/8][KT keys][8] bf16: K-major, unswizzled
+    static constexpr int STAGE = V_BYTES + K_BYTES;
+    static constexpr int Q_BYTES = BQ * M * 2;            // [M/8][128 rows][8] bf16
+    static constexpr int S_COLS = KT;                     // one score buffer; P (bf16 pairs) reuses its first half
+    static constexpr int O_COL = 2 * S_COLS;
+    static constexpr int TMEM_COLS = 256;                 // 2 score buffers + the output accumulator, rounded up
+    static constexpr size_t SMEM = (size_t)NS * STAGE + Q_BYTES + 1024;
+    static_assert(STAGE % 1024 == 0, "stages must keep the swizzle phase");
+};
+
+constexpr int MH_THREADS = 192;
+
+template <int M>
+__global__ void __launch_bounds__(MH_THREADS)
+mhat_attention_kernel(int32_t G, int32_t nblocks, int32_t N, const int32_t* __restrict__ mk_off,
+                      const int32_t* __restrict__ mk_cnt, const int32_t* __restrict__ mk_key,
+                      const uint4* __restrict__ mk_val, const __nv_bfloat16* __restrict__ phiQ,
+                      const __nv_bfloat16* __restrict__ phiK, const __grid_constant__ CUtensorMap map_v,
+                      __nv_bfloat16* __restrict__ out, float* __restrict__ den_out, int* __restrict__ error_word)
+{
+    using Sh = MhShape<M>;
+    constexpr int NS = Sh::NS, D = Sh::D;
+    extern __shared__ unsigned char smem_dyn[];
+    // kv_full, kv_empty per stage; s_full, p_full, s_free per score buffer; acc_done; drain
+    __shared__ __align__(8) unsigned long long bars[2 * NS + 6 + 2];
+    __shared__ uint32_t tmem_slot;
+    __shared__ int abort_flag;
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int32_t g = (int32_t)(blockIdx.x % (uint32_t)G);
+    const int32_t blk = mk_cnt[nblocks + (int32_t)(blockIdx.x / (uint32_t)G)];   // blocks by decreasing key count
+    const uint32_t stage_base = (smem_u32(smem_dyn) + 1023u) & ~1023u;
+    unsigned char* stage_generic = smem_dyn + (stage_base - smem_u32(smem_dyn));
+    const uint32_t q_base = stage_base + (uint32_t)NS * Sh::STAGE;
+    const uint32_t bar_base = smem_u32(bars);
+    auto kv_full = [&](int s) { return bar_base + 8u * (uint32_t)s; };
+    auto kv_empty = [&](int s) { return bar_base + 8u * (uint32_t)(NS + s); };
+    auto s_full = [&](int b) { return bar_base + 8u * (uint32_t)(2 * NS + b); };
+    auto p_full = [&](int b) { return bar_base + 8u * (uint32_t)(2 * NS + 2 + b); };
+    auto s_free = [&](int b) { return bar_base + 8u * (uint32_t)(2 * NS + 4 + b); };
+    const uint32_t acc_done = bar_base + 8u * (uint32_t)(2 * NS + 6);
+    const uint32_t drain_bar = bar_base + 8u * (uint32_t)(2 * NS + 7);
+
+    if (tid == 0) {
+        for (int s = 0; s < NS; ++s) { mbar_init(kv_full(s), 2); mbar_init(kv_empty(s), 1); }
+        for (int b = 0; b < 2; ++b) { mbar_init(s_full(b), 1); mbar_init(p_full(b), 4); mbar_init(s_free(b), 1); }
+        mbar_init(acc_done, 1);
+        mbar_init(drain_bar, 1);
+        abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 5) tmem_alloc(&tmem_slot, (uint32_t)Sh::TMEM_COLS);
+    // the block's queries in the K-major operand layout: 16-byte chunk c of row r at (c * 128 + r) * 16
+    if (tid < BQ) {
+        const int32_t row = blk * BQ + tid;
+        const uint4* qp = reinterpret_cast<const uint4*>(phiQ + ((size_t)g * N + min(row, N - 1)) * M);
+#pragma unroll
+        for (int c = 0; c < M / 8; ++c) {
+            const uint4 x = row < N ? __ldg(qp + c) : make_uint4(0u, 0u, 0u, 0u);
+            *reinterpret_cast<uint4*>(stage_generic + (size_t)NS * Sh::STAGE + ((size_t)c * BQ + tid) * 16) = x;
+        }
+    }
+    fence_async_smem();
+    fence_before_sync();
+    __syncthreads();
+    fence_after_sync();
+    const uint32_t tmem_base = tmem_slot;
+
+    const int32_t off = mk_off[blk];
+    const int32_t T = mk_cnt[blk] / KT;                   // key tiles of this block
+
+    if (warp < 4) {
+        // ------------------------------------------------------------ row threads: P = S * Mhat, row sums, epilogue
+        const int32_t row = blk * BQ + tid;
+        const uint32_t lane_field = (uint32_t)(warp * 32) << 16;
+        const uint4* mrow = mk_val + (size_t)(off / 8) * BQ + tid;      // chunk x of this row: mrow[x * BQ]
+        float den = 0.0f;
+        uint4 mk[KT / 8];
+        if (T > 0) {
+#pragma unroll
+            for (int c = 0; c < KT / 8; ++c) mk[c] = __ldg(mrow + (size_t)c * BQ);
+        }
+        bool ok = true;
+        for (int32_t t = 0; t < T; ++t) {
+            const int buf = t & 1;
+            if (!mbar_wait(s_full(buf), (uint32_t)(t >> 1) & 1u, &abort_flag)) ok = false;
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
+            fence_after_sync();
+            const uint32_t s_addr = tmem_base + lane_field + (uint32_t)(buf * Sh::S_COLS);
+#pragma unroll
+            for (int c16 = 0; c16 < KT / 16; ++c16) {
+                uint32_t sv[16];
+                tmem_ld16(s_addr + (uint32_t)(c16 * 16), sv);
+                uint32_t pw[8];
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {
+                    const uint4 mm = mk[2 * c16 + h];
+                    const uint32_t mw[4] = {mm.x, mm.y, mm.z, mm.w};
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        const float p0 = __uint_as_float(sv[8 * h + 2 * e]) * __uint_as_float(mw[e] << 16);
+                        const float p1 = __uint_as_float(sv[8 * h + 2 * e + 1]) * __uint_as_float(mw[e] & 0xffff0000u);
+                        const __nv_bfloat162 pb = __floats2bfloat162_rn(p0, p1);
+                        // the denominator adds the same rounded values the second product multiplies
+                        den += __low2float(pb) + __high2float(pb);
+                        pw[4 * h + e] = *reinterpret_cast<const uint32_t*>(&pb);
+                    }
+                }
+                tmem_st8(s_addr + (uint32_t)(c16 * 8), pw);
+            }
+            // next tile's mask values travel while the products run
+            if (t + 1 < T) {
+#pragma unroll
+                for (int c = 0; c < KT / 8; ++c) mk[c] = __ldg(mrow + (size_t)((t + 1) * (KT / 8) + c) * BQ);
+            }
+            tmem_st_wait();
+            fence_before_sync();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(p_full(buf));
+        }
+        if (ok && T > 0) ok = mbar_wait(acc_done, 0u, &abort_flag);
+        ok = __all_sync(0xffffffffu, ok);
+        fence_after_sync();
+        const bool live = row < N;
+        const float inv = (den != 0.0f) ? 1.0f / den : 0.0f;
+        if (live && ok && den_out) den_out[(size_t)g * N + row] = den;
+        __nv_bfloat16* orow = out + ((size_t)g * N + row) * D;
+#pragma unroll
+        for (int c0 = 0; c0 < D; c0 += 16) {
+            uint32_t r[16];
+#pragma unroll
+            for (int e = 0; e < 16; ++e) r[e] = 0u;
+            if (ok && T > 0) tmem_ld16(tmem_base + lane_field + (uint32_t)(Sh::O_COL + c0), r);
+            if (live && ok) {
+                uint32_t w[8];
+#pragma unroll
+                for (int e = 0; e < 8; ++e) {
+                    __nv_bfloat162 h = __floats2bfloat162_rn(__uint_as_float(r[2 * e]) * inv, __uint_as_float(r[2 * e + 1]) * inv);
+                    w[e] = *reinterpret_cast<uint32_t*>(&h);
+                }
+                uint4* dst = reinterpret_cast<uint4*>(orow + c0);
+                dst[0] = make_uint4(w[0], w[1], w[2], w[3]);
+                dst[1] = make_uint4(w[4], w[5], w[6], w[7]);
+            }
+        }
+    } else if (warp == 4) {
+        // ------------------------------------------------------------ producer: gathers of a tile's 64 keys
+        // Lane x holds keys x and x + 32 of the tile.  Value rows: lanes 0-15 each gather four rows through the
+        // tensor map (they land in the swizzled layout and complete on the stage's barrier by byte count).
+        // Key-feature rows: every lane copies its two keys' rows in 16-byte pieces, piece c of key y going to
+        // (c * 64 + y) * 16; the lane's copies of one tile form one group, and a stage is handed over one tile
+        // late, after its group has completed and a proxy fence.
+        const __nv_bfloat16* Kg = phiK + (size_t)g * N * M;
+        const int32_t row0 = g * N;
+        bool ok = true;
+        int32_t issued = 0;
+        auto hand_over = [&](int32_t t) {
+            fence_async_smem();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(kv_full(t % NS));
+        };
+        for (int32_t t = 0; t < T; ++t) {
+            const int s = t % NS;
+            if (t >= NS && !mbar_wait(kv_empty(s), (uint32_t)(t / NS - 1) & 1u, &abort_flag)) ok = false;
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
+            const int32_t k0 = __ldg(mk_key + off + t * KT + lane), k1 = __ldg(mk_key + off + t * KT + 32 + lane);
+            const uint32_t v_st = stage_base + (uint32_t)s * Sh::STAGE, k_st = v_st + Sh::V_BYTES;
+            if (lane == 0) mbar_expect_tx(kv_full(s), (uint32_t)Sh::V_BYTES);
+            __syncwarp();
+            int32_t r4[4];
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                const int32_t key = 4 * (lane & 15) + e;
+                const int32_t a = __shfl_sync(0xffffffffu, k0, key & 31), b = __shfl_sync(0xffffffffu, k1, key & 31);
+                r4[e] = row0 + (key < 32 ? a : b);
+            }
+            if (lane < 16) tma_gather4(v_st + (uint32_t)lane * 512u, &map_v, r4[0], r4[1], r4[2], r4[3], kv_full(s));
+#pragma unroll
+            for (int c = 0; c < M / 8; ++c) {
+                asm volatile("cp.async.ca.shared.global [%0], [%1], 16;"
+                             ::"r"(k_st + (uint32_t)(c * KT + lane) * 16u), "l"(Kg + (size_t)k0 * M + c * 8) : "memory");
+                asm volatile("cp.async.ca.shared.global [%0], [%1], 16;"
+                             ::"r"(k_st + (uint32_t)(c * KT + 32 + lane) * 16u), "l"(Kg + (size_t)k1 * M + c * 8) : "memory");
+            }
+            asm volatile("cp.async.commit_group;" ::: "memory");
+            issued = t + 1;
+            if (t >= 1) {
+                asm volatile("cp.async.wait_group 1;" ::: "memory");
+                hand_over(t - 1);
+            }
+        }
+        asm volatile("cp.async.wait_group 0;" ::: "memory");
+        if (ok && T > 0) hand_over(T - 1);
+        if (!ok) {
+            // gave up: let the gathers still in flight land (bounded) before the CTA's shared memory is released
+            for (int32_t t = issued > NS ? issued - NS : 0; t < issued; ++t) {
+                if (lane == 0 && t == issued - 1) mbar_arrive(kv_full(t % NS));   // its second arrival never came
+                __syncwarp();
+                mbar_drain(kv_full(t % NS), (uint32_t)(t / NS) & 1u, 20000000ll);
+            }
+        }
+    } else {
+        // ------------------------------------------------------------ MMA issuer (the whole warp runs the loop in step)
+        constexpr uint32_t idesc_s = instr_desc(KT, false, false);     // S = Q K^T: both operands K-major
+        constexpr uint32_t idesc_o = instr_desc(D, false, true);       // O += P V: V is MN-major (rows of d values)
+        bool ok = true;
+        auto weighted_values = [&](int32_t u) {                        // O += P_u V_u
+            const int buf = u & 1, s = u % NS;
+            if (!__all_sync(0xffffffffu, mbar_wait(p_full(buf), (uint32_t)(u >> 1) & 1u, &abort_flag))) { ok = false; return; }
+            fence_after_sync();
+            const uint32_t p_op = tmem_base + (uint32_t)(buf * Sh::S_COLS);
+            const uint32_t v_st = stage_base + (uint32_t)s * Sh::STAGE;
+#pragma unroll
+            for (int ks = 0; ks < KT / 16; ++ks) {
+                const uint64_t bd = swizzled_desc(v_st + (uint32_t)ks * 2048u, 1024u, 1024u, 2);
+                mma_bf16_ts(tmem_base + (uint32_t)Sh::O_COL, p_op + (uint32_t)ks * 8u, bd, idesc_o, (u > 0 || ks > 0) ? 1u : 0u);
+            }
+            mma_commit(kv_empty(s));
+            mma_commit(s_free(buf));
+        };
+        for (int32_t t = 0; t < T && ok; ++t) {
+            const int buf = t & 1, s = t % NS;
+            if (!__all_sync(0xffffffffu, mbar_wait(kv_full(s), (uint32_t)(t / NS) & 1u, &abort_flag))) { ok = false; break; }
+            // the score buffer is free once the second product of the tile two back has read its P
+            if (t >= 2 && !__all_sync(0xffffffffu, mbar_wait(s_free(buf), (uint32_t)((t - 2) >> 1) & 1u, &abort_flag))) { ok = false; break; }
+            fence_after_sync();
+            const uint32_t k_st = stage_base + (uint32_t)s * Sh::STAGE + Sh::V_BYTES;
+#pragma unroll
+            for (int k = 0; k < M / 16; ++k) {
+                const uint64_t ad = operand_desc(q_base + (uint32_t)k * 2u * (BQ * 16), BQ * 16, 128);
+                const uint64_t bd = operand_desc(k_st + (uint32_t)k * 2u * (KT * 16), KT * 16, 128);
+                mma_bf16_ss(tmem_base + (uint32_t)(buf * Sh::S_COLS), ad, bd, idesc_s, k > 0 ? 1u : 0u);
+            }
+            mma_commit(s_full(buf));
+            if (t >= 1) weighted_values(t - 1);
+        }
+        if (ok && T > 0) weighted_values(T - 1);
+        if (T > 0) mma_commit(acc_done);
+        if (!ok) {
+            mma_commit(drain_bar);
+            mbar_drain(drain_bar, 0u, 20000000ll);
+        }
+        __syncwarp();
+    }
+
+    fence_before_sync();
+    __syncthreads();
+    if (warp == 5) tmem_dealloc(tmem_base, (uint32_t)Sh::TMEM_COLS);
+    if (tid == 0 && abort_flag) atomicExch(error_word, 1);
+}
+
+}  // namespace
+
+void grf_mask_invalidate(grf_features* feat) { feat->mask.ready = false; }
+
+void grf_mask_release(grf_features* feat)
+{
+    grf_mask_dev& K = feat->mask;
+    grf_buf_release(&K.off); grf_buf_release(&K.cnt); grf_buf_release(&K.key); grf_buf_release(&K.total); grf_buf_release(&K.val);
+    K.ready = false;
+}
+
+extern "C" int grf_features_materialise(grf_ctx* ctx, grf_features* feat)
+{
+    if (!ctx || !feat) return GRF_ERR_INVALID;
+    GRF_CUDA_TRY(cudaSetDevice(ctx->device));
+    grf_mask_dev& K = feat->mask;
+    K.ready = false;
+    const int32_t N = feat->phi.rows, Nk = feat->psi.rows;
+    const size_t words = ((size_t)Nk + 31) / 32;
+    // the values kernel keeps the key bitmap, its prefix counts and the accumulators in shared memory
+    const size_t smem_values = words * 8 + (size_t)MASK_WARPS * MASK_SEG * sizeof(float);
+    if (smem_values > 200 * 1024) return GRF_ERR_TOO_LARGE;
+    GRF_TRY(grf_ensure_block_plan(ctx, feat));
+    if (!feat->plan_ready) return GRF_ERR_TOO_LARGE;          // rows of a block share too little
+    const int32_t nblocks = feat->plan_blocks;
+    GRF_TRY(grf_buf_reserve(&K.cnt, sizeof(int32_t) * 2 * (size_t)nblocks));
+    GRF_TRY(grf_buf_reserve(&K.off, sizeof(int32_t) * ((size_t)nblocks + 1)));
+    GRF_CUDA_TRY(cudaFuncSetAttribute(mask_keys_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(words * 4)));
+    auto keys_pass = [&](int pass) {
+        grf_launch_scope scope(ctx, 7);
+        mask_keys_kernel<<<nblocks, 256, words * 4, ctx->stream>>>(
+            Nk, (const int32_t*)feat->plan_off.ptr, (const int32_t*)feat->plan_cnt.ptr, (const int32_t*)feat->plan_col.ptr,
+            (const int32_t*)feat->psit.rowptr.ptr, (const int32_t*)feat->psit.col.ptr, pass,
+            (const int32_t*)K.off.ptr, (int32_t*)K.cnt.ptr, (int32_t*)K.key.ptr);
+    };
+    keys_pass(0);
+    GRF_CUDA_TRY(cudaGetLastError());
+    GRF_TRY(grf_exclusive_scan(ctx, (const int32_t*)K.cnt.ptr, (int32_t*)K.off.ptr, nblocks, 1));
+    GRF_CUDA_TRY(cudaMemcpyAsync(ctx->pinned + 5, (const int32_t*)K.off.ptr + nblocks, sizeof(int32_t),
+                                 cudaMemcpyDeviceToHost, ctx->stream));
+    GRF_CUDA_TRY(cudaStreamSynchronize(ctx->stream));          // the sizes of the key lists are known only now
+    const int64_t entries = ctx->pinned[5];
+    if (entries < 0) return GRF_ERR_TOO_LARGE;
+    const size_t val_bytes = (size_t)entries * BQ * sizeof(__nv_bfloat16);
+    if (val_bytes > ((size_t)8 << 30)) return GRF_ERR_TOO_LARGE;   // no locality: the S/z route serves this object
+    if (K.key.bytes < (size_t)entries * 4) GRF_TRY(grf_buf_reserve(&K.key, ((size_t)entries + (size_t)entries / 8 + 64) * 4));
+    if (K.val.bytes < val_bytes) GRF_TRY(grf_buf_reserve(&K.val, val_bytes + val_bytes / 8 + 256));
+    keys_pass(1);
+    {
+        grf_launch_scope scope(ctx, 7);
+        mask_order_kernel<<<grf_ceil_div(nblocks, 256), 256, 0, ctx->stream>>>(nblocks, (int32_t*)K.cnt.ptr);
+    }
+    GRF_CUDA_TRY(cudaFuncSetAttribute(mask_values_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_values));
+    {
+        grf_launch_scope scope(ctx, 7);
+        mask_values_kernel<<<nblocks, MASK_WARPS * 32, smem_values, ctx->stream>>>(
+            N, Nk, (const int32_t*)feat->phi.rowptr.ptr, (const int32_t*)feat->phi.col.ptr, (const float*)feat->phi.val.ptr,
+            (const int32_t*)feat->psit.rowptr.ptr, (const int32_t*)feat->psit.col.ptr, (const float*)feat->psit.val.ptr,
+            (const int32_t*)K.off.ptr, (const int32_t*)K.cnt.ptr, (const int32_t*)K.key.ptr, (__nv_bfloat16*)K.val.ptr);
+    }
+    GRF_CUDA_TRY(cudaGetLastError());
+    K.blocks = nblocks;
+    K.entries = entries;
+    K.ready = true;
+    return GRF_OK;
+}
+
+extern "C" int grf_mask_stats(const grf_features* feat, int32_t* blocks, int64_t* key_entries, int64_t* bytes)
+{
+    if (!feat || !feat->mask.ready) return GRF_ERR_INVALID;
+    if (blocks) *blocks = feat->mask.blocks;
+    if (key_entries) *key_entries = feat->mask.entries;
+    if (bytes) *bytes = feat->mask.entries * (int64_t)(BQ * sizeof(__nv_bfloat16) + sizeof(int32_t));
+    return GRF_OK;
+}
+
+extern "C" int grf_mask_rows(grf_ctx* ctx, const grf_features* feat, int32_t n, const int32_t* rows, float* out)
+{
+    if (!ctx || !feat || n <= 0 || !rows || !out) return GRF_ERR_INVALID;
+    if (!feat->mask.ready) return GRF_ERR_INVALID;
+    GRF_CUDA_TRY(cudaSetDevice(ctx->device));
+    const grf_mask_dev& K = feat->mask;
+    {
+        grf_launch_scope scope(ctx, 7);
+        mask_rows_kernel<<<n, 256, 0, ctx->stream>>>(feat->psi.rows, rows, (const int32_t*)K.off.ptr, (const int32_t*)K.cnt.ptr,
+                                                     (const int32_t*)K.key.ptr, (const __nv_bfloat16*)K.val.ptr, out);
+    }
+    return cudaGetLastError() == cudaSuccess ? GRF_OK : GRF_ERR_CUDA;
+}
+
+template <int M>
+static int launch_mhat(grf_ctx* ctx, const grf_features* feat, int32_t G, int32_t N, const void* phiQ, const void* phiK,
+                       const void* V, void* out, float* den_out)
+{
+    using Sh = MhShape<M>;
+    const grf_mask_dev& K = feat->mask;
+    CUtensorMap map_v;
+    if (!grf_make_row_gather_map(&map_v, V, (uint64_t)G * N, 64)) return GRF_ERR_INVALID;
+    // at most two CTAs per SM: each holds half of the SM's tensor memory
+    const size_t smem = Sh::SMEM > 78 * 1024 ? Sh::SMEM : 78 * 1024;
+    GRF_CUDA_TRY(cudaFuncSetAttribute(mhat_attention_kernel<M>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    {
+        grf_launch_scope scope(ctx, 5);
+        mhat_attention_kernel<M><<<(unsigned)K.blocks * (unsigned)G, MH_THREADS, smem, ctx->stream>>>(
+            G, K.blocks, N, (const int32_t*)K.off.ptr, (const int32_t*)K.cnt.ptr, (const int32_t*)K.key.ptr,
+            (const uint4*)K.val.ptr, (const __nv_bfloat16*)phiQ, (const __nv_bfloat16*)phiK, map_v,
+            (__nv_bfloat16*)out, den_out, ctx->error_word);
+    }
+    return cudaGetLastError() == cudaSuccess ? GRF_OK : GRF_ERR_CUDA;
+}
+
+extern "C" int grf_masked_attn_mhat(grf_ctx* ctx, const grf_features* feat, int32_t G, int32_t N, int32_t m, int32_t d,
+                                    int dtype, const void* phiQ, const void* phiK, const void* V, void* out, float* den_out)
+{
+    if (!ctx || !feat || !phiQ || !phiK || !V || !out || G <= 0 || N <= 0) return GRF_ERR_INVALID;
+    if (dtype != GRF_DTYPE_BF16 || d != 64 || (m != 16 && m != 32 && m != 64)) return GRF_ERR_INVALID;
+    if (!feat->mask.ready || feat->phi.rows != N || feat->psi.rows != N) return GRF_ERR_INVALID;
+    if ((int64_t)G * N > 0x7fffffffll || (int64_t)G * feat->mask.blocks > 0x7fffffffll) return GRF_ERR_TOO_LARGE;
+    if (((uintptr_t)phiQ | (uintptr_t)phiK | (uintptr_t)V | (uintptr_t)out) & 15u) return GRF_ERR_INVALID;
+    GRF_CUDA_TRY(cudaSetDevice(ctx->device));
+    if (m == 16) return launch_mhat<16>(ctx, feat, G, N, phiQ, phiK, V, out, den_out);
+    if (m == 32) return launch_mhat<32>(ctx, feat, G, N, phiQ, phiK, V, out, den_out);
+    return launch_mhat<64>(ctx, feat, G, N, phiQ, phiK, V, out, den_out);
+}

@@ -17,96 +17,15 @@
 //                        write the node's record: the tile in the gather kernel's operand layout, then z_l.
 // The summation order over j is fixed by the instruction order (ascending j), so results are reproducible.
 // All mbarrier waits are bounded; a wait that gives up raises the context's error word.
-#include <cuda.h>
-
-#include "grf_internal.cuh"
+#include "tc_common.cuh"
 
 namespace {
 
-constexpr long long WAIT_CYCLES = 4000000000ll;
 constexpr int ITEM_KEYS = 64;        // keys per item = 4 K-steps of 16
 constexpr int NODES_PER_CTA = 64;
 constexpr int ST_THREADS = 288;      // warps 0-3 epilogue, warp 4 MMA issuer, warps 5-8 producers
 
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
-{
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar)
-{
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
-{
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-    return ok != 0;
-}
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag)
-{
-    long long t0 = 0;
-    for (uint32_t it = 0;; ++it) {
-        if (mbar_try_wait(bar, parity)) return true;
-        if ((it & 63u) == 63u) {
-            if (*abort_flag) return false;
-            const long long now = clock64();
-            if (t0 == 0) t0 = now;
-            else if (now - t0 > WAIT_CYCLES) { *abort_flag = 1; return false; }
-        }
-    }
-}
-
-// Unswizzled MN-major operand: 8 (K) x 16-byte core matrices; lbo = bytes between K blocks of 8,
-// sbo = bytes between blocks of 8 along M/N.
-__device__ __forceinline__ uint64_t operand_desc(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes)
-{
-    uint64_t d = (uint64_t)((saddr & 0x3FFFFu) >> 4);
-    d |= (uint64_t)(lbo_bytes >> 4) << 16;
-    d |= (uint64_t)(sbo_bytes >> 4) << 32;
-    d |= (uint64_t)1 << 46;  // descriptor version of this architecture
-    return d;
-}
-// bf16 x bf16 -> fp32, both operands MN-major, M = 128, N = n
-__host__ __device__ constexpr uint32_t instr_desc_mn(int n)
-{
-    return (1u << 4) | (1u << 7) | (1u << 10) | (1u << 15) | (1u << 16) | ((uint32_t)(n >> 3) << 17) |
-           ((uint32_t)(128 >> 4) << 24);
-}
-// The two issuing helpers are called by ALL lanes of a converged warp with the same arguments; elect.sync
-// picks the lane that issues.  (Issued from a branch that only one lane takes, the same instruction costs
-// its thread about three times as many cycles: the operands of tcgen05 instructions are warp-uniform.)
-__device__ __forceinline__ void mma_bf16_ss(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
-                                            uint32_t accumulate)
-{
-    asm volatile(
-        "{\n\t.reg .pred p, q;\n\t"
-        "setp.ne.b32 p, %4, 0;\n\t"
-        "elect.sync _|q, 0xffffffff;\n\t"
-        "@q tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-        ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
-}
-__device__ __forceinline__ void mma_commit(uint32_t bar)
-{
-    asm volatile(
-        "{\n\t.reg .pred q;\n\t"
-        "elect.sync _|q, 0xffffffff;\n\t"
-        "@q tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n\t}"
-        ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16])
-{
-    asm volatile(
-        "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
-        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
-          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
-        : "r"(taddr));
-    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-}
+using namespace grf_tc;
 
 template <int M, int D> struct StShape {
     // Blocks of 8 along M/N sit 144, 160 or 192 bytes apart, not 128: the eight lanes of a quarter warp copy
@@ -128,6 +47,112 @@ template <int M, int D> struct StShape {
     static constexpr size_t SMEM = (size_t)NS * STAGE + 1024;
 };
 
+constexpr long long DRAIN_CYCLES = 20000000ll;   // after an abort: how long a warp waits for its own work in flight
+
+// MMA issuer of both kernels: walks the CTA's nodes in order, item by item; `descs(s, ks, ad, bd)` gives the two
+// operand descriptors of K step ks of stage s.  Barriers are addressed as base + 8 * index.
+template <int M, int NS, int ACC_COLS, class Descs>
+__device__ __forceinline__ void state_mma_issuer(int32_t nnodes, const int32_t* node_beg, uint32_t full0, uint32_t empty0,
+                                                 uint32_t acc_full0, uint32_t acc_free0, uint32_t drain_bar,
+                                                 uint32_t tmem_base, volatile int* abort_flag, Descs descs)
+{
+    constexpr uint32_t idesc = instr_desc(M, true, true);
+    int32_t q = 0;
+    bool ok = true;
+    for (int32_t nn = 0; nn < nnodes && ok; ++nn) {
+        const int32_t c = node_beg[nn + 1] - node_beg[nn];
+        const int32_t nitems = c > 0 ? (c + ITEM_KEYS - 1) / ITEM_KEYS : 1;
+        const int buf = nn & 1;
+        // the accumulator buffer must have been read out by the epilogue of the node two back
+        if (!__all_sync(0xffffffffu, mbar_wait(acc_free0 + 8u * buf, ((uint32_t)(nn >> 1) & 1u) ^ 1u, abort_flag))) { ok = false; break; }
+        const uint32_t acc = tmem_base + (uint32_t)(buf * ACC_COLS);
+        for (int32_t it = 0; it < nitems; ++it, ++q) {
+            const int s = q % NS;
+            const int32_t n = min(ITEM_KEYS, c - it * ITEM_KEYS);
+            const int32_t ksteps = n > 0 ? (n + 15) / 16 : 1;
+            if (!__all_sync(0xffffffffu, mbar_wait(full0 + 8u * s, (uint32_t)(q / NS) & 1u, abort_flag))) { ok = false; break; }
+            fence_after_sync();
+            for (int32_t ks = 0; ks < ksteps; ++ks) {
+                uint64_t ad, bd;
+                descs(s, ks, ad, bd);
+                mma_bf16_ss(acc, ad, bd, idesc, (it > 0 || ks > 0) ? 1u : 0u);
+            }
+            mma_commit(empty0 + 8u * s);
+            if (it == nitems - 1) mma_commit(acc_full0 + 8u * buf);
+        }
+    }
+    if (!ok) {
+        // aborted: the products already issued must have drained before tensor memory is released
+        mma_commit(drain_bar);
+        mbar_drain(drain_bar, 0u, DRAIN_CYCLES);
+    }
+}
+
+// Epilogue of both kernels (warps 0-3): accumulator rows -> the node's record (tile in the gather kernel's operand
+// layout, z_l in fp32 and once more in bf16).
+template <int M, int D, int ACC_COLS>
+__device__ __forceinline__ void state_epilogue(int warp, int lane, int32_t g, int32_t R, int32_t l0, int32_t l1,
+                                               uint32_t acc_full0, uint32_t acc_free0, uint32_t tmem_base,
+                                               volatile int* abort_flag, unsigned char* __restrict__ records)
+{
+    constexpr size_t REC = grf_record_bytes<__nv_bfloat16>(M, D);
+    const int row = warp * 32 + lane;                   // accumulator row = TMEM lane
+    const bool warp_has_rows = warp * 32 <= D;          // S rows 0..D-1 and the z row D
+    int32_t nn = 0;
+    bool ok = true;
+    for (int32_t l = l0; l < l1; ++l, ++nn) {
+        const int buf = nn & 1;
+        if (ok && !mbar_wait(acc_full0 + 8u * buf, (uint32_t)(nn >> 1) & 1u, abort_flag)) ok = false;
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) break;
+        fence_after_sync();
+        if (warp_has_rows) {
+            unsigned char* rec = records + ((size_t)g * R + l) * REC;
+            __nv_bfloat16* tile = reinterpret_cast<__nv_bfloat16*>(rec);
+            float* zl = reinterpret_cast<float*>(rec + (size_t)M * D * 2);
+            const uint32_t taddr = tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)(buf * ACC_COLS);
+#pragma unroll
+            for (int c0 = 0; c0 < M; c0 += 16) {
+                uint32_t r[16];
+                tmem_ld16(taddr + (uint32_t)c0, r);
+                if (row < D) {
+                    // columns c0..c0+15 of row b = feature rows a of column b: two 16-byte chunks of the tile
+#pragma unroll
+                    for (int half = 0; half < 2; ++half) {
+                        uint32_t w[4];
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {
+                            __nv_bfloat162 t2 = __floats2bfloat162_rn(__uint_as_float(r[8 * half + 2 * e]),
+                                                                      __uint_as_float(r[8 * half + 2 * e + 1]));
+                            w[e] = *reinterpret_cast<uint32_t*>(&t2);
+                        }
+                        *reinterpret_cast<uint4*>(tile + grf_tile_index<__nv_bfloat16>(c0 + 8 * half, row, D)) =
+                            make_uint4(w[0], w[1], w[2], w[3]);
+                    }
+                } else if (row == D) {
+#pragma unroll
+                    for (int e = 0; e < 16; e += 4)
+                        *reinterpret_cast<float4*>(zl + c0 + e) = make_float4(__uint_as_float(r[e]), __uint_as_float(r[e + 1]),
+                                                                              __uint_as_float(r[e + 2]), __uint_as_float(r[e + 3]));
+                    // and once more in bf16, for the denominators kernel
+                    uint32_t zw[8];
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) {
+                        __nv_bfloat162 t2 = __floats2bfloat162_rn(__uint_as_float(r[2 * e]), __uint_as_float(r[2 * e + 1]));
+                        zw[e] = *reinterpret_cast<uint32_t*>(&t2);
+                    }
+                    uint4* zb = reinterpret_cast<uint4*>(rec + (size_t)M * D * 2 + (size_t)M * 4 + (size_t)c0 * 2);
+                    zb[0] = make_uint4(zw[0], zw[1], zw[2], zw[3]);
+                    zb[1] = make_uint4(zw[4], zw[5], zw[6], zw[7]);
+                }
+            }
+        }
+        fence_before_sync();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(acc_free0 + 8u * buf);
+    }
+}
+
 template <int M, int D>
 __global__ void __launch_bounds__(ST_THREADS)
 build_states_tc_kernel(int32_t R, int32_t N, const int32_t* __restrict__ t_rowptr, const int32_t* __restrict__ t_col,
@@ -139,7 +164,7 @@ build_states_tc_kernel(int32_t R, int32_t N, const int32_t* __restrict__ t_rowpt
     constexpr int NS = Sh::NS;
     static_assert(D <= 64 && D % 8 == 0 && M % 16 == 0 && M <= 128, "shape not covered by this kernel");
     extern __shared__ unsigned char smem_dyn[];
-    __shared__ __align__(8) unsigned long long bars[2 * NS + 4];   // full, empty per stage; acc_full[2], acc_free[2]
+    __shared__ __align__(8) unsigned long long bars[2 * NS + 5];   // full, empty per stage; acc_full[2], acc_free[2]; drain
     __shared__ uint32_t tmem_slot;
     __shared__ int abort_flag;
     __shared__ int32_t node_beg[NODES_PER_CTA + 1];   // row pointers of the CTA's nodes
@@ -154,10 +179,12 @@ build_states_tc_kernel(int32_t R, int32_t N, const int32_t* __restrict__ t_rowpt
     auto empty = [&](int s) { return bar_base + 8u * (uint32_t)(NS + s); };
     auto acc_full = [&](int b) { return bar_base + 8u * (uint32_t)(2 * NS + b); };
     auto acc_free = [&](int b) { return bar_base + 8u * (uint32_t)(2 * NS + 2 + b); };
+    const uint32_t drain_bar = bar_base + 8u * (uint32_t)(2 * NS + 4);   // used only after an abort
 
     if (tid == 0) {
         for (int s = 0; s < NS; ++s) { mbar_init(full(s), 1); mbar_init(empty(s), 1); }
         for (int b = 0; b < 2; ++b) { mbar_init(acc_full(b), 1); mbar_init(acc_free(b), 4); }
+        mbar_init(drain_bar, 1);
         abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -289,96 +316,16 @@ build_states_tc_kernel(int32_t R, int32_t N, const int32_t* __restrict__ t_rowpt
         }
     } else if (warp == 4) {
         // ------------------------------------------------------------ MMA issuer
-        constexpr uint32_t idesc = instr_desc_mn(M);
-        int32_t q = 0, nn = 0;
-        bool ok = true;
-        for (int32_t l = l0; l < l1 && ok; ++l, ++nn) {
-            const int32_t c = t_rowptr[l + 1] - t_rowptr[l];
-            const int32_t nitems = c > 0 ? (c + ITEM_KEYS - 1) / ITEM_KEYS : 1;
-            const int buf = nn & 1;
-            // the accumulator buffer must have been read out by the epilogue of the node two back
-            if (!__all_sync(0xffffffffu, mbar_wait(acc_free(buf), ((uint32_t)(nn >> 1) & 1u) ^ 1u, &abort_flag))) { ok = false; break; }
-            const uint32_t acc = tmem_base + (uint32_t)(buf * Sh::ACC_COLS);
-            for (int32_t it = 0; it < nitems; ++it, ++q) {
-                const int s = q % NS;
-                const int32_t n = min(ITEM_KEYS, c - it * ITEM_KEYS);
-                const int32_t ksteps = n > 0 ? (n + 15) / 16 : 1;
-                if (!__all_sync(0xffffffffu, mbar_wait(full(s), (uint32_t)(q / NS) & 1u, &abort_flag))) { ok = false; break; }
-                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                const uint32_t a_op = stage_base + (uint32_t)s * Sh::STAGE;
-                const uint32_t b_op = a_op + Sh::A_BYTES;
-                for (int32_t ks = 0; ks < ksteps; ++ks) {
-                    const uint64_t ad = operand_desc(a_op + (uint32_t)ks * Sh::A_KSTEP, Sh::A_LBO, Sh::A_SBO);
-                    const uint64_t bd = operand_desc(b_op + (uint32_t)ks * Sh::B_KSTEP, Sh::B_LBO, Sh::B_SBO);
-                    mma_bf16_ss(acc, ad, bd, idesc, (it > 0 || ks > 0) ? 1u : 0u);
-                }
-                mma_commit(empty(s));
-                if (it == nitems - 1) mma_commit(acc_full(buf));
-            }
-        }
-        if (!ok) {
-            // aborted: let the MMAs already issued drain (bounded) before tensor memory is released
-            const long long t0 = clock64();
-            while (clock64() - t0 < 2000000ll) {}
-        }
+        state_mma_issuer<M, NS, Sh::ACC_COLS>(l1 - l0, node_beg, full(0), empty(0), acc_full(0), acc_free(0), drain_bar,
+                                              tmem_base, &abort_flag,
+                                              [&](int s, int32_t ks, uint64_t& ad, uint64_t& bd) {
+            const uint32_t a_op = stage_base + (uint32_t)s * Sh::STAGE;
+            ad = operand_desc(a_op + (uint32_t)ks * Sh::A_KSTEP, Sh::A_LBO, Sh::A_SBO);
+            bd = operand_desc(a_op + Sh::A_BYTES + (uint32_t)ks * Sh::B_KSTEP, Sh::B_LBO, Sh::B_SBO);
+        });
     } else {
         // ------------------------------------------------------------ epilogue: accumulator -> record
-        constexpr size_t REC = grf_record_bytes<__nv_bfloat16>(M, D);
-        const int row = warp * 32 + lane;                   // accumulator row = TMEM lane
-        const bool warp_has_rows = warp * 32 <= D;          // S rows 0..D-1 and the z row D
-        int32_t nn = 0;
-        bool ok = true;
-        for (int32_t l = l0; l < l1; ++l, ++nn) {
-            const int buf = nn & 1;
-            if (ok && !mbar_wait(acc_full(buf), (uint32_t)(nn >> 1) & 1u, &abort_flag)) ok = false;
-            ok = __all_sync(0xffffffffu, ok);
-            if (!ok) break;
-            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-            if (warp_has_rows) {
-                unsigned char* rec = records + ((size_t)g * R + l) * REC;
-                __nv_bfloat16* tile = reinterpret_cast<__nv_bfloat16*>(rec);
-                float* zl = reinterpret_cast<float*>(rec + (size_t)M * D * 2);
-                const uint32_t taddr = tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)(buf * Sh::ACC_COLS);
-#pragma unroll
-                for (int c0 = 0; c0 < M; c0 += 16) {
-                    uint32_t r[16];
-                    tmem_ld16(taddr + (uint32_t)c0, r);
-                    if (row < D) {
-                        // columns c0..c0+15 of row b = feature rows a of column b: two 16-byte chunks of the tile
-#pragma unroll
-                        for (int half = 0; half < 2; ++half) {
-                            uint32_t w[4];
-#pragma unroll
-                            for (int e = 0; e < 4; ++e) {
-                                __nv_bfloat162 t2 = __floats2bfloat162_rn(__uint_as_float(r[8 * half + 2 * e]),
-                                                                          __uint_as_float(r[8 * half + 2 * e + 1]));
-                                w[e] = *reinterpret_cast<uint32_t*>(&t2);
-                            }
-                            *reinterpret_cast<uint4*>(tile + grf_tile_index<__nv_bfloat16>(c0 + 8 * half, row, D)) =
-                                make_uint4(w[0], w[1], w[2], w[3]);
-                        }
-                    } else if (row == D) {
-#pragma unroll
-                        for (int e = 0; e < 16; e += 4)
-                            *reinterpret_cast<float4*>(zl + c0 + e) = make_float4(__uint_as_float(r[e]), __uint_as_float(r[e + 1]),
-                                                                                  __uint_as_float(r[e + 2]), __uint_as_float(r[e + 3]));
-                        // and once more in bf16, for the denominators kernel
-                        uint32_t zw[8];
-#pragma unroll
-                        for (int e = 0; e < 8; ++e) {
-                            __nv_bfloat162 t2 = __floats2bfloat162_rn(__uint_as_float(r[2 * e]), __uint_as_float(r[2 * e + 1]));
-                            zw[e] = *reinterpret_cast<uint32_t*>(&t2);
-                        }
-                        uint4* zb = reinterpret_cast<uint4*>(rec + (size_t)M * D * 2 + (size_t)M * 4 + (size_t)c0 * 2);
-                        zb[0] = make_uint4(zw[0], zw[1], zw[2], zw[3]);
-                        zb[1] = make_uint4(zw[4], zw[5], zw[6], zw[7]);
-                    }
-                }
-            }
-            asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-            __syncwarp();
-            if (lane == 0) mbar_arrive(acc_free(buf));
-        }
+        state_epilogue<M, D, Sh::ACC_COLS>(warp, lane, g, R, l0, l1, acc_full(0), acc_free(0), tmem_base, &abort_flag, records);
     }
 
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
@@ -432,25 +379,6 @@ template <int M> struct TmaShape {
     static_assert(STAGE % 1024 == 0, "stages must keep the swizzle phase");
 };
 
-__device__ __forceinline__ uint64_t swizzled_desc(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes, uint64_t layout)
-{
-    uint64_t d = (uint64_t)((saddr & 0x3FFFFu) >> 4);
-    d |= (uint64_t)((lbo_bytes >> 4) & 0x3FFFu) << 16;
-    d |= (uint64_t)((sbo_bytes >> 4) & 0x3FFFu) << 32;
-    d |= (uint64_t)1 << 46;
-    d |= layout << 61;
-    return d;
-}
-__device__ __forceinline__ void tma_gather4(uint32_t dst, const CUtensorMap* map, int32_t r0, int32_t r1, int32_t r2,
-                                            int32_t r3, uint32_t bar)
-{
-    asm volatile(
-        "cp.async.bulk.tensor.2d.shared::cluster.global.tile::gather4.mbarrier::complete_tx::bytes"
-        " [%0], [%1, {%2, %3, %4, %5, %6}], [%7];"
-        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(0), "r"(r0), "r"(r1), "r"(r2), "r"(r3), "r"(bar)
-        : "memory");
-}
-
 template <int M>
 __global__ void __launch_bounds__(ST_THREADS)
 build_states_tma_kernel(int32_t R, int32_t N, const int32_t* __restrict__ t_rowptr, const int32_t* __restrict__ t_col,
@@ -461,7 +389,7 @@ build_states_tma_kernel(int32_t R, int32_t N, const int32_t* __restrict__ t_rowp
     using Sh = TmaShape<M>;
     constexpr int NS = Sh::NS, D = Sh::D;
     extern __shared__ unsigned char smem_dyn[];
-    __shared__ __align__(8) unsigned long long bars[3 * NS + 4];   // landed, full, empty per stage; acc_full[2], acc_free[2]
+    __shared__ __align__(8) unsigned long long bars[3 * NS + 5];   // landed, full, empty per stage; acc_full[2], acc_free[2]; drain
     __shared__ uint32_t tmem_slot;
     __shared__ int abort_flag;
     __shared__ int32_t node_beg[NODES_PER_CTA + 1];
@@ -478,10 +406,12 @@ build_states_tma_kernel(int32_t R, int32_t N, const int32_t* __restrict__ t_rowp
     auto empty = [&](int s) { return bar_base + 8u * (uint32_t)(2 * NS + s); };
     auto acc_full = [&](int b) { return bar_base + 8u * (uint32_t)(3 * NS + b); };
     auto acc_free = [&](int b) { return bar_base + 8u * (uint32_t)(3 * NS + 2 + b); };
+    const uint32_t drain_bar = bar_base + 8u * (uint32_t)(3 * NS + 4);   // used only after an abort
 
     if (tid == 0) {
         for (int s = 0; s < NS; ++s) { mbar_init(landed(s), 1); mbar_init(full(s), 1); mbar_init(empty(s), 1); }
         for (int b = 0; b < 2; ++b) { mbar_init(acc_full(b), 1); mbar_init(acc_free(b), 4); }
+        mbar_init(drain_bar, 1);
         abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -595,109 +525,32 @@ build_states_tma_kernel(int32_t R, int32_t N, const int32_t* __restrict__ t_rowp
             }
             if (!mbar_wait(landed(s), use & 1u, &abort_flag)) ok = false;
             ok = __all_sync(0xffffffffu, ok);
-            if (!ok) break;
+            if (!ok) {
+                // gave up with this item's gathers possibly still in flight: let them land (bounded) before the
+                // CTA's shared memory is released
+                mbar_drain(landed(s), use & 1u, DRAIN_CYCLES);
+                break;
+            }
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
             __syncwarp();
             if (lane == 0) mbar_arrive(full(s));
             cur = nxt;
         }
         asm volatile("cp.async.wait_all;" ::: "memory");
-        if (!ok) {
-            // aborted: give copies that may still be in flight time to land before the CTA's memory is released
-            const long long t0 = clock64();
-            while (clock64() - t0 < 2000000ll) {}
-        }
     } else if (warp == 4) {
         // ------------------------------------------------------------ MMA issuer
-        constexpr uint32_t idesc = instr_desc_mn(M);
-        int32_t q = 0, nn = 0;
-        bool ok = true;
-        for (int32_t l = l0; l < l1 && ok; ++l, ++nn) {
-            const int32_t c = node_beg[l - l0 + 1] - node_beg[l - l0];
-            const int32_t nitems = c > 0 ? (c + ITEM_KEYS - 1) / ITEM_KEYS : 1;
-            const int buf = nn & 1;
-            if (!__all_sync(0xffffffffu, mbar_wait(acc_free(buf), ((uint32_t)(nn >> 1) & 1u) ^ 1u, &abort_flag))) { ok = false; break; }
-            const uint32_t acc = tmem_base + (uint32_t)(buf * Sh::ACC_COLS);
-            for (int32_t it = 0; it < nitems; ++it, ++q) {
-                const int s = q % NS;
-                const int32_t n = min(ITEM_KEYS, c - it * ITEM_KEYS);
-                const int32_t ksteps = n > 0 ? (n + 15) / 16 : 1;
-                if (!__all_sync(0xffffffffu, mbar_wait(full(s), (uint32_t)(q / NS) & 1u, &abort_flag))) { ok = false; break; }
-                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                const uint32_t a_op = stage_base + (uint32_t)s * Sh::STAGE;
-                const uint32_t b_op = a_op + Sh::A_BYTES;
-                for (int32_t ks = 0; ks < ksteps; ++ks) {
-                    // A: two atoms along M (gathered rows, then the constant atom), 8-key groups 1024 bytes apart
-                    // (every K step points its second atom at the same constant 2 KB)
-                    const uint64_t ad = swizzled_desc(a_op + (uint32_t)ks * 2048u, const_base - (a_op + (uint32_t)ks * 2048u), 1024u, 2);
-                    const uint64_t bd = operand_desc(b_op + (uint32_t)ks * Sh::B_KSTEP, Sh::B_LBO, Sh::B_SBO);
-                    mma_bf16_ss(acc, ad, bd, idesc, (it > 0 || ks > 0) ? 1u : 0u);
-                }
-                mma_commit(empty(s));
-                if (it == nitems - 1) mma_commit(acc_full(buf));
-            }
-        }
-        if (!ok) {
-            const long long t0 = clock64();
-            while (clock64() - t0 < 2000000ll) {}
-        }
+        state_mma_issuer<M, NS, Sh::ACC_COLS>(l1 - l0, node_beg, full(0), empty(0), acc_full(0), acc_free(0), drain_bar,
+                                              tmem_base, &abort_flag,
+                                              [&](int s, int32_t ks, uint64_t& ad, uint64_t& bd) {
+            // A: two atoms along M (gathered rows, then the constant atom), 8-key groups 1024 bytes apart
+            // (every K step points its second atom at the same constant 2 KB)
+            const uint32_t a_op = stage_base + (uint32_t)s * Sh::STAGE + (uint32_t)ks * 2048u;
+            ad = swizzled_desc(a_op, const_base - a_op, 1024u, 2);
+            bd = operand_desc(stage_base + (uint32_t)s * Sh::STAGE + Sh::A_BYTES + (uint32_t)ks * Sh::B_KSTEP, Sh::B_LBO, Sh::B_SBO);
+        });
     } else {
         // ------------------------------------------------------------ epilogue: accumulator -> record
-        constexpr size_t REC = grf_record_bytes<__nv_bfloat16>(M, D);
-        const int row = warp * 32 + lane;                   // accumulator row = TMEM lane
-        const bool warp_has_rows = warp * 32 <= D;          // S rows 0..D-1 and the z row D
-        int32_t nn = 0;
-        bool ok = true;
-        for (int32_t l = l0; l < l1; ++l, ++nn) {
-            const int buf = nn & 1;
-            if (ok && !mbar_wait(acc_full(buf), (uint32_t)(nn >> 1) & 1u, &abort_flag)) ok = false;
-            ok = __all_sync(0xffffffffu, ok);
-            if (!ok) break;
-            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-            if (warp_has_rows) {
-                unsigned char* rec = records + ((size_t)g * R + l) * REC;
-                __nv_bfloat16* tile = reinterpret_cast<__nv_bfloat16*>(rec);
-                float* zl = reinterpret_cast<float*>(rec + (size_t)M * D * 2);
-                const uint32_t taddr = tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)(buf * Sh::ACC_COLS);
-#pragma unroll
-                for (int c0 = 0; c0 < M; c0 += 16) {
-                    uint32_t r[16];
-                    tmem_ld16(taddr + (uint32_t)c0, r);
-                    if (row < D) {
-#pragma unroll
-                        for (int half = 0; half < 2; ++half) {
-                            uint32_t w[4];
-#pragma unroll
-                            for (int e = 0; e < 4; ++e) {
-                                __nv_bfloat162 t2 = __floats2bfloat162_rn(__uint_as_float(r[8 * half + 2 * e]),
-                                                                          __uint_as_float(r[8 * half + 2 * e + 1]));
-                                w[e] = *reinterpret_cast<uint32_t*>(&t2);
-                            }
-                            *reinterpret_cast<uint4*>(tile + grf_tile_index<__nv_bfloat16>(c0 + 8 * half, row, D)) =
-                                make_uint4(w[0], w[1], w[2], w[3]);
-                        }
-                    } else if (row == D) {
-#pragma unroll
-                        for (int e = 0; e < 16; e += 4)
-                            *reinterpret_cast<float4*>(zl + c0 + e) = make_float4(__uint_as_float(r[e]), __uint_as_float(r[e + 1]),
-                                                                                  __uint_as_float(r[e + 2]), __uint_as_float(r[e + 3]));
-                        // and once more in bf16, for the denominators kernel
-                        uint32_t zw[8];
-#pragma unroll
-                        for (int e = 0; e < 8; ++e) {
-                            __nv_bfloat162 t2 = __floats2bfloat162_rn(__uint_as_float(r[2 * e]), __uint_as_float(r[2 * e + 1]));
-                            zw[e] = *reinterpret_cast<uint32_t*>(&t2);
-                        }
-                        uint4* zb = reinterpret_cast<uint4*>(rec + (size_t)M * D * 2 + (size_t)M * 4 + (size_t)c0 * 2);
-                        zb[0] = make_uint4(zw[0], zw[1], zw[2], zw[3]);
-                        zb[1] = make_uint4(zw[4], zw[5], zw[6], zw[7]);
-                    }
-                }
-            }
-            asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-            __syncwarp();
-            if (lane == 0) mbar_arrive(acc_free(buf));
-        }
+        state_epilogue<M, D, Sh::ACC_COLS>(warp, lane, g, R, l0, l1, acc_full(0), acc_free(0), tmem_base, &abort_flag, records);
     }
 
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
@@ -708,37 +561,6 @@ build_states_tma_kernel(int32_t R, int32_t N, const int32_t* __restrict__ t_rowp
     if (tid == 0 && abort_flag) atomicExch(error_word, 1);
 }
 
-// cuTensorMapEncodeTiled, looked up through the runtime (the library does not link the driver directly)
-typedef CUresult (*encode_tiled_fn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
-                                    const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
-                                    CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-encode_tiled_fn tensor_map_encoder()
-{
-    static encode_tiled_fn fn = []() -> encode_tiled_fn {
-        void* p = nullptr;
-        cudaDriverEntryPointQueryResult qres;
-        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) != cudaSuccess ||
-            qres != cudaDriverEntryPointSuccess)
-            return nullptr;
-        return reinterpret_cast<encode_tiled_fn>(p);
-    }();
-    return fn;
-}
-// A [rows x cols] bf16 matrix whose rows are gathered one at a time (box = one row of at most 64 elements).
-bool make_row_gather_map(CUtensorMap* map, const void* base, uint64_t rows, uint32_t cols)
-{
-    encode_tiled_fn enc = tensor_map_encoder();
-    if (!enc || (reinterpret_cast<uintptr_t>(base) & 15u) != 0) return false;
-    const cuuint64_t dims[2] = {cols, rows};
-    const cuuint64_t strides[1] = {(cuuint64_t)cols * 2};
-    const cuuint32_t box[2] = {cols, 1};
-    const cuuint32_t estr[2] = {1, 1};
-    const CUtensorMapSwizzle sw = cols * 2 == 32 ? CU_TENSOR_MAP_SWIZZLE_32B
-                                : (cols * 2 == 64 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_128B);
-    return enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
-               CU_TENSOR_MAP_INTERLEAVE_NONE, sw, CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
-}
-
 // 1 when the tensor maps cannot be made (the caller then takes the kernel above)
 template <int M>
 int launch_state_tma(grf_ctx* ctx, const grf_csr_dev& psit, int32_t G, int32_t N, const void* phiK, const void* V,
@@ -747,7 +569,7 @@ int launch_state_tma(grf_ctx* ctx, const grf_csr_dev& psit, int32_t G, int32_t N
     using Sh = TmaShape<M>;
     if ((int64_t)G * N > 0x7fffffffll) return 1;
     CUtensorMap map_v;
-    if ((reinterpret_cast<uintptr_t>(phiK) & 15u) != 0 || !make_row_gather_map(&map_v, V, (uint64_t)G * N, 64)) return 1;
+    if ((reinterpret_cast<uintptr_t>(phiK) & 15u) != 0 || !grf_make_row_gather_map(&map_v, V, (uint64_t)G * N, 64)) return 1;
     GRF_CUDA_TRY(cudaFuncSetAttribute(build_states_tma_kernel<M>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Sh::SMEM));
     const dim3 grid(grf_ceil_div(psit.rows, NODES_PER_CTA), G);
     {

@@ -89,10 +89,23 @@ struct grf_kept_walks {
     grf_buf dep_ptr[2], dep_t[2], dep_load[2];
 };
 
+// The mask estimate Mhat = Phi Psi^T held as dense blocks: for every block of GRF_PLAN_BLOCK consecutive rows the
+// sorted list of the keys j that any of its rows reaches (padded to a multiple of GRF_MASK_TILE with the last key
+// and zero values) and the block's values in bf16, laid out [group of 8 keys][row of the block][8 keys].
+#define GRF_MASK_TILE 64
+struct grf_mask_dev {
+    bool ready = false;
+    int32_t blocks = 0;
+    int64_t entries = 0;            // padded key entries over all blocks
+    grf_buf off, cnt, key, total;   // cnt holds [blocks] padded counts, then [blocks] the blocks by decreasing count
+    grf_buf val;
+};
+
 struct grf_features {
     int device = 0;
     grf_csr_dev phi, psi, psit;
     grf_kept_walks kept;
+    grf_mask_dev mask;
     // block plan of Phi: per block of GRF_PLAN_BLOCK rows, the sorted distinct columns
     grf_buf plan_off, plan_cnt, plan_col, plan_total;
     grf_buf plan_coef;              // dense bf16 coefficients [quad of union entries][row of the block][4]
@@ -136,6 +149,9 @@ int grf_build_states_tc(grf_ctx* ctx, const grf_csr_dev& psit, int32_t G, int32_
                         const void* phiK, const void* V, void* records);
 int grf_gather_contract_alu(grf_ctx* ctx, const grf_csr_dev& phi, int32_t G, int32_t N, int32_t m, int32_t d,
                             int dtype, const void* phiQ, const void* records, void* out, float* den_out);
+// attn_mhat.cu
+void grf_mask_invalidate(grf_features* feat);
+void grf_mask_release(grf_features* feat);
 // attn_gather_tc.cu
 int grf_build_block_plan(grf_ctx* ctx, grf_features* feat);
 int grf_ensure_block_plan(grf_ctx* ctx, const grf_features* feat);   // builds it if Phi changed since the last build

@@ -468,6 +468,7 @@ static int sample_into(grf_ctx* ctx, grf_features* feat, const grf_walk_params& 
                                  (float*)feat->psit.val.ptr));
     feat->plan_stale = true;       // the block plan of Phi is built by the first attention call that needs it
     feat->plan_ready = false;
+    grf_mask_invalidate(feat);
     return GRF_OK;
 }
 
@@ -500,7 +501,8 @@ extern "C" int grf_debug_walks(grf_ctx* ctx, int32_t N, const int32_t* rowptr, c
 {
     if (!ctx || !rowptr || !col || !w || !traj || !load) return GRF_ERR_INVALID;
     grf_walk_params P;
-    static const float ones[GRF_MAX_WALK_LEN + 1] = {1.0f};
+    float ones[GRF_MAX_WALK_LEN + 1];
+    for (float& x : ones) x = 1.0f;
     GRF_TRY(grf_walk_params_init(&P, N, seed, n_walks, p_halt, max_len, ones, ones));
     GRF_CUDA_TRY(cudaSetDevice(ctx->device));
     const int64_t total = 2ll * N * n_walks;
@@ -548,5 +550,6 @@ extern "C" int grf_remodulate(grf_ctx* ctx, grf_features* feat, int32_t max_len,
                                  (float*)feat->psit.val.ptr));
     feat->plan_stale = true;       // the coefficient table of the tensor-core gather holds Phi's old values
     feat->plan_ready = false;
+    grf_mask_invalidate(feat);
     return GRF_OK;
 }
