@@ -173,6 +173,7 @@ def run_ours(args):
     g = w.graph()
     N, E = g.N, g.E
     asym = args.route == "asym"
+    mhat = args.route == "mhat"
     if asym:      # Alg. 2: f_phi = alpha, f_psi = delta_0 (no key-side walks contribute, Psi = I)
         f = w.alpha.astype(np.float32)
         f_psi = np.zeros(w.max_len + 1, np.float32); f_psi[0] = 1.0
@@ -194,7 +195,10 @@ def run_ours(args):
     feat = api.Features(ctx, None)
 
     def attention():
-        if asym:
+        if mhat:
+            B.grf_features_materialise(ctx.handle, feat.handle)
+            B.grf_masked_attn_mhat(ctx.handle, feat.handle, w.G, N, w.m, w.d, dt, qd, kd, vd, out, None)
+        elif asym:
             B.grf_masked_attn_asym(ctx.handle, feat.handle, w.G, N, w.m, w.d, dt,
                                    B.GRF_KERNEL_SOFTMAX if args.softmax else B.GRF_KERNEL_LINEAR, qd, kd, vd, out, None)
         else:
@@ -257,7 +261,7 @@ def run_ours(args):
                         f, None, w.G, w.m, w.d, dt, qh, kh, vh, oh)
 
     e2e_ms = float("nan")
-    if not asym:
+    if not asym and not mhat:
         host_step(0)
         barrier()
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -288,18 +292,24 @@ def run_ours(args):
     if rank == 0:
         peak_gbs, peak_kind = peaks()
         alg = algorithmic_bytes(w, N, nnz_phi, nnz_psi, E)
+        if mhat:   # Q, K, V read once, out written once, the mask blocks written once and read once
+            es = 2
+            mblocks, mentries, mbytes = B.grf_mask_stats(feat.handle)
+            alg["mhat_attention"] = w.G * N * (2 * w.m + 2 * w.d) * es + mbytes
+            alg["mask_build"] = mbytes + 2 * (nnz_phi + nnz_psi) * 8
         if asym:   # Q, K, V, Phi read once, out written once; no states
             es = 2 if w.dtype == "bf16" else 4
             alg["gather_contract"] = w.G * N * (2 * w.m + 2 * w.d) * es + nnz_phi * 8 + (N + 1) * 4
         per_kernel = {}
         for name, (ms, n) in ktimes.items():
             per = ms / max(n, 1)
+            a = alg.get(name, 0)
             per_kernel[name] = {"ms_per_step": ms / args.steps, "launch_groups": n,
-                                "algorithmic_gb": alg[name] / 1e9,
-                                "achieved_gbs": alg[name] / 1e9 / (per * 1e-3) if n else None}
+                                "algorithmic_gb": a / 1e9,
+                                "achieved_gbs": a / 1e9 / (per * 1e-3) if n else None}
         dom = max(ktimes, key=lambda kname: ktimes[kname][0])
         dom_ms = ktimes[dom][0] / max(ktimes[dom][1], 1)
-        achieved = alg[dom] / 1e9 / (dom_ms * 1e-3)
+        achieved = alg.get(dom, 0) / 1e9 / (dom_ms * 1e-3)
         result = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": total_ms / args.steps, "higher_is_better": True,
@@ -311,16 +321,18 @@ def run_ours(args):
                        "l2": "256 MiB flush write between steps, outside the per-step events",
                        "step": ("grf_sample (f_psi = delta_0) + grf_masked_attn_asym (Alg. 2, %s similarity), features "
                                 "resampled every step" % ("softmax" if args.softmax else "linear")) if asym else
+                               ("grf_sample (both ensembles) + grf_features_materialise + grf_masked_attn_mhat, features "
+                                "resampled and the mask rebuilt every step") if mhat else
                                "grf_sample (both ensembles) + grf_masked_linear_attn, features resampled every step"},
             "clocks": clocks,
             "gpu_launches": launches,
-            "e2e": None if asym else
+            "e2e": None if (asym or mhat) else
                    {"value": tokens_per_step / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
                     "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms, "entry_point": "grf_step_host"},
             "roofline": {"kernel": dom, "bound": "hbm", "achieved": achieved, "peak": peak_gbs, "unit": "GB/s",
                          "frac": achieved / peak_gbs, "peak_source": peak_kind,
-                         "traffic": None if asym else NCU_TRAFFIC_BYTES.get(w.name, {}).get(dom),
-                         "algorithmic_bytes": alg[dom], "ms_per_launch": dom_ms},
+                         "traffic": None if (asym or mhat) else NCU_TRAFFIC_BYTES.get(w.name, {}).get(dom),
+                         "algorithmic_bytes": alg.get(dom, 0), "ms_per_launch": dom_ms},
             "phases": {"sample_ms": statistics.mean(sample_ms), "attn_ms": statistics.mean(attn_ms),
                        "sample_ms_min_med_max": [min(sample_ms), statistics.median(sample_ms), max(sample_ms)],
                        "attn_ms_min_med_max": [min(attn_ms), statistics.median(attn_ms), max(attn_ms)],
@@ -392,7 +404,7 @@ def main():
     ap.add_argument("--workload", default="pc32768")
     ap.add_argument("--cpu-heads", type=int, default=1, help="problems of the batch the CPU baseline really runs")
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--route", choices=["sz", "asym"], default="sz",
+    ap.add_argument("--route", choices=["sz", "asym", "mhat"], default="sz",
                     help="sz: Alg. 1 (per-node states, the default); asym: Alg. 2 (asymmetric features, Psi = I), "
                          "a variant outside the headline metric, no end-to-end leg")
     ap.add_argument("--softmax", action="store_true", help="with --route asym: A_ij = exp(q_i . k_j)")

@@ -264,8 +264,9 @@ int64_t grf_ctx_launch_count(const grf_ctx* ctx);
  * the elapsed times since the previous read to ms[GRF_KERNEL_CLASSES] / launches[GRF_KERNEL_CLASSES]
  * (HOST arrays, overwritten) and clears the record.  Classes: 0 walk+merge, 1 prefix scans, 2 row
  * compaction, 3 column regrouping (histogram, scatter, ordering), 4 state build (S, z), 5 gather-contract,
- * 6 denominators pass of the tensor-core gather, 7 block plan of the tensor-core gather. */
-#define GRF_KERNEL_CLASSES 8
+ * 6 denominators pass of the tensor-core gather, 7 block plan of the tensor-core gather, 8 building the
+ * materialised mask, 9 attention over the materialised mask. */
+#define GRF_KERNEL_CLASSES 10
 int grf_ctx_enable_timing(grf_ctx* ctx, int enable);
 int grf_ctx_kernel_times(grf_ctx* ctx, float* ms, int64_t* launches);
 

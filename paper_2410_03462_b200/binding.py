@@ -127,7 +127,7 @@ def grf_ctx_use_tensor_cores(ctx: int, enable: bool):
 
 
 KERNEL_CLASSES = ("walk_merge", "scan", "compact", "regroup", "build_states", "gather_contract", "row_denominators",
-                  "block_plan")
+                  "block_plan", "mask_build", "mhat_attention")
 
 
 def grf_ctx_enable_timing(ctx: int, enable: bool):

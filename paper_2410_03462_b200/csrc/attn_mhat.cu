@@ -27,18 +27,17 @@ constexpr int BQ = GRF_PLAN_BLOCK;      // queries per block
 constexpr int KT = GRF_MASK_TILE;       // keys per tile
 
 // ---------------------------------------------------------------------------------------------------
-// Key lists: one CTA per block of rows.  Two passes: pass 0 counts (the counts, padded to whole tiles, are then
-// scanned into offsets), pass 1 writes the sorted lists.
+// Key sets: one CTA per block of rows marks, in a bitmap, the keys of Psi^T's rows over the block's node list.
+// A warp takes 32 nodes at a time (lane x holds node x's extent in Psi^T) and fetches the keys of four nodes
+// together, so that several loads are in flight.  The bitmap and the count (padded to whole tiles) are kept.
 
 __global__ void __launch_bounds__(256)
-mask_keys_kernel(int32_t Nk, const int32_t* __restrict__ plan_off, const int32_t* __restrict__ plan_cnt,
-                 const int32_t* __restrict__ plan_col, const int32_t* __restrict__ t_rowptr,
-                 const int32_t* __restrict__ t_col, int pass, const int32_t* __restrict__ mk_off,
-                 int32_t* __restrict__ mk_cnt, int32_t* __restrict__ mk_key)
+mask_bitmap_kernel(int32_t Nk, const int32_t* __restrict__ plan_off, const int32_t* __restrict__ plan_cnt,
+                   const int32_t* __restrict__ plan_col, const int32_t* __restrict__ t_rowptr,
+                   const int32_t* __restrict__ t_col, uint32_t* __restrict__ bits, int32_t* __restrict__ mk_cnt)
 {
     extern __shared__ uint32_t bitmap[];        // one bit per key
     __shared__ int32_t warp_sums[8];
-    __shared__ int32_t block_total;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int32_t blk = blockIdx.x;
     const int32_t words = (Nk + 31) >> 5;
@@ -46,14 +45,74 @@ mask_keys_kernel(int32_t Nk, const int32_t* __restrict__ plan_off, const int32_t
     __syncthreads();
     const int32_t* ulist = plan_col + plan_off[blk];
     const int32_t ucnt = plan_cnt[blk];
-    for (int32_t u = warp; u < ucnt; u += 8) {
-        const int32_t l = ulist[u];
-        for (int32_t p = t_rowptr[l] + lane; p < t_rowptr[l + 1]; p += 32) {
-            const int32_t j = t_col[p];
-            atomicOr(&bitmap[j >> 5], 1u << (j & 31));
+    for (int32_t u0 = warp * 32; u0 < ucnt; u0 += 8 * 32) {
+        const int32_t n = min(32, ucnt - u0);
+        const int32_t my_l = lane < n ? __ldg(ulist + u0 + lane) : 0;
+        const int32_t my_beg = lane < n ? __ldg(t_rowptr + my_l) : 0;
+        const int32_t my_end = lane < n ? __ldg(t_rowptr + my_l + 1) : 0;
+        for (int32_t e0 = 0; e0 < n; e0 += 4) {
+            int32_t jj[4][4];
+            int32_t ebeg[4], eend[4];
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                ebeg[e] = e0 + e < n ? __shfl_sync(0xffffffffu, my_beg, (e0 + e) & 31) : 0;
+                eend[e] = e0 + e < n ? __shfl_sync(0xffffffffu, my_end, (e0 + e) & 31) : 0;
+#pragma unroll
+                for (int sl = 0; sl < 4; ++sl) {
+                    const int32_t q = ebeg[e] + sl * 32 + lane;
+                    jj[e][sl] = q < eend[e] ? __ldg(t_col + q) : -1;
+                }
+            }
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+#pragma unroll
+                for (int sl = 0; sl < 4; ++sl)
+                    if (jj[e][sl] >= 0) atomicOr(&bitmap[jj[e][sl] >> 5], 1u << (jj[e][sl] & 31));
+                for (int32_t q = ebeg[e] + 128 + lane; q < eend[e]; q += 32) {
+                    const int32_t j = __ldg(t_col + q);
+                    atomicOr(&bitmap[j >> 5], 1u << (j & 31));
+                }
+            }
         }
     }
     __syncthreads();
+    // the bitmap, and behind it the number of set bits before each of its words
+    const int32_t per = (words + 255) / 256;
+    const int32_t w0 = min(words, tid * per), w1 = min(words, w0 + per);
+    int32_t mine = 0;
+    for (int32_t x = w0; x < w1; ++x) mine += __popc(bitmap[x]);
+    int32_t inc = mine;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const int32_t y = __shfl_up_sync(0xffffffffu, inc, o);
+        if (lane >= o) inc += y;
+    }
+    if (lane == 31) warp_sums[warp] = inc;
+    __syncthreads();
+    int32_t run = inc - mine;
+    for (int w = 0; w < warp; ++w) run += warp_sums[w];
+    uint32_t* dst = bits + (size_t)blk * 2 * words;
+    for (int32_t x = w0; x < w1; ++x) {
+        const uint32_t b = bitmap[x];
+        dst[x] = b;
+        dst[words + x] = (uint32_t)run;
+        run += __popc(b);
+    }
+    if (tid == 255) mk_cnt[blk] = (run + KT - 1) / KT * KT;
+}
+
+// Key lists: the set bits of a block's bitmap in ascending order, padded to whole tiles with the last key
+// (whose mask values in the padding are zeros).
+__global__ void __launch_bounds__(256)
+mask_list_kernel(int32_t Nk, const uint32_t* __restrict__ bits, const int32_t* __restrict__ mk_off,
+                 const int32_t* __restrict__ mk_cnt, int32_t* __restrict__ mk_key)
+{
+    __shared__ int32_t warp_sums[8];
+    __shared__ int32_t block_total;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int32_t blk = blockIdx.x;
+    const int32_t words = (Nk + 31) >> 5;
+    const uint32_t* bitmap = bits + (size_t)blk * 2 * words;
     // each thread owns a contiguous range of words so that the list comes out sorted
     const int32_t per = (words + 255) / 256;
     const int32_t w0 = min(words, tid * per), w1 = min(words, w0 + per);
@@ -69,25 +128,19 @@ mask_keys_kernel(int32_t Nk, const int32_t* __restrict__ plan_off, const int32_t
     __syncthreads();
     int32_t before = inc - mine;
     for (int w = 0; w < warp; ++w) before += warp_sums[w];
-    if (tid == 255) {
-        block_total = before + mine;
-        if (pass == 0) mk_cnt[blk] = (block_total + KT - 1) / KT * KT;
-    }
-    if (pass == 0) return;
-    __syncthreads();
+    if (tid == 255) block_total = before + mine;
     const int32_t base_off = mk_off[blk];
     int32_t o = base_off + before;
     for (int32_t x = w0; x < w1; ++x) {
-        uint32_t bits = bitmap[x];
-        while (bits) {
-            const int b = __ffs(bits) - 1;
-            bits &= bits - 1;
-            mk_key[o++] = (x << 5) + b;
+        uint32_t b = bitmap[x];
+        while (b) {
+            const int k = __ffs(b) - 1;
+            b &= b - 1;
+            mk_key[o++] = (x << 5) + k;
         }
     }
     __syncthreads();
-    // padding: the last key again (its mask values are zeros)
-    const int32_t padded = (block_total + KT - 1) / KT * KT;
+    const int32_t padded = mk_cnt[blk];
     if (block_total > 0)
         for (int32_t e = block_total + tid; e < padded; e += 256) mk_key[base_off + e] = mk_key[base_off + block_total - 1];
 }
@@ -108,85 +161,130 @@ __global__ void __launch_bounds__(256) mask_order_kernel(int32_t nblocks, int32_
 
 // ---------------------------------------------------------------------------------------------------
 // Mask values: Mhat_ij = sum_l Phi_il Psi_jl for the rows i of one block and the keys j of its list.
-// One CTA per block, one warp per row at a time.  The warp keeps the row's accumulators (fp32, one per key of a
-// segment of the list) in shared memory; for every non-zero Phi_il, taken in ascending l, its lanes add
-// Phi_il * Psi_jl at the position of key j, found from a bitmap of the block's keys and the number of set bits
-// before each bitmap word.  Keys of one l are distinct, so no two lanes meet at one position, and the warp is
-// synchronised between two l: the order of every sum is fixed.  Lists longer than a segment take further passes.
+// A CTA takes MASK_ROWS rows of one block (the blocks with the longest key lists first), one warp per row at a
+// time.  The warp keeps the row's accumulators (fp32, one per key of a segment of the list) in shared memory; for
+// every non-zero Phi_il, taken in ascending l, its lanes add Phi_il * Psi_jl at the position of key j, found from
+// the bitmap of the block's keys and the number of set bits before each bitmap word.  Keys of one l are distinct,
+// so no two lanes meet at one position, and the warp is synchronised between two l: the order of every sum is
+// fixed.  The keys of four nodes are fetched together and the next four are on their way while these are added.
+// Lists longer than a segment take further passes.
 
 constexpr int MASK_SEG = 4096;          // accumulators per warp
-constexpr int MASK_WARPS = 8;
+constexpr int MASK_WARPS = 4;
+constexpr int MASK_ROWS = 8;            // rows of a block per CTA
+
+struct MaskGroup {                      // the keys of four nodes l, up to 128 each: lane x holds keys x, x+32, x+64, x+96
+    int32_t j[4][4];
+    float v[4][4];
+    int32_t beg[4], end[4];
+};
 
 __global__ void __launch_bounds__(MASK_WARPS * 32)
 mask_values_kernel(int32_t N, int32_t Nk, const int32_t* __restrict__ phi_rowptr, const int32_t* __restrict__ phi_col,
                    const float* __restrict__ phi_val, const int32_t* __restrict__ t_rowptr,
                    const int32_t* __restrict__ t_col, const float* __restrict__ t_val,
                    const int32_t* __restrict__ mk_off, const int32_t* __restrict__ mk_cnt,
-                   const int32_t* __restrict__ mk_key, __nv_bfloat16* __restrict__ mk_val)
+                   const uint32_t* __restrict__ bits, __nv_bfloat16* __restrict__ mk_val)
 {
     extern __shared__ uint32_t smem_mask[];     // bitmap, set bits before each word, accumulators
-    __shared__ int32_t warp_sums[MASK_WARPS];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int32_t blk = blockIdx.x;
+    constexpr int GROUPS = BQ / MASK_ROWS;
+    const int32_t nblocks = (N + BQ - 1) / BQ;
+    const int32_t blk = mk_cnt[nblocks + blockIdx.x / GROUPS];     // blocks by decreasing key count
+    const int32_t rg = blockIdx.x % GROUPS;
     const int32_t words = (Nk + 31) >> 5;
+    const int32_t words_al = (words + 1) & ~1;
     uint32_t* bitmap = smem_mask;
-    int32_t* before_word = reinterpret_cast<int32_t*>(smem_mask + words);
-    float* acc = reinterpret_cast<float*>(smem_mask + 2 * (size_t)words) + (size_t)warp * MASK_SEG;
+    int32_t* before_word = reinterpret_cast<int32_t*>(smem_mask + words_al);
+    // (the accumulators are read as float4: they start at a multiple of 16 bytes)
+    float* acc = reinterpret_cast<float*>(smem_mask + 2 * (size_t)words_al) + (size_t)warp * MASK_SEG;
     const int32_t off = mk_off[blk], cnt = mk_cnt[blk];
-    for (int32_t x = tid; x < words; x += MASK_WARPS * 32) bitmap[x] = 0u;
-    __syncthreads();
-    for (int32_t e = tid; e < cnt; e += MASK_WARPS * 32) {
-        const int32_t j = mk_key[off + e];
-        atomicOr(&bitmap[j >> 5], 1u << (j & 31));
+    // the block's bitmap and prefix counts as the key-set kernel left them
+    const uint32_t* src = bits + (size_t)blk * 2 * words;
+    for (int32_t x = tid; x < words; x += MASK_WARPS * 32) {
+        bitmap[x] = src[x];
+        before_word[x] = (int32_t)src[words + x];
     }
-    __syncthreads();
-    {
-        const int32_t per = (words + MASK_WARPS * 32 - 1) / (MASK_WARPS * 32);
-        const int32_t w0 = min(words, tid * per), w1 = min(words, w0 + per);
-        int32_t mine = 0;
-        for (int32_t x = w0; x < w1; ++x) mine += __popc(bitmap[x]);
-        int32_t inc = mine;
-#pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-            const int32_t y = __shfl_up_sync(0xffffffffu, inc, o);
-            if (lane >= o) inc += y;
-        }
-        if (lane == 31) warp_sums[warp] = inc;
-        __syncthreads();
-        int32_t run = inc - mine;
-        for (int w = 0; w < warp; ++w) run += warp_sums[w];
-        for (int32_t x = w0; x < w1; ++x) { before_word[x] = run; run += __popc(bitmap[x]); }
-    }
+    for (int32_t x = lane; x < MASK_SEG; x += 32) acc[x] = 0.0f;
     __syncthreads();
     const int32_t r0 = blk * BQ;
     for (int32_t seg0 = 0; seg0 < cnt; seg0 += MASK_SEG) {
         const int32_t seglen = min(MASK_SEG, cnt - seg0);       // a multiple of the tile, hence of 8
-        for (int32_t rr = warp; rr < BQ; rr += MASK_WARPS) {
+        auto position = [&](int32_t j) {
+            const int32_t ps = before_word[j >> 5] + __popc(bitmap[j >> 5] & ((1u << (j & 31)) - 1u)) - seg0;
+            return (ps >= 0 && ps < seglen) ? ps : -1;
+        };
+        for (int32_t rr = rg * MASK_ROWS + warp; rr < (rg + 1) * MASK_ROWS; rr += MASK_WARPS) {
             const int32_t r = r0 + rr;
-            for (int32_t x = lane; x < seglen; x += 32) acc[x] = 0.0f;
-            __syncwarp();
             if (r < N) {
-                for (int32_t p = phi_rowptr[r]; p < phi_rowptr[r + 1]; ++p) {
-                    const int32_t l = __ldg(phi_col + p);
-                    const float phi = __ldg(phi_val + p);
-                    for (int32_t q = __ldg(t_rowptr + l) + lane; q < __ldg(t_rowptr + l + 1); q += 32) {
-                        const int32_t j = __ldg(t_col + q);
-                        const int32_t pos = before_word[j >> 5] + __popc(bitmap[j >> 5] & ((1u << (j & 31)) - 1u)) - seg0;
-                        if (pos >= 0 && pos < seglen) acc[pos] = fmaf(phi, __ldg(t_val + q), acc[pos]);
+                const int32_t pbeg = phi_rowptr[r], pend = phi_rowptr[r + 1];
+                for (int32_t p0 = pbeg; p0 < pend; p0 += 32) {
+                    // 32 non-zeros of the row at a time: lane x holds node l_x, Phi_il and the extent of row l_x of Psi^T
+                    const int32_t n = min(32, pend - p0);
+                    const int32_t my_l = lane < n ? __ldg(phi_col + p0 + lane) : 0;
+                    const float my_phi = lane < n ? __ldg(phi_val + p0 + lane) : 0.0f;
+                    const int32_t my_beg = lane < n ? __ldg(t_rowptr + my_l) : 0;
+                    const int32_t my_end = lane < n ? __ldg(t_rowptr + my_l + 1) : 0;
+                    auto fetch = [&](int32_t e0, MaskGroup& gq) {
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {
+                            gq.beg[e] = e0 + e < n ? __shfl_sync(0xffffffffu, my_beg, (e0 + e) & 31) : 0;
+                            gq.end[e] = e0 + e < n ? __shfl_sync(0xffffffffu, my_end, (e0 + e) & 31) : 0;
+#pragma unroll
+                            for (int sl = 0; sl < 4; ++sl) {
+                                const int32_t q = gq.beg[e] + sl * 32 + lane;
+                                const bool valid = q < gq.end[e];
+                                gq.j[e][sl] = valid ? __ldg(t_col + q) : -1;
+                                gq.v[e][sl] = valid ? __ldg(t_val + q) : 0.0f;
+                            }
+                        }
+                    };
+                    auto add = [&](int32_t e0, MaskGroup& gq) {
+#pragma unroll
+                        for (int e = 0; e < 4; ++e)
+#pragma unroll
+                            for (int sl = 0; sl < 4; ++sl) gq.j[e][sl] = gq.j[e][sl] >= 0 ? position(gq.j[e][sl]) : -1;
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {
+                            const float phi = __shfl_sync(0xffffffffu, my_phi, (e0 + e) & 31);
+                            float a[4];
+                            // one node's keys are distinct: a lane's four additions go side by side
+#pragma unroll
+                            for (int sl = 0; sl < 4; ++sl) a[sl] = gq.j[e][sl] >= 0 ? acc[gq.j[e][sl]] : 0.0f;
+#pragma unroll
+                            for (int sl = 0; sl < 4; ++sl)
+                                if (gq.j[e][sl] >= 0) acc[gq.j[e][sl]] = fmaf(phi, gq.v[e][sl], a[sl]);
+                            for (int32_t q = gq.beg[e] + 128 + lane; q < gq.end[e]; q += 32) {   // nodes with more than 128 keys
+                                const int32_t ps = position(__ldg(t_col + q));
+                                if (ps >= 0) acc[ps] = fmaf(phi, __ldg(t_val + q), acc[ps]);
+                            }
+                            __syncwarp();
+                        }
+                    };
+                    MaskGroup ga, gb;
+                    fetch(0, ga);
+                    for (int32_t e0 = 0; e0 < n; e0 += 8) {
+                        if (e0 + 4 < n) fetch(e0 + 4, gb);
+                        add(e0, ga);
+                        if (e0 + 4 < n) {
+                            if (e0 + 8 < n) fetch(e0 + 8, ga);
+                            add(e0 + 4, gb);
+                        }
                     }
-                    __syncwarp();
                 }
             }
-            // the row's values of this segment, eight keys (16 bytes) per lane at a time
+            // the row's values of this segment, eight keys (16 bytes) per lane at a time; the accumulators are
+            // cleared for the next row as they are read
             for (int32_t c8 = lane; c8 < seglen / 8; c8 += 32) {
-                uint32_t w[4];
-#pragma unroll
-                for (int e = 0; e < 4; ++e) {
-                    const __nv_bfloat162 h = __floats2bfloat162_rn(acc[c8 * 8 + 2 * e], acc[c8 * 8 + 2 * e + 1]);
-                    w[e] = *reinterpret_cast<const uint32_t*>(&h);
-                }
+                float4* a4 = reinterpret_cast<float4*>(acc + c8 * 8);
+                const float4 x0 = a4[0], x1 = a4[1];
+                a4[0] = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+                a4[1] = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+                const __nv_bfloat162 h0 = __floats2bfloat162_rn(x0.x, x0.y), h1 = __floats2bfloat162_rn(x0.z, x0.w);
+                const __nv_bfloat162 h2 = __floats2bfloat162_rn(x1.x, x1.y), h3 = __floats2bfloat162_rn(x1.z, x1.w);
                 uint4* dst = reinterpret_cast<uint4*>(mk_val + ((size_t)((off + seg0) / 8 + c8) * BQ + rr) * 8);
-                *dst = make_uint4(w[0], w[1], w[2], w[3]);
+                *dst = make_uint4(*reinterpret_cast<const uint32_t*>(&h0), *reinterpret_cast<const uint32_t*>(&h1),
+                                  *reinterpret_cast<const uint32_t*>(&h2), *reinterpret_cast<const uint32_t*>(&h3));
             }
             __syncwarp();
         }
@@ -481,7 +579,7 @@ void grf_mask_invalidate(grf_features* feat) { feat->mask.ready = false; }
 void grf_mask_release(grf_features* feat)
 {
     grf_mask_dev& K = feat->mask;
-    grf_buf_release(&K.off); grf_buf_release(&K.cnt); grf_buf_release(&K.key); grf_buf_release(&K.total); grf_buf_release(&K.val);
+    grf_buf_release(&K.off); grf_buf_release(&K.cnt); grf_buf_release(&K.key); grf_buf_release(&K.bits); grf_buf_release(&K.val);
     K.ready = false;
 }
 
@@ -494,22 +592,22 @@ extern "C" int grf_features_materialise(grf_ctx* ctx, grf_features* feat)
     const int32_t N = feat->phi.rows, Nk = feat->psi.rows;
     const size_t words = ((size_t)Nk + 31) / 32;
     // the values kernel keeps the key bitmap, its prefix counts and the accumulators in shared memory
-    const size_t smem_values = words * 8 + (size_t)MASK_WARPS * MASK_SEG * sizeof(float);
+    const size_t smem_values = ((words + 1) & ~(size_t)1) * 8 + (size_t)MASK_WARPS * MASK_SEG * sizeof(float);
     if (smem_values > 200 * 1024) return GRF_ERR_TOO_LARGE;
     GRF_TRY(grf_ensure_block_plan(ctx, feat));
     if (!feat->plan_ready) return GRF_ERR_TOO_LARGE;          // rows of a block share too little
     const int32_t nblocks = feat->plan_blocks;
     GRF_TRY(grf_buf_reserve(&K.cnt, sizeof(int32_t) * 2 * (size_t)nblocks));
     GRF_TRY(grf_buf_reserve(&K.off, sizeof(int32_t) * ((size_t)nblocks + 1)));
-    GRF_CUDA_TRY(cudaFuncSetAttribute(mask_keys_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(words * 4)));
-    auto keys_pass = [&](int pass) {
-        grf_launch_scope scope(ctx, 7);
-        mask_keys_kernel<<<nblocks, 256, words * 4, ctx->stream>>>(
+    GRF_TRY(grf_buf_reserve(&K.bits, sizeof(uint32_t) * 2 * (size_t)nblocks * words));
+    GRF_CUDA_TRY(cudaFuncSetAttribute(mask_bitmap_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(words * 4)));
+    {
+        grf_launch_scope scope(ctx, 8);
+        mask_bitmap_kernel<<<nblocks, 256, words * 4, ctx->stream>>>(
             Nk, (const int32_t*)feat->plan_off.ptr, (const int32_t*)feat->plan_cnt.ptr, (const int32_t*)feat->plan_col.ptr,
-            (const int32_t*)feat->psit.rowptr.ptr, (const int32_t*)feat->psit.col.ptr, pass,
-            (const int32_t*)K.off.ptr, (int32_t*)K.cnt.ptr, (int32_t*)K.key.ptr);
-    };
-    keys_pass(0);
+            (const int32_t*)feat->psit.rowptr.ptr, (const int32_t*)feat->psit.col.ptr, (uint32_t*)K.bits.ptr,
+            (int32_t*)K.cnt.ptr);
+    }
     GRF_CUDA_TRY(cudaGetLastError());
     GRF_TRY(grf_exclusive_scan(ctx, (const int32_t*)K.cnt.ptr, (int32_t*)K.off.ptr, nblocks, 1));
     GRF_CUDA_TRY(cudaMemcpyAsync(ctx->pinned + 5, (const int32_t*)K.off.ptr + nblocks, sizeof(int32_t),
@@ -521,18 +619,22 @@ extern "C" int grf_features_materialise(grf_ctx* ctx, grf_features* feat)
     if (val_bytes > ((size_t)8 << 30)) return GRF_ERR_TOO_LARGE;   // no locality: the S/z route serves this object
     if (K.key.bytes < (size_t)entries * 4) GRF_TRY(grf_buf_reserve(&K.key, ((size_t)entries + (size_t)entries / 8 + 64) * 4));
     if (K.val.bytes < val_bytes) GRF_TRY(grf_buf_reserve(&K.val, val_bytes + val_bytes / 8 + 256));
-    keys_pass(1);
     {
-        grf_launch_scope scope(ctx, 7);
+        grf_launch_scope scope(ctx, 8);
+        mask_list_kernel<<<nblocks, 256, 0, ctx->stream>>>(Nk, (const uint32_t*)K.bits.ptr, (const int32_t*)K.off.ptr,
+                                                           (const int32_t*)K.cnt.ptr, (int32_t*)K.key.ptr);
+    }
+    {
+        grf_launch_scope scope(ctx, 8);
         mask_order_kernel<<<grf_ceil_div(nblocks, 256), 256, 0, ctx->stream>>>(nblocks, (int32_t*)K.cnt.ptr);
     }
     GRF_CUDA_TRY(cudaFuncSetAttribute(mask_values_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_values));
     {
-        grf_launch_scope scope(ctx, 7);
-        mask_values_kernel<<<nblocks, MASK_WARPS * 32, smem_values, ctx->stream>>>(
+        grf_launch_scope scope(ctx, 8);
+        mask_values_kernel<<<nblocks * (BQ / MASK_ROWS), MASK_WARPS * 32, smem_values, ctx->stream>>>(
             N, Nk, (const int32_t*)feat->phi.rowptr.ptr, (const int32_t*)feat->phi.col.ptr, (const float*)feat->phi.val.ptr,
             (const int32_t*)feat->psit.rowptr.ptr, (const int32_t*)feat->psit.col.ptr, (const float*)feat->psit.val.ptr,
-            (const int32_t*)K.off.ptr, (const int32_t*)K.cnt.ptr, (const int32_t*)K.key.ptr, (__nv_bfloat16*)K.val.ptr);
+            (const int32_t*)K.off.ptr, (const int32_t*)K.cnt.ptr, (const uint32_t*)K.bits.ptr, (__nv_bfloat16*)K.val.ptr);
     }
     GRF_CUDA_TRY(cudaGetLastError());
     K.blocks = nblocks;
@@ -557,7 +659,7 @@ extern "C" int grf_mask_rows(grf_ctx* ctx, const grf_features* feat, int32_t n, 
     GRF_CUDA_TRY(cudaSetDevice(ctx->device));
     const grf_mask_dev& K = feat->mask;
     {
-        grf_launch_scope scope(ctx, 7);
+        grf_launch_scope scope(ctx, 8);
         mask_rows_kernel<<<n, 256, 0, ctx->stream>>>(feat->psi.rows, rows, (const int32_t*)K.off.ptr, (const int32_t*)K.cnt.ptr,
                                                      (const int32_t*)K.key.ptr, (const __nv_bfloat16*)K.val.ptr, out);
     }
@@ -576,7 +678,7 @@ static int launch_mhat(grf_ctx* ctx, const grf_features* feat, int32_t G, int32_
     const size_t smem = Sh::SMEM > 78 * 1024 ? Sh::SMEM : 78 * 1024;
     GRF_CUDA_TRY(cudaFuncSetAttribute(mhat_attention_kernel<M>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     {
-        grf_launch_scope scope(ctx, 5);
+        grf_launch_scope scope(ctx, 9);
         mhat_attention_kernel<M><<<(unsigned)K.blocks * (unsigned)G, MH_THREADS, smem, ctx->stream>>>(
             G, K.blocks, N, (const int32_t*)K.off.ptr, (const int32_t*)K.cnt.ptr, (const int32_t*)K.key.ptr,
             (const uint4*)K.val.ptr, (const __nv_bfloat16*)phiQ, (const __nv_bfloat16*)phiK, map_v,

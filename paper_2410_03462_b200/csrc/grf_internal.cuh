@@ -97,7 +97,8 @@ struct grf_mask_dev {
     bool ready = false;
     int32_t blocks = 0;
     int64_t entries = 0;            // padded key entries over all blocks
-    grf_buf off, cnt, key, total;   // cnt holds [blocks] padded counts, then [blocks] the blocks by decreasing count
+    grf_buf off, cnt, key;          // cnt holds [blocks] padded counts, then [blocks] the blocks by decreasing count
+    grf_buf bits;                   // per block one bit per key: the block's key set
     grf_buf val;
 };
 
