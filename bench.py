@@ -1,9 +1,15 @@
 #!/usr/bin/env python
 """Benchmark of the GRF-masked linear-attention path: one step = sample the graph random features
-(walks, merge, CSR, regrouping) and evaluate the masked attention (state build, gather-contract) for one
-batch of synthetic inputs.  Prints ONE JSON line.
+(walks, merge, CSR, regrouping) and evaluate the masked attention for one batch of synthetic inputs.
+Prints ONE JSON line.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload pc32768] [--impl ours|reference]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload pc32768] [--route sz|mhat|asym]
+                    [--frozen] [--impl ours|reference]
+    python bench.py --suite        every workload, the unsorted point cloud, the scaling sweep and the operation
+                                   counts of Sec. 4: a summary (.md) and one JSON line per run (.jsonl) in --suite-dir
+
+Routes: sz = Alg. 1 through the per-node states S_l, z_l (Eq. 12; the headline); mhat = Eqs. 1-2 over the
+materialised mask Phi Psi^T; asym = Alg. 2 (asymmetric features, Psi = I).
 
 With N > 1 (launched by torch.distributed.run) every rank runs the same-sized, independently seeded batch
 on its own GPU (the problems are independent: no data-path collective); the value is the sum of all
@@ -12,7 +18,9 @@ ranks' tokens over the slowest rank's time.
 from __future__ import annotations
 
 import argparse
+import hashlib
 import json
+import math
 import os
 import statistics
 import subprocess
@@ -29,17 +37,12 @@ if ROOT not in sys.path:
 METRIC = "grf_masked_linear_attention_tokens_per_s"
 UNIT = "tokens/s"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0}
-# DRAM bytes (read + write) of one launch at the default workload, from the ncu capture summarised in
-# profiles/kernels_pointcloud32768_2heads.md (taken with 2 of the 8 heads; traffic grows in proportion to the
-# heads, so the figures are scaled by 4).  Set an entry to None when its kernel changes after the capture.
-NCU_TRAFFIC_BYTES = {
-    "pointcloud-gmm16-N32768": {
-        "gather_contract": 4 * (1.133120e9 + 12.062208e6),
-        "build_states": 4 * (0.062991e9 + 226.052096e6),
-        "row_denominators": 4 * (0.037775e9 + 0.042496e6),
-        "walk_merge": 0.005105e9 + 6.034688e6,
-    }
-}
+CSRC = os.path.join(ROOT, "paper_2410_03462_b200", "csrc")
+COUNTERS_FILE = os.path.join(ROOT, "profiles", "ncu_counters.md")
+# Delivery of randomly addressed 4 KB bulk copies into shared memory with two issuing warps per SM (the gather
+# kernel's configuration), measured once with a stand-alone copy loop on this GPU type: the resource that bounds
+# the gather of state tiles.  Plain 16-byte loads of an L2-resident region reach 19.5 TB/s.
+SMEM_FILL_PEAK_GBS = 6800.0
 
 
 def make_workload(name: str):
@@ -56,8 +59,41 @@ def peaks():
     if os.path.exists(path):
         with open(path) as fh:
             p = json.load(fh)
-        return float(p["hbm_gbs"]), "measured"
-    return FALLBACK_PEAKS["hbm_gbs"], "fallback"
+        return {"hbm_gbs": float(p["hbm_gbs"]), "bf16_tflops": float(p["bf16_tflops"]),
+                "bf16_tflops_sustained": float(p.get("bf16_tflops_sustained", p["bf16_tflops"])), "source": "measured"}
+    return {"hbm_gbs": FALLBACK_PEAKS["hbm_gbs"], "bf16_tflops": FALLBACK_PEAKS["bf16_tflops"],
+            "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+def source_hash(files) -> str:
+    """Hash of the kernel sources a profile entry was taken from (first 16 hex digits of SHA-256)."""
+    h = hashlib.sha256()
+    for f in files:
+        with open(os.path.join(CSRC, f), "rb") as fh:
+            h.update(fh.read())
+    return h.hexdigest()[:16]
+
+
+def load_counters():
+    """The tracked table of profiler counters, one row per kernel class:
+    | class | sources | source hash | workload | heads captured | dram bytes per launch at capture | issue % | tensor % | lsu % |
+    A row whose hash no longer matches the sources is stale: its figures are reported as null."""
+    out = {}
+    if not os.path.exists(COUNTERS_FILE):
+        return out
+    with open(COUNTERS_FILE) as fh:
+        for line in fh:
+            cells = [c.strip() for c in line.strip().strip("|").split("|")]
+            if len(cells) < 9 or cells[0] in ("class", "") or set(cells[0]) <= set("-: "):
+                continue
+            try:
+                files = cells[1].split()
+                out[cells[0]] = {"sources": files, "hash": cells[2], "workload": cells[3], "heads": int(cells[4]),
+                                 "dram_bytes": float(cells[5]), "issue_pct": float(cells[6]), "tensor_pct": float(cells[7]),
+                                 "lsu_pct": float(cells[8]), "stale": source_hash(files) != cells[2]}
+            except (ValueError, OSError):
+                continue
+    return out
 
 
 class ClockSampler:
@@ -139,6 +175,75 @@ def algorithmic_bytes(w, N, nnz_phi, nnz_psi, E):
     }
 
 
+def binding_report(w, N, nnz_phi, nnz_psi, ktimes, steps, pk, counters, plan_entries, mask_entries):
+    """For each big kernel, the rates of the resources that can bind it (from counts of this run and the CUDA-event
+    time of the kernel) and, where the tracked profile of the same sources exists, the profiler's busy fractions.
+    `binds` names the resource with the largest fraction of its peak."""
+    es = 2 if w.dtype == "bf16" else 4
+    G, m, d = w.G, w.m, w.d
+    rep = {}
+
+    def per_launch_s(name):
+        ms, n = ktimes.get(name, (0.0, 0))
+        return (ms / n) * 1e-3 if n else None
+
+    def prof(name):
+        c = counters.get(name)
+        if not c or c["stale"]:
+            return {"profile": "none for these sources" if not c else "stale (sources changed since the capture)"}
+        return {"issue_slots_busy_pct": c["issue_pct"], "tensor_pipe_busy_pct": c["tensor_pct"],
+                "lsu_pipe_busy_pct": c["lsu_pct"], "profile": f"{c['workload']}, {c['heads']} heads"}
+
+    def finish(name, r, fracs):
+        r["binds"] = max(fracs, key=fracs.get)
+        r["fraction_of_binding_peak"] = fracs[r["binds"]]
+        r.update(prof(name))
+        rep[name] = r
+
+    t = per_launch_s("gather_contract")
+    if t and plan_entries and w.dtype == "bf16":
+        issued = plan_entries * G * 2.0 * 128 * m * d / t / 1e12
+        useful = 2.0 * nnz_phi * m * d * G / t / 1e12
+        fill = plan_entries * G * m * d * es / t / 1e9
+        hbm = (G * N * m * d * es) / t / 1e9
+        finish("gather_contract", {
+            "tensor_issued_tflops": issued, "tensor_useful_tflops": useful, "tensor_peak_tflops": pk["bf16_tflops"],
+            "smem_fill_gbs": fill, "smem_fill_peak_gbs": SMEM_FILL_PEAK_GBS, "hbm_algorithmic_gbs": hbm},
+            {"tensor_issue": issued / pk["bf16_tflops"], "smem_fill": fill / SMEM_FILL_PEAK_GBS, "hbm": hbm / pk["hbm_gbs"]})
+    t = per_launch_s("build_states")
+    if t and w.dtype == "bf16":
+        gathered = (nnz_psi * G * (m + d) * es + G * N * (m * d * es + m * 6)) / t / 1e9
+        issued = 2.0 * 128 * m * (nnz_psi + 8 * N) * G / t / 1e12       # keys padded to steps of 16 (8 on average)
+        hbm = G * N * (m * d * es + m * 6) / t / 1e9
+        finish("build_states", {
+            "delivered_gbs": gathered, "delivery_peak_gbs": SMEM_FILL_PEAK_GBS, "tensor_issued_tflops": issued,
+            "tensor_peak_tflops": pk["bf16_tflops"], "hbm_algorithmic_gbs": hbm},
+            {"row_delivery": gathered / SMEM_FILL_PEAK_GBS, "tensor_issue": issued / pk["bf16_tflops"], "hbm": hbm / pk["hbm_gbs"]})
+    t = per_launch_s("walk_merge")
+    if t:
+        keep = 1.0 - w.p_halt
+        visits = (1.0 - keep ** (w.max_len + 1)) / w.p_halt        # expected nodes visited per walk (no dead ends)
+        walks = 2.0 * N * w.n_walks
+        c = counters.get("walk_merge")
+        issue = (c["issue_pct"] / 100.0) if c and not c["stale"] else None
+        r = {"walks_per_s": walks / t, "expected_hops_per_s": walks * (visits - 1.0) / t,
+             "hbm_algorithmic_gbs": (8 * (nnz_phi + nnz_psi)) / t / 1e9}
+        fr = {"hbm": r["hbm_algorithmic_gbs"] / pk["hbm_gbs"]}
+        if issue is not None:
+            fr["integer_issue"] = issue
+        finish("walk_merge", r, fr)
+    t = per_launch_s("mhat_attention")
+    if t and mask_entries:
+        issued = mask_entries * G * 2.0 * 128 * (m + d) / t / 1e12
+        masked = mask_entries * 128.0 * G / t / 1e9                 # score entries multiplied by the mask per second
+        hbm = (mask_entries * 260 + G * N * (2 * m + 2 * d) * es) / t / 1e9
+        finish("mhat_attention", {
+            "tensor_issued_tflops": issued, "tensor_peak_tflops": pk["bf16_tflops"], "masked_scores_g_per_s": masked,
+            "hbm_algorithmic_gbs": hbm},
+            {"tensor_issue": issued / pk["bf16_tflops"], "hbm": hbm / pk["hbm_gbs"]})
+    return rep
+
+
 def rank_seed(base: int, rank: int) -> int:
     """Every rank draws its own batch: same shapes, different values."""
     return base + rank
@@ -150,30 +255,33 @@ def aggregate_over_ranks(local_ms: float, tokens_per_rank_step: int, steps: int,
     return total_ms, tokens_per_rank_step * world * steps / (total_ms * 1e-3)
 
 
-def run_ours(args):
+DTYPE_NOTE = {
+    "sz": "bf16 storage, fp32 accumulation; tensor-core path multiplies bf16(Phi_il)*phi(q) and bf16(Psi_jl)*phi(k) rounded to bf16",
+    "mhat": "bf16 storage, fp32 scores and mask sums; the mask and the masked scores are rounded to bf16",
+    "asym": "bf16 storage, fp32 accumulation",
+}
+
+
+def measure(args, workload_name, route, with_cpu_baseline, with_e2e, frozen=False, steps=None, warmup=None):
     import torch
     import torch.distributed as dist
 
     from paper_2410_03462_b200 import api, binding as B
     from workloads import configs, tensors
 
+    steps = steps or args.steps
+    warmup = warmup or args.warmup
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local = int(os.environ.get("LOCAL_RANK", "0"))
-    if world != args.gpus:
-        raise SystemExit(f"--gpus {args.gpus} but WORLD_SIZE={world}")
-    torch.cuda.set_device(local)
-    if world > 1:
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
 
-    w = make_workload(args.workload)
+    w = make_workload(workload_name)
     if args.heads > 0:
         w.heads = args.heads
         w.name += f"-heads{args.heads}"
     g = w.graph()
     N, E = g.N, g.E
-    asym = args.route == "asym"
-    mhat = args.route == "mhat"
+    asym, mhat = route == "asym", route == "mhat"
     if asym:      # Alg. 2: f_phi = alpha, f_psi = delta_0 (no key-side walks contribute, Psi = I)
         f = w.alpha.astype(np.float32)
         f_psi = np.zeros(w.max_len + 1, np.float32); f_psi[0] = 1.0
@@ -188,15 +296,25 @@ def run_ours(args):
         q, k = (q.float() * 0.25).to(q.dtype), (k.float() * 0.25).to(k.dtype)
     qd, kd, vd = q.cuda(), k.cuda(), v.cuda()
     dt = B.dtype_code(qd)
-    ws_bytes = B.grf_attn_workspace_bytes(w.G, N, w.m, w.d, dt)
-    ws = torch.empty(ws_bytes, dtype=torch.uint8, device="cuda")
+    ws = None
+    ws_bytes = 0
+    if route == "sz":
+        ws_bytes = B.grf_attn_workspace_bytes(w.G, N, w.m, w.d, dt)
+        ws = torch.empty(ws_bytes, dtype=torch.uint8, device="cuda")
     out = torch.empty_like(vd)
     flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
     feat = api.Features(ctx, None)
 
-    def attention():
+    def sample(seed):
+        feat.handle = B.grf_sample(ctx.handle, N, dg.rowptr, dg.col, dg.w, seed, w.n_walks, w.p_halt, w.max_len, f, f_psi,
+                                   feat.handle)
+
+    def prepare():        # what a feature object needs once before the attention can use it
         if mhat:
             B.grf_features_materialise(ctx.handle, feat.handle)
+
+    def attention():
+        if mhat:
             B.grf_masked_attn_mhat(ctx.handle, feat.handle, w.G, N, w.m, w.d, dt, qd, kd, vd, out, None)
         elif asym:
             B.grf_masked_attn_asym(ctx.handle, feat.handle, w.G, N, w.m, w.d, dt,
@@ -204,15 +322,19 @@ def run_ours(args):
         else:
             B.grf_masked_linear_attn(ctx.handle, feat.handle, w.G, N, w.m, w.d, dt, qd, kd, vd, out, None, ws, ws_bytes)
 
-    def step(i):
-        feat.handle = B.grf_sample(ctx.handle, N, dg.rowptr, dg.col, dg.w, configs.WALK_SEED + i, w.n_walks, w.p_halt,
-                                   w.max_len, f, f_psi, feat.handle)
+    def step(seed):
+        if not frozen:
+            sample(seed)
+            prepare()
         attention()
 
     sampler = ClockSampler(local) if rank == 0 else None
     B.grf_ctx_enable_timing(ctx.handle, True)      # per-kernel events exist before the timed region starts
-    for i in range(args.warmup):
-        step(i)
+    if frozen:                                      # walks "pre-computed and frozen" (Sec. 4): outside the step
+        sample(configs.WALK_SEED)
+        prepare()
+    for i in range(warmup):
+        step(configs.WALK_SEED + i)
     torch.cuda.synchronize()
     B.grf_ctx_kernel_times(ctx.handle)             # discard the warm-up record
 
@@ -224,17 +346,19 @@ def run_ours(args):
     # ---- timed region: K steps, each bracketed by CUDA events on the stream the kernels run on;
     # L2 is flushed between steps, outside the events
     launches0 = ctx.launches
-    evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
-    ev_mid = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]
+    evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+    ev_mid = [torch.cuda.Event(enable_timing=True) for _ in range(steps)]
     barrier()
     t_wall0 = time.perf_counter()
     t_epoch0 = time.time()
-    for i in range(args.steps):
+    for i in range(steps):
         flush.zero_()
         evs[i][0].record()
-        feat.handle = B.grf_sample(ctx.handle, N, dg.rowptr, dg.col, dg.w, configs.WALK_SEED + 1000 + i, w.n_walks,
-                                   w.p_halt, w.max_len, f, f_psi, feat.handle)
+        if not frozen:
+            sample(configs.WALK_SEED + 1000 + i)
         ev_mid[i].record()
+        if not frozen:
+            prepare()
         attention()
         evs[i][1].record()
     barrier()
@@ -248,20 +372,28 @@ def run_ours(args):
     ktimes = B.grf_ctx_kernel_times(ctx.handle)
     B.grf_ctx_enable_timing(ctx.handle, False)
     nnz_phi, nnz_psi = feat.shape(0)[2], feat.shape(1)[2]
+    plan_entries = mask_entries = None
+    if route == "sz" and w.dtype == "bf16":
+        try:
+            plan_entries = B.grf_plan_stats(ctx.handle, feat.handle)[1]
+        except B.GrfError:
+            plan_entries = None                     # no plan: the plain-ALU gather ran
+    if mhat:
+        mask_entries = B.grf_mask_stats(feat.handle)[1]
 
     # ---- end to end through the host-buffer entry point (pinned host memory; copies inside the timing)
-    qh, kh, vh = q.pin_memory(), k.pin_memory(), v.pin_memory()
-    oh = torch.empty_like(v).pin_memory()
-    rp_h = torch.from_numpy(g.rowptr).pin_memory(); c_h = torch.from_numpy(g.col).pin_memory()
-    w_h = torch.from_numpy(g.w).pin_memory()
-    e2e_steps = max(2, min(args.steps, 5))
+    e2e = None
+    if with_e2e and route == "sz" and not frozen:
+        qh, kh, vh = q.pin_memory(), k.pin_memory(), v.pin_memory()
+        oh = torch.empty_like(v).pin_memory()
+        rp_h = torch.from_numpy(g.rowptr).pin_memory(); c_h = torch.from_numpy(g.col).pin_memory()
+        w_h = torch.from_numpy(g.w).pin_memory()
+        e2e_steps = max(2, min(steps, 5))
 
-    def host_step(i):
-        B.grf_step_host(ctx.handle, N, rp_h, c_h, w_h, configs.WALK_SEED + 2000 + i, w.n_walks, w.p_halt, w.max_len,
-                        f, None, w.G, w.m, w.d, dt, qh, kh, vh, oh)
+        def host_step(i):
+            B.grf_step_host(ctx.handle, N, rp_h, c_h, w_h, configs.WALK_SEED + 2000 + i, w.n_walks, w.p_halt, w.max_len,
+                            f, None, w.G, w.m, w.d, dt, qh, kh, vh, oh)
 
-    e2e_ms = float("nan")
-    if not asym and not mhat:
         host_step(0)
         barrier()
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -270,9 +402,9 @@ def run_ours(args):
             host_step(1 + i)
         e1.record()
         barrier()
-        e2e_ms = e0.elapsed_time(e1) / e2e_steps
-    h2d = (rp_h.numel() + c_h.numel() + w_h.numel()) * 4 + sum(t.numel() * t.element_size() for t in (qh, kh, vh))
-    d2h = oh.numel() * oh.element_size()
+        e2e = {"ms": e0.elapsed_time(e1) / e2e_steps,
+               "h2d": (rp_h.numel() + c_h.numel() + w_h.numel()) * 4 + sum(t.numel() * t.element_size() for t in (qh, kh, vh)),
+               "d2h": oh.numel() * oh.element_size()}
 
     clocks = sampler.stop(t_epoch0, t_epoch1) if sampler else None
 
@@ -284,95 +416,149 @@ def run_ours(args):
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
         return float(t.item())
 
-    total_ms, value = aggregate_over_ranks(total_ms, w.batch * N, args.steps, world, rmax)
-    e2e_ms = rmax(e2e_ms)
+    total_ms, value = aggregate_over_ranks(total_ms, w.batch * N, steps, world, rmax)
+    if e2e:
+        e2e["ms"] = rmax(e2e["ms"])
     tokens_per_step = w.batch * N * world
 
     result = None
     if rank == 0:
-        peak_gbs, peak_kind = peaks()
+        pk = peaks()
+        counters = load_counters()
         alg = algorithmic_bytes(w, N, nnz_phi, nnz_psi, E)
-        if mhat:   # Q, K, V read once, out written once, the mask blocks written once and read once
-            es = 2
-            mblocks, mentries, mbytes = B.grf_mask_stats(feat.handle)
+        es = 2 if w.dtype == "bf16" else 4
+        if mhat:   # Q, K, V read once, out written once; the mask blocks written once, read once
+            mbytes = B.grf_mask_stats(feat.handle)[2]
             alg["mhat_attention"] = w.G * N * (2 * w.m + 2 * w.d) * es + mbytes
             alg["mask_build"] = mbytes + 2 * (nnz_phi + nnz_psi) * 8
         if asym:   # Q, K, V, Phi read once, out written once; no states
-            es = 2 if w.dtype == "bf16" else 4
             alg["gather_contract"] = w.G * N * (2 * w.m + 2 * w.d) * es + nnz_phi * 8 + (N + 1) * 4
         per_kernel = {}
         for name, (ms, n) in ktimes.items():
-            per = ms / max(n, 1)
+            if n == 0:
+                continue
+            per = ms / n
             a = alg.get(name, 0)
-            per_kernel[name] = {"ms_per_step": ms / args.steps, "launch_groups": n,
-                                "algorithmic_gb": a / 1e9,
-                                "achieved_gbs": a / 1e9 / (per * 1e-3) if n else None}
+            per_kernel[name] = {"ms_per_step": ms / steps, "launch_groups": n, "algorithmic_gb": a / 1e9,
+                                "achieved_gbs": a / 1e9 / (per * 1e-3), "hbm_frac": a / 1e9 / (per * 1e-3) / pk["hbm_gbs"]}
         dom = max(ktimes, key=lambda kname: ktimes[kname][0])
         dom_ms = ktimes[dom][0] / max(ktimes[dom][1], 1)
         achieved = alg.get(dom, 0) / 1e9 / (dom_ms * 1e-3)
+        binding = binding_report(w, N, nnz_phi, nnz_psi, ktimes, steps, pk, counters, plan_entries, mask_entries)
+        # DRAM traffic of the dominant kernel from the tracked profile of the same sources, scaled to this run's heads
+        traffic = None
+        c = counters.get(dom)
+        if c and not c["stale"] and c["workload"] == w.name.split("-heads")[0]:
+            traffic = c["dram_bytes"] * (w.G / c["heads"] if dom != "walk_merge" else 1.0)
+        binds = binding.get(dom, {}).get("binds")
+        bound = {"tensor_issue": "tensor", "hbm": "hbm", "integer_issue": "alu"}.get(binds, "hbm" if binds is None else "smem")
+        step_text = {"sz": "grf_sample (both ensembles) + grf_masked_linear_attn",
+                     "mhat": "grf_sample (both ensembles) + grf_features_materialise + grf_masked_attn_mhat",
+                     "asym": "grf_sample (f_psi = delta_0) + grf_masked_attn_asym (Alg. 2, %s similarity)"
+                             % ("softmax" if args.softmax else "linear")}[route]
         result = {
-            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
-            "warmup": args.warmup, "ms_per_step": total_ms / args.steps, "higher_is_better": True,
-            "scaling": "weak", "vs_baseline": None, "dtype": "f32 accumulate, " + w.dtype + " storage",
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": steps,
+            "warmup": warmup, "ms_per_step": total_ms / steps, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None,
+            "dtype": ("bf16" if w.dtype == "bf16" else "f32"), "dtype_note": DTYPE_NOTE[route] if w.dtype == "bf16" else "fp32 throughout",
             "data": "synthetic",
-            "config": {"workload": w.name, "N": N, "edges": E, "batch": w.batch, "heads": w.heads, "m": w.m, "d": w.d,
-                       "n_walks": w.n_walks, "p_halt": w.p_halt, "max_len": w.max_len,
+            "config": {"workload": w.name, "route": route, "N": N, "edges": E, "batch": w.batch, "heads": w.heads, "m": w.m,
+                       "d": w.d, "n_walks": w.n_walks, "p_halt": w.p_halt, "max_len": w.max_len,
                        "nnz_phi": nnz_phi, "nnz_psi": nnz_psi,
+                       "node_order": "as given" if "unsorted" in w.name else
+                                     ("Morton order of the points" if "pointcloud" in w.name else "generator's order"),
+                       "features": "frozen: sampled once before the timed region" if frozen else "resampled every step",
                        "l2": "256 MiB flush write between steps, outside the per-step events",
-                       "step": ("grf_sample (f_psi = delta_0) + grf_masked_attn_asym (Alg. 2, %s similarity), features "
-                                "resampled every step" % ("softmax" if args.softmax else "linear")) if asym else
-                               ("grf_sample (both ensembles) + grf_features_materialise + grf_masked_attn_mhat, features "
-                                "resampled and the mask rebuilt every step") if mhat else
-                               "grf_sample (both ensembles) + grf_masked_linear_attn, features resampled every step"},
+                       "step": step_text + (", attention only (features frozen)" if frozen else ", features resampled every step")},
             "clocks": clocks,
             "gpu_launches": launches,
-            "e2e": None if (asym or mhat) else
-                   {"value": tokens_per_step / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
-                    "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms, "entry_point": "grf_step_host"},
-            "roofline": {"kernel": dom, "bound": "hbm", "achieved": achieved, "peak": peak_gbs, "unit": "GB/s",
-                         "frac": achieved / peak_gbs, "peak_source": peak_kind,
-                         "traffic": None if (asym or mhat) else NCU_TRAFFIC_BYTES.get(w.name, {}).get(dom),
-                         "algorithmic_bytes": alg.get(dom, 0), "ms_per_launch": dom_ms},
+            "e2e": None if not e2e else
+                   {"value": tokens_per_step / (e2e["ms"] * 1e-3), "unit": UNIT, "h2d_bytes_per_step": e2e["h2d"],
+                    "d2h_bytes_per_step": e2e["d2h"], "ms_per_step": e2e["ms"], "entry_point": "grf_step_host"},
+            "roofline": {"kernel": dom, "bound": bound, "frac_of": "hbm (the metric's roofline)", "achieved": achieved,
+                         "peak": pk["hbm_gbs"], "unit": "GB/s", "frac": achieved / pk["hbm_gbs"], "peak_source": pk["source"],
+                         "traffic": traffic, "algorithmic_bytes": alg.get(dom, 0),
+                         "algorithmic_bytes_per_token_head": alg.get(dom, 0) / (w.G * N), "ms_per_launch": dom_ms,
+                         "binding_resource": binds,
+                         "fraction_of_binding_peak": binding.get(dom, {}).get("fraction_of_binding_peak")},
+            "binding": binding,
             "phases": {"sample_ms": statistics.mean(sample_ms), "attn_ms": statistics.mean(attn_ms),
                        "sample_ms_min_med_max": [min(sample_ms), statistics.median(sample_ms), max(sample_ms)],
                        "attn_ms_min_med_max": [min(attn_ms), statistics.median(attn_ms), max(attn_ms)],
-                       "walks_per_s": 2 * N * w.n_walks / (statistics.mean(sample_ms) * 1e-3),
+                       "walks_per_s": None if frozen else 2 * N * w.n_walks / (statistics.mean(sample_ms) * 1e-3),
                        "attn_tokens_per_s": w.batch * N / (statistics.mean(attn_ms) * 1e-3),
+                       "attn_hbm_frac": (2 * w.G * N * w.m * w.d * es + w.G * N * (2 * w.m + 2 * w.d) * es) / 1e9 /
+                                        (statistics.mean(attn_ms) * 1e-3) / pk["hbm_gbs"] if route == "sz" else None,
                        "wall_s_timed_region": wall},
             "kernels": per_kernel,
         }
-        if not args.no_cpu_baseline and world == 1:
-            result["cpu_baseline"] = cpu_baseline(w, g, f, args.cpu_heads)
+        if with_cpu_baseline and world == 1:
+            result["cpu_baseline"] = cpu_baseline(w, g, f)
     feat.free()
     ctx.close()
-    if world > 1:
-        dist.destroy_process_group()
+    del ws, out, flush, qd, kd, vd
+    torch.cuda.empty_cache()
     return result
 
 
-def cpu_baseline(w, g, f, heads: int = 1):
-    """The oracle as it stands, timed on this host: the whole sampler plus `heads` of the batch's heads of
-    the S/z-route attention; the step time is extrapolated linearly to all heads."""
+_POOL_STATE = {}
+
+
+def _cpu_pool_init(phi, psit):
+    import oracle
+    _POOL_STATE["Phi"] = oracle.CSR(*phi)
+    _POOL_STATE["PsiT"] = oracle.CSR(*psit)
+    oracle._load()
+
+
+def _cpu_attn_head(qkv):
+    import oracle
+    q, k, v = qkv
+    t0 = time.perf_counter()
+    oracle.attn_sparse(q, k, v, _POOL_STATE["Phi"], _POOL_STATE["PsiT"], with_abs=False)
+    return time.perf_counter() - t0
+
+
+def cpu_baseline(w, g, f, max_heads=None):
+    """The oracle as it stands, timed on this host: the whole sampler (one thread: it is a serial program) and the
+    S/z-route attention of the batch's problems, one oracle process per problem on the cores this process may use
+    (a spawn pool; the problems are independent, the oracle itself is not changed or tuned).  When there are fewer
+    cores than problems, or `max_heads` bounds the sample, only that many problems run and the attention time is
+    scaled to the whole batch."""
+    import multiprocessing as mp
+
     import oracle
     from workloads import configs, tensors
+    cores_avail = len(os.sched_getaffinity(0))
     t0 = time.perf_counter()
     Phi, Psi, PsiT, _, _ = oracle.sample(g.rowptr, g.col, g.w, configs.WALK_SEED, w.n_walks, w.p_halt, w.max_len, f)
     t_sample = time.perf_counter() - t0
-    heads = max(1, min(heads, w.G))
+    heads = max(1, min(w.G, cores_avail, max_heads or w.G))
     q, k, v = tensors.qkv(heads, g.N, w.m, w.d, w.dtype, configs.QKV_SEED)
     qf, kf, vf = tensors.widen(q), tensors.widen(k), tensors.widen(v)
-    t0 = time.perf_counter()
-    oracle.attn_sparse(qf, kf, vf, Phi, PsiT, with_abs=False)
-    t_attn = (time.perf_counter() - t0) * (w.G / heads)
+    pack = lambda M: (M.rowptr, M.col, M.val, None, M.shape)
+    with mp.get_context("spawn").Pool(heads, initializer=_cpu_pool_init, initargs=(pack(Phi), pack(PsiT))) as pool:
+        pool.map(_cpu_noop, range(heads))                     # workers started and the oracle loaded before the clock
+        t0 = time.perf_counter()
+        per_head = pool.map(_cpu_attn_head, [(qf[h:h + 1], kf[h:h + 1], vf[h:h + 1]) for h in range(heads)], chunksize=1)
+        t_wall = time.perf_counter() - t0
+    t_attn = t_wall * (w.G / heads)
     step = t_sample + t_attn
-    return {"value": w.batch * g.N / step, "unit": UNIT, "cores": 1, "kind": "oracle",
-            "sample": f"full sampler ({t_sample:.2f} s) + {heads} of {w.G} problems of the attention, "
-                      f"attention time scaled by {w.G}/{heads} ({t_attn:.2f} s)",
-            "sampler_s": t_sample, "attn_s_extrapolated": t_attn}
+    return {"value": w.batch * g.N / step, "unit": UNIT, "cores": heads, "cores_available": cores_avail, "kind": "oracle",
+            "sample": f"full sampler on one core ({t_sample:.2f} s) + {heads} of {w.G} problems of the attention, one "
+                      f"oracle process each ({t_wall:.2f} s wall, {statistics.mean(per_head):.2f} s per problem)"
+                      + ("" if heads == w.G else f", attention time scaled by {w.G}/{heads}"),
+            "sampler_s": t_sample, "attn_s": t_attn, "attn_s_per_problem_one_core": statistics.mean(per_head),
+            "single_core_value": w.batch * g.N / (t_sample + statistics.mean(per_head) * w.G)}
+
+
+def _cpu_noop(_):
+    return 0
 
 
 def run_reference(args):
-    """The CPU oracle timed as the reference arm: K steps, each a bounded sample of the workload."""
+    """The CPU oracle timed as the reference arm: K steps, each the whole sampler plus a bounded sample of the
+    batch's problems (at most four, one process each), sized so that the run ends within a few minutes."""
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return None
@@ -380,19 +566,129 @@ def run_reference(args):
     w = make_workload(args.workload)
     g = w.graph()
     f = oracle.deconvolve(w.alpha).astype(np.float32)
-    steps = max(1, min(args.steps, 3))
-    for _ in range(min(args.warmup, 1)):
-        cpu_baseline(w, g, f, 1)
-    vals = [cpu_baseline(w, g, f, args.cpu_heads) for _ in range(steps)]
+    warm = min(args.warmup, 1)
+    for _ in range(warm):
+        cpu_baseline(w, g, f, max_heads=4)
+    t0 = time.perf_counter()
+    vals = []
+    for _ in range(args.steps):
+        vals.append(cpu_baseline(w, g, f, max_heads=4))
+        if time.perf_counter() - t0 > 240 and len(vals) >= 3:     # keep the arm within a few minutes
+            break
     value = statistics.mean(x["value"] for x in vals)
     ms = w.batch * g.N / value * 1e3
     base = dict(vals[-1]); base["value"] = value
-    return {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": steps,
-            "warmup": min(args.warmup, 1), "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
+    return {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": len(vals),
+            "warmup": warm, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-            "config": {"workload": w.name, "N": g.N, "batch": w.batch, "heads": w.heads, "m": w.m, "d": w.d},
+            "config": {"workload": w.name, "route": "sz", "N": g.N, "batch": w.batch, "heads": w.heads, "m": w.m, "d": w.d},
             "cpu_baseline": base,
             "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+
+
+def flops_figure(args):
+    """Sec. 4 "Time complexity": operation counts against the number of nodes on 1-D grids, n = 4 walkers,
+    p_halt = 0.5, m = d = 8, the masked count averaged over 10 seeds (features sampled on the GPU)."""
+    from paper_2410_03462_b200 import api, binding as B
+    from workloads import graphs
+    ctx = api.Context(int(os.environ.get("LOCAL_RANK", "0")))
+    L = 8
+    f = B.grf_deconvolve(0.5 ** np.arange(L + 1)).astype(np.float32)
+    rows = []
+    for k in range(6, 15):
+        N = 1 << k
+        dg = api.DeviceGraph(graphs.path_graph(N, 0.5))
+        masked = []
+        for seed in range(10):
+            feat = api.sample(ctx, dg, seed, 4, 0.5, L, f)
+            mk, lin, sm = B.grf_attn_flops(feat.handle, 8, 8)
+            masked.append(mk)
+            feat.free()
+        rows.append({"N": N, "masked_mean": float(np.mean(masked)), "masked_std": float(np.std(masked)),
+                     "unmasked_linear": lin, "softmax": sm})
+    ctx.close()
+    return rows
+
+
+def loglog_slope(xs, ys):
+    lx, ly = np.log(np.asarray(xs, float)), np.log(np.asarray(ys, float))
+    return float(np.polyfit(lx, ly, 1)[0])
+
+
+def run_suite(args):
+    """All workloads on both symmetric routes, the unsorted point cloud, frozen features, the sweep 2^10..2^20 (sz
+    route) with the fitted slopes, and the operation counts; writes <dir>/bench_suite.jsonl and <dir>/bench_suite.md."""
+    os.makedirs(args.suite_dir, exist_ok=True)
+    lines, md = [], []
+
+    def run(name, route, frozen=False, steps=10):
+        from paper_2410_03462_b200 import binding as B
+        case = f"{name}/{route}" + ("/frozen" if frozen else "")
+        try:
+            r = measure(args, name, route, False, route == "sz" and not frozen and name in ("pc32768", "vit", "pc4096"),
+                        frozen=frozen, steps=steps, warmup=3)
+        except B.GrfError as e:          # e.g. the materialised mask of a graph without locality exceeds its limit
+            lines.append({"suite_case": case, "error": str(e)})
+            md.append(f"| {case} | not run: {e} |")
+            return None
+        r["suite_case"] = case
+        lines.append(r)
+        return r
+
+    md.append("| case | N | G | ms/step | sampler ms | attention ms | M tokens/s | G walks/s | dominant kernel | its ms | HBM frac | binds (fraction of that peak) |")
+    md.append("|---|---|---|---|---|---|---|---|---|---|---|---|")
+
+    def row(r):
+        if r is None:
+            return
+        c, ph, rf = r["config"], r["phases"], r["roofline"]
+        fb = rf.get("fraction_of_binding_peak")
+        md.append(f"| {r['suite_case']} | {c['N']} | {c['batch'] * c['heads']} | {r['ms_per_step']:.3f} | {ph['sample_ms']:.3f} | "
+                  f"{ph['attn_ms']:.3f} | {r['value'] / 1e6:.2f} | "
+                  f"{'-' if ph['walks_per_s'] is None else format(ph['walks_per_s'] / 1e9, '.2f')} | {rf['kernel']} | "
+                  f"{rf['ms_per_launch']:.3f} | {rf['frac']:.3f} | {rf['binding_resource']} ({'-' if fb is None else format(fb, '.2f')}) |")
+
+    for name in ("tiny", "vit", "pc4096", "pc32768", "pc32768-unsorted"):
+        row(run(name, "sz"))
+        if name != "tiny":
+            row(run(name, "sz", frozen=True))
+            row(run(name, "mhat"))
+            row(run(name, "mhat", frozen=True))
+    sweep = []
+    for k in range(10, 21):
+        r = run(f"sweep{k}", "sz", steps=10 if k < 18 else 4)
+        row(r)
+        if r is not None:
+            sweep.append(r)
+    big = [r for r in sweep if r["config"]["N"] >= 1 << 14]
+    Ns = [r["config"]["N"] for r in big]
+    slopes = {"sampler": loglog_slope(Ns, [r["phases"]["sample_ms"] for r in big]),
+              "attention": loglog_slope(Ns, [r["phases"]["attn_ms"] for r in big])}
+    md.append("")
+    md.append(f"Sweep (8-regular graphs, sz route), log-log slope of time against N for N >= 2^14: sampler "
+              f"{slopes['sampler']:.3f}, attention {slopes['attention']:.3f} (1.0 = linear time).")
+    md.append("Attention time per token-head (ns): " + ", ".join(
+        f"2^{int(math.log2(r['config']['N']))}: {r['phases']['attn_ms'] * 1e6 / (r['config']['N'] * r['config']['heads']):.1f}"
+        for r in sweep) + " (the per-problem records outgrow L2, 126 MB, between 2^13 and 2^15).")
+    fl = flops_figure(args)
+    md.append("")
+    md.append("Operation counts (Sec. 4 \"Time complexity\": 1-D grids, n = 4, p_halt = 0.5, m = d = 8, 10 seeds):")
+    md.append("")
+    md.append("| N | GRF-masked linear (mean) | std | unmasked linear | softmax | masked / unmasked linear |")
+    md.append("|---|---|---|---|---|---|")
+    for x in fl:
+        md.append(f"| {x['N']} | {x['masked_mean']:.0f} | {x['masked_std']:.0f} | {x['unmasked_linear']} | {x['softmax']} | "
+                  f"{x['masked_mean'] / x['unmasked_linear']:.2f} |")
+    md.append("")
+    md.append(f"log-log slope of the masked count against N: {loglog_slope([x['N'] for x in fl], [x['masked_mean'] for x in fl]):.3f}; "
+              f"of the softmax count: {loglog_slope([x['N'] for x in fl], [x['softmax'] for x in fl]):.3f}.")
+    with open(os.path.join(args.suite_dir, "bench_suite.jsonl"), "w") as fh:
+        for r in lines:
+            fh.write(json.dumps(r) + "\n")
+        fh.write(json.dumps({"sweep_slopes": slopes, "flops_figure": fl}) + "\n")
+    with open(os.path.join(args.suite_dir, "bench_suite.md"), "w") as fh:
+        fh.write("\n".join(md) + "\n")
+    return {"suite": "done", "cases": len(lines), "sweep_slopes": slopes, "dir": args.suite_dir}
 
 
 def main():
@@ -402,17 +698,37 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--workload", default="pc32768")
-    ap.add_argument("--cpu-heads", type=int, default=1, help="problems of the batch the CPU baseline really runs")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--route", choices=["sz", "asym", "mhat"], default="sz",
-                    help="sz: Alg. 1 (per-node states, the default); asym: Alg. 2 (asymmetric features, Psi = I), "
-                         "a variant outside the headline metric, no end-to-end leg")
+                    help="sz: Alg. 1 through per-node states (the default and the headline); mhat: Eqs. 1-2 over the "
+                         "materialised mask Phi Psi^T; asym: Alg. 2 (asymmetric features, Psi = I); the last two are "
+                         "variants outside the headline metric, without an end-to-end leg")
+    ap.add_argument("--frozen", action="store_true", help="features sampled (and prepared) once, outside the timed steps")
     ap.add_argument("--softmax", action="store_true", help="with --route asym: A_ij = exp(q_i . k_j)")
     ap.add_argument("--heads", type=int, default=0, help="override the workload's head count (profiling of a smaller case)")
+    ap.add_argument("--suite", action="store_true")
+    ap.add_argument("--suite-dir", default=os.path.join(ROOT, "gpurun_out"))
     args = ap.parse_args()
     if args.warmup < 3 and args.impl == "ours":
         args.warmup = 3
-    res = run_reference(args) if args.impl == "reference" else run_ours(args)
+    if args.impl == "reference":
+        res = run_reference(args)
+    else:
+        import torch
+        import torch.distributed as dist
+        world = int(os.environ.get("WORLD_SIZE", "1"))
+        local = int(os.environ.get("LOCAL_RANK", "0"))
+        if world != args.gpus:
+            raise SystemExit(f"--gpus {args.gpus} but WORLD_SIZE={world}")
+        torch.cuda.set_device(local)
+        if world > 1:
+            dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+        if args.suite:
+            res = run_suite(args)
+        else:
+            res = measure(args, args.workload, args.route, not args.no_cpu_baseline, True, frozen=args.frozen)
+        if world > 1:
+            dist.destroy_process_group()
     if res is not None:
         print(json.dumps(res))
 

@@ -256,6 +256,12 @@ int grf_ctx_check(grf_ctx* ctx);
  * 0 = plain-ALU kernels always.  Results agree within the stated tolerance. */
 int grf_ctx_use_tensor_cores(grf_ctx* ctx, int enable);
 
+/* The block plan of Phi that the tensor-core gather uses (built here if absent; waits for the stream then): HOST
+ * outputs, any may be NULL: number of 128-row blocks, and the node-list entries summed over the blocks (each is one
+ * state tile a block brings into shared memory per problem).  GRF_ERR_TOO_LARGE when the object has no plan (see
+ * grf_masked_linear_attn). */
+int grf_plan_stats(grf_ctx* ctx, const grf_features* feat, int32_t* blocks, int64_t* entries);
+
 /* Number of kernels the context has launched since it was created (for accounting in benchmarks). */
 int64_t grf_ctx_launch_count(const grf_ctx* ctx);
 

@@ -51,6 +51,7 @@ _SIGNATURES = {
     "grf_masked_attn_mhat": (_int, [_vp, _vp, _i32, _i32, _i32, _i32, _int, _vp, _vp, _vp, _vp, _vp]),
     "grf_step_host": (_int, [_vp, _i32, _vp, _vp, _vp, _u64, _i32, _f32, _i32, _vp, _vp,
                              _i32, _i32, _i32, _int, _vp, _vp, _vp, _vp]),
+    "grf_plan_stats": (_int, [_vp, _vp, ctypes.POINTER(_i32), ctypes.POINTER(_i64)]),
     "grf_ctx_launch_count": (_i64, [_vp]),
     "grf_ctx_check": (_int, [_vp]),
     "grf_ctx_use_tensor_cores": (_int, [_vp, _int]),
@@ -112,6 +113,13 @@ def grf_ctx_create(device: int = 0, stream: int | None = None) -> int:
 
 def grf_ctx_destroy(ctx: int):
     _check(lib.grf_ctx_destroy(ctx), "grf_ctx_destroy")
+
+
+def grf_plan_stats(ctx, features):
+    """(blocks, node-list entries over all blocks) of the tensor-core gather's block plan."""
+    b, e = _i32(), _i64()
+    _check(lib.grf_plan_stats(ctx, features, ctypes.byref(b), ctypes.byref(e)), "grf_plan_stats")
+    return b.value, e.value
 
 
 def grf_ctx_launch_count(ctx: int) -> int:

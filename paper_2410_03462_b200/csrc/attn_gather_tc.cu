@@ -538,7 +538,19 @@ int grf_build_block_plan(grf_ctx* ctx, grf_features* feat)
     }
     GRF_CUDA_TRY(cudaGetLastError());
     feat->plan_blocks = nblocks;
+    feat->plan_entries = (int64_t)entries;
     feat->plan_ready = true;
+    return GRF_OK;
+}
+
+extern "C" int grf_plan_stats(grf_ctx* ctx, const grf_features* feat, int32_t* blocks, int64_t* entries)
+{
+    if (!ctx || !feat) return GRF_ERR_INVALID;
+    GRF_CUDA_TRY(cudaSetDevice(ctx->device));
+    GRF_TRY(grf_ensure_block_plan(ctx, feat));
+    if (!feat->plan_ready) return GRF_ERR_TOO_LARGE;
+    if (blocks) *blocks = feat->plan_blocks;
+    if (entries) *entries = feat->plan_entries;
     return GRF_OK;
 }
 

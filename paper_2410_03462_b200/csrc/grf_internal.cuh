@@ -111,6 +111,7 @@ struct grf_features {
     grf_buf plan_off, plan_cnt, plan_col, plan_total;
     grf_buf plan_coef;              // dense bf16 coefficients [quad of union entries][row of the block][4]
     int32_t plan_blocks = 0;
+    int64_t plan_entries = 0;       // node-list entries over all blocks (padded to multiples of 4)
     bool plan_ready = false;
     bool plan_stale = true;         // Phi changed since the plan was built: the gather kernel's launcher rebuilds it
 };
