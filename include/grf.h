@@ -30,7 +30,7 @@ extern "C" {
 #define GRF_ERR_WORKSPACE  (-3)  /* caller's workspace too small                                                 */
 #define GRF_ERR_CUDA       (-4)  /* a CUDA runtime call failed                                                   */
 #define GRF_ERR_NOMEM      (-5)  /* device or host allocation failed                                             */
-#define GRF_ERR_BADGRAPH   (-6)  /* CSR input inconsistent (host-side checks of host-resident graphs only)       */
+#define GRF_ERR_BADGRAPH   (-6)  /* CSR input inconsistent (grf_step_host always checks; grf_sample on request)   */
 #define GRF_ERR_TIMEOUT    (-7)  /* a kernel gave up a bounded wait; its outputs are not valid                   */
 
 #define GRF_DTYPE_F32  0
@@ -246,6 +246,13 @@ int grf_step_host(grf_ctx* ctx, int32_t N, const int32_t* rowptr, const int32_t*
                   const float* f_phi, const float* f_psi,
                   int32_t G, int32_t m, int32_t d, int dtype,
                   const void* phiQ, const void* phiK, const void* V, void* out);
+
+/* Debugging aid: while enabled, grf_sample first validates the device-resident graph with a kernel (row pointers
+ * start at 0 and never decrease, column indices in [0, N); col is only read inside [0, rowptr[N])) and waits for
+ * the result: GRF_ERR_BADGRAPH, and no walk is taken, if it is inconsistent.  Off by default (one extra pass over
+ * the graph and one wait per call).  Kernel launches are also named as NVTX ranges ("grf:walk_merge", ...) for
+ * profilers' timelines; that costs nothing when no tool is attached. */
+int grf_ctx_check_graphs(grf_ctx* ctx, int enable);
 
 /* Waits for the context's stream and reports whether any kernel since the previous check gave up one of its
  * bounded waits (GRF_ERR_TIMEOUT; the affected outputs are invalid), else GRF_OK. */

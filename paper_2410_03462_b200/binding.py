@@ -54,6 +54,7 @@ _SIGNATURES = {
     "grf_plan_stats": (_int, [_vp, _vp, ctypes.POINTER(_i32), ctypes.POINTER(_i64)]),
     "grf_ctx_launch_count": (_i64, [_vp]),
     "grf_ctx_check": (_int, [_vp]),
+    "grf_ctx_check_graphs": (_int, [_vp, _int]),
     "grf_ctx_use_tensor_cores": (_int, [_vp, _int]),
     "grf_ctx_enable_timing": (_int, [_vp, _int]),
     "grf_ctx_kernel_times": (_int, [_vp, _vp, _vp]),
@@ -128,6 +129,10 @@ def grf_ctx_launch_count(ctx: int) -> int:
 
 def grf_ctx_check(ctx: int):
     _check(lib.grf_ctx_check(ctx), "grf_ctx_check")
+
+
+def grf_ctx_check_graphs(ctx: int, enable: bool):
+    _check(lib.grf_ctx_check_graphs(ctx, int(enable)), "grf_ctx_check_graphs")
 
 
 def grf_ctx_use_tensor_cores(ctx: int, enable: bool):

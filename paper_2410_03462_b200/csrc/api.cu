@@ -3,6 +3,8 @@
 #include <cstring>
 #include <new>
 
+#include <nvtx3/nvToolsExt.h>
+
 #include "grf_internal.cuh"
 
 int grf_buf_reserve(grf_buf* b, size_t bytes)
@@ -44,8 +46,8 @@ extern "C" int grf_ctx_create(grf_ctx** out, int device, void* cuda_stream)
     c->stream = (cudaStream_t)cuda_stream;
     if (cudaDeviceGetAttribute(&c->sm_count, cudaDevAttrMultiProcessorCount, device) != cudaSuccess ||
         cudaMallocHost((void**)&c->pinned, 64) != cudaSuccess ||
-        cudaMalloc((void**)&c->error_word, sizeof(int)) != cudaSuccess ||
-        cudaMemset(c->error_word, 0, sizeof(int)) != cudaSuccess) {
+        cudaMalloc((void**)&c->error_word, 2 * sizeof(int)) != cudaSuccess ||
+        cudaMemset(c->error_word, 0, 2 * sizeof(int)) != cudaSuccess) {
         cudaGetLastError();
         delete c;
         return GRF_ERR_CUDA;
@@ -87,8 +89,14 @@ static cudaEvent_t take_event(grf_ctx* c)
     return e;
 }
 
+// names of the kernel classes, as ranges in a profiler's timeline
+static const char* const kernel_class_names[GRF_KERNEL_CLASSES] = {
+    "grf:walk_merge", "grf:scan", "grf:compact", "grf:regroup", "grf:build_states", "grf:gather_contract",
+    "grf:row_denominators", "grf:block_plan", "grf:mask_build", "grf:mhat_attention"};
+
 grf_launch_scope::grf_launch_scope(grf_ctx* c, int cls_, int n_launches) : ctx(c), cls(cls_), n(n_launches)
 {
+    nvtxRangePushA(kernel_class_names[cls]);     // costs nothing unless a tool is attached
     if (!ctx->timing) return;
     beg = take_event(ctx); end = take_event(ctx);
     if (beg && end) cudaEventRecord(beg, ctx->stream);
@@ -96,6 +104,7 @@ grf_launch_scope::grf_launch_scope(grf_ctx* c, int cls_, int n_launches) : ctx(c
 
 grf_launch_scope::~grf_launch_scope()
 {
+    nvtxRangePop();
     ctx->launches += n;
     if (!ctx->timing || !beg || !end) return;
     cudaEventRecord(end, ctx->stream);
@@ -106,6 +115,13 @@ extern "C" int grf_ctx_use_tensor_cores(grf_ctx* ctx, int enable)
 {
     if (!ctx) return GRF_ERR_INVALID;
     ctx->use_tensor_cores = enable != 0;
+    return GRF_OK;
+}
+
+extern "C" int grf_ctx_check_graphs(grf_ctx* ctx, int enable)
+{
+    if (!ctx) return GRF_ERR_INVALID;
+    ctx->check_graphs = enable != 0;
     return GRF_OK;
 }
 

@@ -320,6 +320,24 @@ debug_walks_kernel(const __grid_constant__ grf_walk_params P,
     for (++t; t < Lp1; ++t) { tr[t] = -1; ld[t] = 0.0f; }
 }
 
+// Consistency of a device-resident CSR graph: row pointers start at 0 and never decrease, column indices lie in
+// [0, N).  A thread reads col only inside its own row's extent after checking that the extent lies inside
+// [0, rowptr[N]], the length the caller vouches for.  Any violation sets *bad.
+__global__ void __launch_bounds__(256)
+check_graph_kernel(int32_t N, const int32_t* __restrict__ rowptr, const int32_t* __restrict__ col, int* __restrict__ bad)
+{
+    const int32_t E = rowptr[N];
+    if (blockIdx.x == 0 && threadIdx.x == 0 && (rowptr[0] != 0 || E < 0)) *bad = 1;
+    for (int32_t i = blockIdx.x * blockDim.x + threadIdx.x; i < N; i += gridDim.x * blockDim.x) {
+        const int32_t beg = rowptr[i], end = rowptr[i + 1];
+        if (beg < 0 || end < beg || end > E) { *bad = 1; continue; }
+        for (int32_t p = beg; p < end; ++p) {
+            const int32_t c = col[p];
+            if (c < 0 || c >= N) *bad = 1;
+        }
+    }
+}
+
 size_t walk_smem_per_warp(const grf_walk_params& P)
 {
     const size_t key_slots = (1 << P.seq_bits) < 32 ? 32 : (size_t)(1 << P.seq_bits);
@@ -480,6 +498,15 @@ extern "C" int grf_sample(grf_ctx* ctx, int32_t N, const int32_t* rowptr, const 
     grf_walk_params P;
     GRF_TRY(grf_walk_params_init(&P, N, seed, n_walks, p_halt, max_len, f_phi, f_psi));
     GRF_CUDA_TRY(cudaSetDevice(ctx->device));
+    if (ctx->check_graphs) {
+        // debugging aid: one pass over the graph and one wait for the device before any walk is taken
+        GRF_CUDA_TRY(cudaMemsetAsync(ctx->error_word + 1, 0, sizeof(int), ctx->stream));
+        check_graph_kernel<<<grf_ceil_div(N, 256) > 1184 ? 1184 : grf_ceil_div(N, 256), 256, 0, ctx->stream>>>(
+            N, rowptr, col, ctx->error_word + 1);
+        GRF_CUDA_TRY(cudaMemcpyAsync(ctx->pinned + 9, ctx->error_word + 1, sizeof(int), cudaMemcpyDeviceToHost, ctx->stream));
+        GRF_CUDA_TRY(cudaStreamSynchronize(ctx->stream));
+        if (ctx->pinned[9] != 0) return GRF_ERR_BADGRAPH;
+    }
     grf_features* feat = *inout;
     if (!feat) {
         feat = new (std::nothrow) grf_features();

@@ -384,3 +384,32 @@ def test_deconvolve_matches_oracle(lib):
     api, B, ctx = lib
     for w in (configs.tiny(), configs.vit_grid()):
         assert np.allclose(B.grf_deconvolve(w.alpha), oracle.deconvolve(w.alpha), rtol=1e-14, atol=0)
+
+
+def test_device_graph_check_rejects_inconsistent_graphs(lib):
+    """With grf_ctx_check_graphs on, a device-resident graph is validated by a kernel before any walk: a
+    decreasing row pointer, a column index out of range and a non-zero first row pointer are all refused."""
+    api, B, ctx = lib
+    w = configs.tiny()
+    g = w.graph()
+    f = oracle.deconvolve(w.alpha).astype(np.float32)
+    B.grf_ctx_check_graphs(ctx.handle, True)
+    try:
+        good = api.sample(ctx, api.DeviceGraph(g), 1, w.n_walks, w.p_halt, w.max_len, f)
+        good.free()
+        for kind in ("rowptr_decreases", "col_too_large", "col_negative", "rowptr0"):
+            dg = api.DeviceGraph(g)
+            if kind == "rowptr_decreases":
+                dg.rowptr[5] = dg.rowptr[4] - 1
+            elif kind == "col_too_large":
+                dg.col[7] = g.N
+            elif kind == "col_negative":
+                dg.col[3] = -2
+            else:
+                dg.rowptr[0] = 1
+            with pytest.raises(B.GrfError) as e:
+                api.sample(ctx, dg, 1, w.n_walks, w.p_halt, w.max_len, f)
+            assert e.value.code == B.GRF_ERR_BADGRAPH, kind
+    finally:
+        B.grf_ctx_check_graphs(ctx.handle, False)
+    B.grf_ctx_check(ctx.handle)
