@@ -312,12 +312,13 @@ mask_rows_kernel(int32_t Nk, const int32_t* __restrict__ rows, const int32_t* __
 }
 
 // ---------------------------------------------------------------------------------------------------
-// The attention kernel.  warps 0-3: row threads (one query = one tensor-memory lane each); warp 4: producer
-// (gathers of key-feature and value rows); warp 5: MMA issuer.
+// The attention kernel.  warps 0-3: row threads (one query = one tensor-memory lane each); warp 4: MMA issuer;
+// warps 5-8: producers (gathers of key-feature and value rows, a quarter of every tile each: a thread's
+// tensor-map gathers are issued one after the other, so they are spread over sixteen threads of four warps).
 
 template <int M> struct MhShape {
     static constexpr int D = 64;
-    static constexpr int NS = 4;                          // key/value stages in flight
+    static constexpr int NS = M <= 32 ? 8 : 6;            // key/value stages in flight
     static constexpr int V_BYTES = KT * 128;              // 64 gathered value rows, 128-byte swizzle
     static constexpr int K_BYTES = KT * M * 2;            // [M/8][KT keys][8] bf16: K-major, unswizzled
     static constexpr int STAGE = V_BYTES + K_BYTES;
@@ -329,7 +330,7 @@ template <int M> struct MhShape {
     static_assert(STAGE % 1024 == 0, "stages must keep the swizzle phase");
 };
 
-constexpr int MH_THREADS = 192;
+constexpr int MH_THREADS = 288;          // warps 0-3: row threads; warp 4: MMA issuer; warps 5-8: producers
 
 template <int M>
 __global__ void __launch_bounds__(MH_THREADS)
@@ -363,14 +364,14 @@ mhat_attention_kernel(int32_t G, int32_t nblocks, int32_t N, const int32_t* __re
     const uint32_t drain_bar = bar_base + 8u * (uint32_t)(2 * NS + 7);
 
     if (tid == 0) {
-        for (int s = 0; s < NS; ++s) { mbar_init(kv_full(s), 2); mbar_init(kv_empty(s), 1); }
+        for (int s = 0; s < NS; ++s) { mbar_init(kv_full(s), 8); mbar_init(kv_empty(s), 1); }
         for (int b = 0; b < 2; ++b) { mbar_init(s_full(b), 1); mbar_init(p_full(b), 4); mbar_init(s_free(b), 1); }
         mbar_init(acc_done, 1);
         mbar_init(drain_bar, 1);
         abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    if (warp == 5) tmem_alloc(&tmem_slot, (uint32_t)Sh::TMEM_COLS);
+    if (warp == 4) tmem_alloc(&tmem_slot, (uint32_t)Sh::TMEM_COLS);
     // the block's queries in the K-major operand layout: 16-byte chunk c of row r at (c * 128 + r) * 16
     if (tid < BQ) {
         const int32_t row = blk * BQ + tid;
@@ -465,15 +466,18 @@ mhat_attention_kernel(int32_t G, int32_t nblocks, int32_t N, const int32_t* __re
                 dst[1] = make_uint4(w[4], w[5], w[6], w[7]);
             }
         }
-    } else if (warp == 4) {
-        // ------------------------------------------------------------ producer: gathers of a tile's 64 keys
-        // Lane x holds keys x and x + 32 of the tile.  Value rows: lanes 0-15 each gather four rows through the
-        // tensor map (they land in the swizzled layout and complete on the stage's barrier by byte count).
-        // Key-feature rows: every lane copies its two keys' rows in 16-byte pieces, piece c of key y going to
-        // (c * 64 + y) * 16; the lane's copies of one tile form one group, and a stage is handed over one tile
-        // late, after its group has completed and a proxy fence.
+    } else if (warp >= 5) {
+        // ------------------------------------------------------------ producers: warp w takes keys 16w .. 16w+15 of every tile
+        // Lanes x and x + 16 hold key x of the warp's sixteen.  Value rows: lanes 0-3 each gather four rows through
+        // the tensor map (they land in the swizzled layout and complete on the stage's barrier by byte count).
+        // Key-feature rows: 16-byte pieces, piece c of key y going to (c * 64 + y) * 16; lanes 0-15 copy the even
+        // pieces, lanes 16-31 the odd ones.  A warp's copies of one tile form one group; it hands its part of a
+        // stage over two tiles late, after that group has completed and a proxy fence.  Key indices are read one
+        // tile ahead.
+        const int pw = warp - 5;
         const __nv_bfloat16* Kg = phiK + (size_t)g * N * M;
         const int32_t row0 = g * N;
+        const int ky = pw * 16 + (lane & 15);                   // this lane's key within the tile
         bool ok = true;
         int32_t issued = 0;
         auto hand_over = [&](int32_t t) {
@@ -481,43 +485,44 @@ mhat_attention_kernel(int32_t G, int32_t nblocks, int32_t N, const int32_t* __re
             __syncwarp();
             if (lane == 0) mbar_arrive(kv_full(t % NS));
         };
+        int32_t kn = T > 0 ? __ldg(mk_key + off + ky) : 0;
         for (int32_t t = 0; t < T; ++t) {
             const int s = t % NS;
+            const int32_t k = kn;
+            if (t + 1 < T) kn = __ldg(mk_key + off + (t + 1) * KT + ky);
             if (t >= NS && !mbar_wait(kv_empty(s), (uint32_t)(t / NS - 1) & 1u, &abort_flag)) ok = false;
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
-            const int32_t k0 = __ldg(mk_key + off + t * KT + lane), k1 = __ldg(mk_key + off + t * KT + 32 + lane);
             const uint32_t v_st = stage_base + (uint32_t)s * Sh::STAGE, k_st = v_st + Sh::V_BYTES;
-            if (lane == 0) mbar_expect_tx(kv_full(s), (uint32_t)Sh::V_BYTES);
-            __syncwarp();
+            expect_tx_elected(kv_full(s), (uint32_t)Sh::V_BYTES / 4);
             int32_t r4[4];
 #pragma unroll
-            for (int e = 0; e < 4; ++e) {
-                const int32_t key = 4 * (lane & 15) + e;
-                const int32_t a = __shfl_sync(0xffffffffu, k0, key & 31), b = __shfl_sync(0xffffffffu, k1, key & 31);
-                r4[e] = row0 + (key < 32 ? a : b);
-            }
-            if (lane < 16) tma_gather4(v_st + (uint32_t)lane * 512u, &map_v, r4[0], r4[1], r4[2], r4[3], kv_full(s));
+            for (int e = 0; e < 4; ++e) r4[e] = row0 + __shfl_sync(0xffffffffu, k, (4 * (lane & 3) + e) & 31);
+            if (lane < 4) tma_gather4(v_st + (uint32_t)(pw * 4 + lane) * 512u, &map_v, r4[0], r4[1], r4[2], r4[3], kv_full(s));
 #pragma unroll
-            for (int c = 0; c < M / 8; ++c) {
+            for (int c2 = 0; c2 < M / 16; ++c2) {
+                const int c = 2 * c2 + (lane >> 4);
                 asm volatile("cp.async.ca.shared.global [%0], [%1], 16;"
-                             ::"r"(k_st + (uint32_t)(c * KT + lane) * 16u), "l"(Kg + (size_t)k0 * M + c * 8) : "memory");
-                asm volatile("cp.async.ca.shared.global [%0], [%1], 16;"
-                             ::"r"(k_st + (uint32_t)(c * KT + 32 + lane) * 16u), "l"(Kg + (size_t)k1 * M + c * 8) : "memory");
+                             ::"r"(k_st + (uint32_t)(c * KT + ky) * 16u), "l"(Kg + (size_t)k * M + c * 8) : "memory");
             }
             asm volatile("cp.async.commit_group;" ::: "memory");
             issued = t + 1;
-            if (t >= 1) {
-                asm volatile("cp.async.wait_group 1;" ::: "memory");
-                hand_over(t - 1);
+            if (t >= 2) {
+                asm volatile("cp.async.wait_group 2;" ::: "memory");
+                hand_over(t - 2);
             }
+        }
+        if (ok && T >= 2) {
+            asm volatile("cp.async.wait_group 1;" ::: "memory");
+            hand_over(T - 2);
         }
         asm volatile("cp.async.wait_group 0;" ::: "memory");
         if (ok && T > 0) hand_over(T - 1);
         if (!ok) {
-            // gave up: let the gathers still in flight land (bounded) before the CTA's shared memory is released
+            // gave up: the last two tiles issued never got this warp's second arrival; then let the gathers still
+            // in flight land (bounded) before the CTA's shared memory is released
             for (int32_t t = issued > NS ? issued - NS : 0; t < issued; ++t) {
-                if (lane == 0 && t == issued - 1) mbar_arrive(kv_full(t % NS));   // its second arrival never came
+                if (lane == 0 && t >= issued - 2) mbar_arrive(kv_full(t % NS));
                 __syncwarp();
                 mbar_drain(kv_full(t % NS), (uint32_t)(t / NS) & 1u, 20000000ll);
             }
@@ -568,7 +573,7 @@ mhat_attention_kernel(int32_t G, int32_t nblocks, int32_t N, const int32_t* __re
 
     fence_before_sync();
     __syncthreads();
-    if (warp == 5) tmem_dealloc(tmem_base, (uint32_t)Sh::TMEM_COLS);
+    if (warp == 4) tmem_dealloc(tmem_base, (uint32_t)Sh::TMEM_COLS);
     if (tid == 0 && abort_flag) atomicExch(error_word, 1);
 }
 
