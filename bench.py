@@ -449,7 +449,12 @@ def measure(args, workload_name, route, with_cpu_baseline, with_e2e, frozen=Fals
         traffic = None
         c = counters.get(dom)
         if c and not c["stale"] and c["workload"] == w.name.split("-heads")[0]:
-            traffic = c["dram_bytes"] * (w.G / c["heads"] if dom != "walk_merge" else 1.0)
+            if dom in ("walk_merge", "mask_build"):            # independent of the head count
+                traffic = c["dram_bytes"]
+            elif dom == "mhat_attention":                      # the mask is read once whatever the head count: no scaling rule
+                traffic = c["dram_bytes"] if w.G == c["heads"] else None
+            else:
+                traffic = c["dram_bytes"] * w.G / c["heads"]
         binds = binding.get(dom, {}).get("binds")
         bound = {"tensor_issue": "tensor", "hbm": "hbm", "integer_issue": "alu"}.get(binds, "hbm" if binds is None else "smem")
         step_text = {"sz": "grf_sample (both ensembles) + grf_masked_linear_attn",
