@@ -84,6 +84,50 @@ def test_bench_workload_asymmetric_route_sampled_rows():
     ctx.close()
 
 
+def test_bench_workload_materialised_mask_route_sampled_rows():
+    """Eqs. 1-2 over the materialised mask at the bench size and launch configuration: sampled rows of the stored mask
+    against the oracle's rows of Phi Psi^T, and sampled query rows of the attention against the brute force."""
+    from paper_2410_03462_b200 import api, binding as B
+    w = configs.point_cloud_32768()
+    g = w.graph()
+    ctx = api.Context(0)
+    f = oracle.deconvolve(w.alpha).astype(np.float32)
+    feat = api.sample(ctx, api.DeviceGraph(g), configs.WALK_SEED, w.n_walks, w.p_halt, w.max_len, f)
+    Phi, Psi, PsiT, _, _ = helpers.oracle_features(w, g, configs.WALK_SEED, f)
+    B.grf_features_materialise(ctx.handle, feat.handle)
+    B.grf_ctx_check(ctx.handle)
+    rng = np.random.default_rng(8)
+    rows = np.unique(np.concatenate([[0, 127, 128, g.N - 1], rng.integers(0, g.N, 260)]))
+    assert len(rows) >= 256
+    Mrows = oracle.mask_rows(Phi, Psi, rows)
+    r_dev = torch.tensor(rows, dtype=torch.int32, device="cuda")
+    got = torch.empty((len(rows), g.N), dtype=torch.float32, device="cuda")
+    B.grf_mask_rows(ctx.handle, feat.handle, len(rows), r_dev, got)
+    torch.cuda.synchronize()
+    got = got.cpu().numpy().astype(np.float64)
+    # one bf16 rounding of an fp32 sum of non-negative terms; values below the bf16 normal range may flush to zero
+    assert (np.abs(got - Mrows) <= 2.0 ** -8 * np.abs(Mrows) + 1e-37).all()
+    assert ((got != 0) <= (Mrows != 0)).all()
+    q, k, v = tensors.qkv(w.G, g.N, w.m, w.d, w.dtype, configs.QKV_SEED)
+    qd, kd, vd = q.cuda(), k.cuda(), v.cuda()
+    ref = oracle.attn_bruteforce(tensors.widen(q), tensors.widen(k), tensors.widen(v), Mrows_full(Mrows, rows, g.N), rows=rows)
+    out, den = api.masked_attn_mhat(ctx, feat, qd, kd, vd, want_den=True)
+    B.grf_ctx_check(ctx.handle)
+    helpers.assert_attn_close(out[:, rows].float().cpu().numpy(), ref, helpers.TOL["bf16"], den[:, rows].cpu().numpy(),
+                              "full size, materialised mask", same_sign=True)
+    assert torch.isfinite(out.float()).all() and (den > 0).all()
+    out2 = api.masked_attn_mhat(ctx, feat, qd, kd, vd)
+    torch.cuda.synchronize()
+    assert torch.equal(out, out2)
+    # and against the route through the per-node states on the same features (two roundings apart)
+    out_sz = api.masked_linear_attn(ctx, feat, qd, kd, vd)
+    torch.cuda.synchronize()
+    a, b = out.float(), out_sz.float()
+    assert ((a - b).abs() <= 4e-2 * (a.abs() + b.abs()) / 2 + 4e-2 * ref["num_abs"].max() / ref["den"].min()).all()
+    feat.free()
+    ctx.close()
+
+
 def Mrows_full(Mrows, rows, N):
     """attn_bruteforce indexes the mask by absolute row: place the sampled rows into an N x N frame lazily."""
     class _Rows:
