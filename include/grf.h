@@ -254,6 +254,12 @@ int grf_step_host(grf_ctx* ctx, int32_t N, const int32_t* rowptr, const int32_t*
  * profilers' timelines; that costs nothing when no tool is attached. */
 int grf_ctx_check_graphs(grf_ctx* ctx, int enable);
 
+/* Self-test of the bounded waits inside the tensor-core kernels: launches one warp that waits, with the kernels' own
+ * wait routine and a limit of `limit_cycles` GPU clock cycles (1 .. 2e9), for a barrier that nothing arrives at.  The
+ * wait gives up and raises the context's error word, so the next grf_ctx_check returns GRF_ERR_TIMEOUT; the device
+ * stays usable.  Asynchronous. */
+int grf_debug_wait_timeout(grf_ctx* ctx, int64_t limit_cycles);
+
 /* Waits for the context's stream and reports whether any kernel since the previous check gave up one of its
  * bounded waits (GRF_ERR_TIMEOUT; the affected outputs are invalid), else GRF_OK. */
 int grf_ctx_check(grf_ctx* ctx);

@@ -54,6 +54,7 @@ _SIGNATURES = {
     "grf_plan_stats": (_int, [_vp, _vp, ctypes.POINTER(_i32), ctypes.POINTER(_i64)]),
     "grf_ctx_launch_count": (_i64, [_vp]),
     "grf_ctx_check": (_int, [_vp]),
+    "grf_debug_wait_timeout": (_int, [_vp, _i64]),
     "grf_ctx_check_graphs": (_int, [_vp, _int]),
     "grf_ctx_use_tensor_cores": (_int, [_vp, _int]),
     "grf_ctx_enable_timing": (_int, [_vp, _int]),
@@ -129,6 +130,10 @@ def grf_ctx_launch_count(ctx: int) -> int:
 
 def grf_ctx_check(ctx: int):
     _check(lib.grf_ctx_check(ctx), "grf_ctx_check")
+
+
+def grf_debug_wait_timeout(ctx: int, limit_cycles: int):
+    _check(lib.grf_debug_wait_timeout(ctx, limit_cycles), "grf_debug_wait_timeout")
 
 
 def grf_ctx_check_graphs(ctx: int, enable: bool):

@@ -364,6 +364,23 @@ row_denominators_kernel(int32_t G, int32_t N, int32_t R, const int32_t* __restri
 }
 
 // ---------------------------------------------------------------------------------------------------
+// Self-test of the bounded waits: a barrier that nothing ever arrives at is waited for with the kernels' own wait
+// routine and a short limit; the wait must give up, raise the CTA's flag and the context's error word.
+__global__ void __launch_bounds__(32) wait_timeout_probe_kernel(long long limit_cycles, int* __restrict__ error_word)
+{
+    __shared__ __align__(8) unsigned long long bar;
+    __shared__ int abort_flag;
+    if (threadIdx.x == 0) {
+        mbar_init(smem_u32(&bar), 1);
+        abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncwarp();
+    const bool ok = mbar_wait(smem_u32(&bar), 0u, &abort_flag, limit_cycles);
+    if (!__all_sync(0xffffffffu, ok) && threadIdx.x == 0 && abort_flag) atomicExch(error_word, 1);
+}
+
+// ---------------------------------------------------------------------------------------------------
 // Block plan: for every block of BQ consecutive rows of Phi, the sorted list of distinct columns.
 
 __global__ void __launch_bounds__(256)
@@ -541,6 +558,15 @@ int grf_build_block_plan(grf_ctx* ctx, grf_features* feat)
     feat->plan_entries = (int64_t)entries;
     feat->plan_ready = true;
     return GRF_OK;
+}
+
+extern "C" int grf_debug_wait_timeout(grf_ctx* ctx, int64_t limit_cycles)
+{
+    if (!ctx || limit_cycles < 1 || limit_cycles > 2000000000ll) return GRF_ERR_INVALID;
+    GRF_CUDA_TRY(cudaSetDevice(ctx->device));
+    wait_timeout_probe_kernel<<<1, 32, 0, ctx->stream>>>((long long)limit_cycles, ctx->error_word);
+    ctx->launches += 1;
+    return cudaGetLastError() == cudaSuccess ? GRF_OK : GRF_ERR_CUDA;
 }
 
 extern "C" int grf_plan_stats(grf_ctx* ctx, const grf_features* feat, int32_t* blocks, int64_t* entries)

@@ -35,7 +35,8 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
 }
 // Bounded wait: false when another thread of the CTA has given up or when this wait lasted too long
 // (then it raises the CTA's abort flag itself).
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag)
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+                                          long long limit_cycles = WAIT_CYCLES)
 {
     long long t0 = 0;
     for (uint32_t it = 0;; ++it) {
@@ -44,7 +45,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
             if (*abort_flag) return false;
             const long long now = clock64();
             if (t0 == 0) t0 = now;
-            else if (now - t0 > WAIT_CYCLES) { *abort_flag = 1; return false; }
+            else if (now - t0 > limit_cycles) { *abort_flag = 1; return false; }
         }
     }
 }

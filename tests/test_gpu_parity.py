@@ -413,3 +413,18 @@ def test_device_graph_check_rejects_inconsistent_graphs(lib):
     finally:
         B.grf_ctx_check_graphs(ctx.handle, False)
     B.grf_ctx_check(ctx.handle)
+
+
+def test_bounded_wait_gives_up_and_reports_timeout(lib):
+    """A wait for a barrier that nothing arrives at runs out after its limit (here about a millisecond), the error
+    word is raised, grf_ctx_check reports GRF_ERR_TIMEOUT once, and the context keeps working afterwards."""
+    api, B, ctx = lib
+    B.grf_ctx_check(ctx.handle)
+    B.grf_debug_wait_timeout(ctx.handle, 2_000_000)
+    with pytest.raises(B.GrfError) as e:
+        B.grf_ctx_check(ctx.handle)
+    assert e.value.code == B.GRF_ERR_TIMEOUT
+    B.grf_ctx_check(ctx.handle)                       # the word was cleared
+    w = configs.tiny()
+    _attn_case(lib, w, w.graph(), 1, same_sign=True)   # and the device is as usable as before
+    B.grf_ctx_check(ctx.handle)
