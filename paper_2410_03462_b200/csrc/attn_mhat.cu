@@ -291,6 +291,232 @@ mask_values_kernel(int32_t N, int32_t Nk, const int32_t* __restrict__ phi_rowptr
     }
 }
 
+// ---------------------------------------------------------------------------------------------------
+// The same sums with the positions looked up once per (block, node) instead of once per (row, node): a node of a
+// block's list is used by nine of the block's rows on average, and the look-up (two shared-memory reads and a
+// population count per key) was most of the work of every addition.
+//   mask_node_offsets_kernel  per block: where each node's positions start (running sum of the lengths of the
+//                             nodes' rows of Psi^T over the block's list) and the block's total;
+//   mask_positions_kernel     per block: the position in the block's key list of every key of every node of the
+//                             list (16 bits each), and for every non-zero Phi_il of the block's rows where the
+//                             positions of node l start;
+//   mask_values_pos_kernel    the row-by-row accumulation, reading positions instead of keys.
+
+__global__ void __launch_bounds__(256)
+mask_node_offsets_kernel(const int32_t* __restrict__ plan_off, const int32_t* __restrict__ plan_cnt,
+                         const int32_t* __restrict__ plan_col, const int32_t* __restrict__ t_rowptr,
+                         int32_t* __restrict__ node_off, int32_t* __restrict__ blk_total,
+                         const int32_t* __restrict__ mk_cnt, int32_t* __restrict__ longest_list)
+{
+    __shared__ int32_t warp_sums[8];
+    __shared__ int32_t carry_s;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int32_t blk = blockIdx.x;
+    const int32_t uoff = plan_off[blk], ucnt = plan_cnt[blk];
+    if (tid == 0) carry_s = 0;
+    __syncthreads();
+    for (int32_t base = 0; base < ucnt; base += 256) {
+        const int32_t u = base + tid;
+        int32_t len = 0;
+        if (u < ucnt) {
+            const int32_t l = plan_col[uoff + u];
+            len = t_rowptr[l + 1] - t_rowptr[l];
+        }
+        int32_t inc = len;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const int32_t y = __shfl_up_sync(0xffffffffu, inc, o);
+            if (lane >= o) inc += y;
+        }
+        if (lane == 31) warp_sums[warp] = inc;
+        __syncthreads();
+        int32_t before = carry_s + inc - len;
+        for (int w = 0; w < warp; ++w) before += warp_sums[w];
+        if (u < ucnt) node_off[uoff + u] = before;
+        __syncthreads();
+        if (tid == 255) carry_s = before + len;
+        __syncthreads();
+    }
+    if (tid == 0) {
+        blk_total[blk] = carry_s;
+        atomicMax(longest_list, mk_cnt[blk]);        // positions are kept in 16 bits: the host checks this
+    }
+}
+
+__global__ void __launch_bounds__(256)
+mask_positions_kernel(int32_t N, int32_t Nk, int32_t R, const int32_t* __restrict__ phi_rowptr,
+                      const int32_t* __restrict__ phi_col, const int32_t* __restrict__ plan_off,
+                      const int32_t* __restrict__ plan_cnt, const int32_t* __restrict__ plan_col,
+                      const int32_t* __restrict__ t_rowptr, const int32_t* __restrict__ t_col,
+                      const uint32_t* __restrict__ bits, const int32_t* __restrict__ node_off,
+                      const int32_t* __restrict__ blk_pos, unsigned short* __restrict__ pos16, int32_t* __restrict__ phi_pos)
+{
+    extern __shared__ uint32_t smem_pos[];      // key bitmap, its prefix counts, node bitmap, its prefix counts
+    __shared__ int32_t warp_sums[8];
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int32_t blk = blockIdx.x;
+    const int32_t wk = (Nk + 31) >> 5, wr = (R + 31) >> 5;
+    uint32_t* kbits = smem_pos;
+    int32_t* kbefore = reinterpret_cast<int32_t*>(smem_pos + wk);
+    uint32_t* nbits = smem_pos + 2 * wk;
+    int32_t* nbefore = reinterpret_cast<int32_t*>(smem_pos + 2 * wk + wr);
+    const uint32_t* src = bits + (size_t)blk * 2 * wk;
+    for (int32_t x = tid; x < wk; x += 256) { kbits[x] = src[x]; kbefore[x] = (int32_t)src[wk + x]; }
+    for (int32_t x = tid; x < wr; x += 256) nbits[x] = 0u;
+    __syncthreads();
+    const int32_t uoff = plan_off[blk], ucnt = plan_cnt[blk];
+    const int32_t* ulist = plan_col + uoff;
+    for (int32_t u = tid; u < ucnt; u += 256) {
+        const int32_t l = ulist[u];
+        atomicOr(&nbits[l >> 5], 1u << (l & 31));
+    }
+    __syncthreads();
+    {
+        const int32_t per = (wr + 255) / 256;
+        const int32_t w0 = min(wr, tid * per), w1 = min(wr, w0 + per);
+        int32_t mine = 0;
+        for (int32_t x = w0; x < w1; ++x) mine += __popc(nbits[x]);
+        int32_t inc = mine;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const int32_t y = __shfl_up_sync(0xffffffffu, inc, o);
+            if (lane >= o) inc += y;
+        }
+        if (lane == 31) warp_sums[warp] = inc;
+        __syncthreads();
+        int32_t run = inc - mine;
+        for (int w = 0; w < warp; ++w) run += warp_sums[w];
+        for (int32_t x = w0; x < w1; ++x) { nbefore[x] = run; run += __popc(nbits[x]); }
+    }
+    __syncthreads();
+    const int32_t base = blk_pos[blk];
+    // positions of the keys of every node of the list
+    for (int32_t u = warp; u < ucnt; u += 8) {
+        const int32_t l = __ldg(ulist + u);
+        const int32_t rb = __ldg(t_rowptr + l), re = __ldg(t_rowptr + l + 1);
+        unsigned short* dst = pos16 + (size_t)base + node_off[uoff + u];
+        for (int32_t q = rb + lane; q < re; q += 32) {
+            const int32_t j = __ldg(t_col + q);
+            dst[q - rb] = (unsigned short)(kbefore[j >> 5] + __popc(kbits[j >> 5] & ((1u << (j & 31)) - 1u)));
+        }
+    }
+    // where the positions of its node start, for every non-zero of the block's rows of Phi (the list holds a node
+    // once, apart from the padding at its end, which repeats the last node: the first occurrence counts)
+    const int32_t r0 = blk * BQ, r1 = min(N, r0 + BQ);
+    for (int32_t p = phi_rowptr[r0] + tid; p < phi_rowptr[r1]; p += 256) {
+        const int32_t l = __ldg(phi_col + p);
+        const int32_t u = nbefore[l >> 5] + __popc(nbits[l >> 5] & ((1u << (l & 31)) - 1u));
+        phi_pos[p] = base + node_off[uoff + u];
+    }
+}
+
+struct MaskPosGroup {                   // the keys of four nodes l, up to 128 each: lane x holds keys x, x+32, x+64, x+96
+    int32_t ps[4][4];
+    float v[4][4];
+    int32_t len[4], beg[4], pbeg[4];
+};
+
+__global__ void __launch_bounds__(MASK_WARPS * 32)
+mask_values_pos_kernel(int32_t N, const int32_t* __restrict__ phi_rowptr, const int32_t* __restrict__ phi_col,
+                       const float* __restrict__ phi_val, const int32_t* __restrict__ phi_pos,
+                       const int32_t* __restrict__ t_rowptr, const float* __restrict__ t_val,
+                       const unsigned short* __restrict__ pos16, const int32_t* __restrict__ mk_off,
+                       const int32_t* __restrict__ mk_cnt, __nv_bfloat16* __restrict__ mk_val)
+{
+    extern __shared__ float smem_acc[];         // the warps' accumulators
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    constexpr int GROUPS = BQ / MASK_ROWS;
+    const int32_t nblocks = (N + BQ - 1) / BQ;
+    const int32_t blk = mk_cnt[nblocks + blockIdx.x / GROUPS];     // blocks by decreasing key count
+    const int32_t rg = blockIdx.x % GROUPS;
+    float* acc = smem_acc + (size_t)warp * MASK_SEG;
+    const int32_t off = mk_off[blk], cnt = mk_cnt[blk];
+    for (int32_t x = lane; x < MASK_SEG; x += 32) acc[x] = 0.0f;
+    __syncwarp();
+    const int32_t r0 = blk * BQ;
+    for (int32_t seg0 = 0; seg0 < cnt; seg0 += MASK_SEG) {
+        const int32_t seglen = min(MASK_SEG, cnt - seg0);       // a multiple of the tile, hence of 8
+        for (int32_t rr = rg * MASK_ROWS + warp; rr < (rg + 1) * MASK_ROWS; rr += MASK_WARPS) {
+            const int32_t r = r0 + rr;
+            if (r < N) {
+                const int32_t pbeg = phi_rowptr[r], pend = phi_rowptr[r + 1];
+                for (int32_t p0 = pbeg; p0 < pend; p0 += 32) {
+                    // 32 non-zeros of the row at a time: lane x holds Phi_il, the start and length of row l_x of Psi^T
+                    // and the start of node l_x's positions
+                    const int32_t n = min(32, pend - p0);
+                    const int32_t my_l = lane < n ? __ldg(phi_col + p0 + lane) : 0;
+                    const float my_phi = lane < n ? __ldg(phi_val + p0 + lane) : 0.0f;
+                    const int32_t my_pbeg = lane < n ? __ldg(phi_pos + p0 + lane) : 0;
+                    const int32_t my_beg = lane < n ? __ldg(t_rowptr + my_l) : 0;
+                    const int32_t my_len = lane < n ? __ldg(t_rowptr + my_l + 1) - my_beg : 0;
+                    auto fetch = [&](int32_t e0, MaskPosGroup& gq) {
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {
+                            gq.beg[e] = __shfl_sync(0xffffffffu, my_beg, (e0 + e) & 31);
+                            gq.pbeg[e] = __shfl_sync(0xffffffffu, my_pbeg, (e0 + e) & 31);
+                            gq.len[e] = e0 + e < n ? __shfl_sync(0xffffffffu, my_len, (e0 + e) & 31) : 0;
+#pragma unroll
+                            for (int sl = 0; sl < 4; ++sl) {
+                                const int32_t x = sl * 32 + lane;
+                                const bool valid = x < gq.len[e];
+                                gq.ps[e][sl] = valid ? (int32_t)__ldg(pos16 + (size_t)gq.pbeg[e] + x) : -1;
+                                gq.v[e][sl] = valid ? __ldg(t_val + gq.beg[e] + x) : 0.0f;
+                            }
+                        }
+                    };
+                    auto add = [&](int32_t e0, MaskPosGroup& gq) {
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {
+                            const float phi = __shfl_sync(0xffffffffu, my_phi, (e0 + e) & 31);
+                            float a[4];
+                            int32_t ps[4];
+                            // one node's keys are distinct: a lane's four additions go side by side
+#pragma unroll
+                            for (int sl = 0; sl < 4; ++sl) {
+                                const int32_t x = gq.ps[e][sl] - seg0;
+                                ps[sl] = (gq.ps[e][sl] >= 0 && x >= 0 && x < seglen) ? x : -1;
+                                a[sl] = ps[sl] >= 0 ? acc[ps[sl]] : 0.0f;
+                            }
+#pragma unroll
+                            for (int sl = 0; sl < 4; ++sl)
+                                if (ps[sl] >= 0) acc[ps[sl]] = fmaf(phi, gq.v[e][sl], a[sl]);
+                            for (int32_t x = 128 + lane; x < gq.len[e]; x += 32) {      // nodes with more than 128 keys
+                                const int32_t y = (int32_t)__ldg(pos16 + (size_t)gq.pbeg[e] + x) - seg0;
+                                if (y >= 0 && y < seglen) acc[y] = fmaf(phi, __ldg(t_val + gq.beg[e] + x), acc[y]);
+                            }
+                            __syncwarp();
+                        }
+                    };
+                    MaskPosGroup ga, gb;
+                    fetch(0, ga);
+                    for (int32_t e0 = 0; e0 < n; e0 += 8) {
+                        if (e0 + 4 < n) fetch(e0 + 4, gb);
+                        add(e0, ga);
+                        if (e0 + 4 < n) {
+                            if (e0 + 8 < n) fetch(e0 + 8, ga);
+                            add(e0 + 4, gb);
+                        }
+                    }
+                }
+            }
+            // the row's values of this segment, eight keys (16 bytes) per lane at a time; the accumulators are
+            // cleared for the next row as they are read
+            for (int32_t c8 = lane; c8 < seglen / 8; c8 += 32) {
+                float4* a4 = reinterpret_cast<float4*>(acc + c8 * 8);
+                const float4 x0 = a4[0], x1 = a4[1];
+                a4[0] = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+                a4[1] = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+                const __nv_bfloat162 h0 = __floats2bfloat162_rn(x0.x, x0.y), h1 = __floats2bfloat162_rn(x0.z, x0.w);
+                const __nv_bfloat162 h2 = __floats2bfloat162_rn(x1.x, x1.y), h3 = __floats2bfloat162_rn(x1.z, x1.w);
+                uint4* dst = reinterpret_cast<uint4*>(mk_val + ((size_t)((off + seg0) / 8 + c8) * BQ + rr) * 8);
+                *dst = make_uint4(*reinterpret_cast<const uint32_t*>(&h0), *reinterpret_cast<const uint32_t*>(&h1),
+                                  *reinterpret_cast<const uint32_t*>(&h2), *reinterpret_cast<const uint32_t*>(&h3));
+            }
+            __syncwarp();
+        }
+    }
+}
+
 // Dense rows of the mask for checking and export: out[x][j] = Mhat[rows[x]][j] (zeros elsewhere), one CTA per row.
 __global__ void __launch_bounds__(256)
 mask_rows_kernel(int32_t Nk, const int32_t* __restrict__ rows, const int32_t* __restrict__ mk_off,
@@ -584,7 +810,8 @@ void grf_mask_invalidate(grf_features* feat) { feat->mask.ready = false; }
 void grf_mask_release(grf_features* feat)
 {
     grf_mask_dev& K = feat->mask;
-    grf_buf_release(&K.off); grf_buf_release(&K.cnt); grf_buf_release(&K.key); grf_buf_release(&K.bits); grf_buf_release(&K.val);
+    grf_buf_release(&K.off); grf_buf_release(&K.cnt); grf_buf_release(&K.key); grf_buf_release(&K.bits); grf_buf_release(&K.val); grf_buf_release(&K.node_off);
+    grf_buf_release(&K.blk_pos); grf_buf_release(&K.pos16); grf_buf_release(&K.phi_pos);
     K.ready = false;
 }
 
@@ -617,9 +844,30 @@ extern "C" int grf_features_materialise(grf_ctx* ctx, grf_features* feat)
     GRF_TRY(grf_exclusive_scan(ctx, (const int32_t*)K.cnt.ptr, (int32_t*)K.off.ptr, nblocks, 1));
     GRF_CUDA_TRY(cudaMemcpyAsync(ctx->pinned + 5, (const int32_t*)K.off.ptr + nblocks, sizeof(int32_t),
                                  cudaMemcpyDeviceToHost, ctx->stream));
+    // where every node's key positions will start (per block, then over the blocks), and the longest key list
+    const int32_t R = feat->psit.rows;
+    GRF_TRY(grf_buf_reserve(&K.node_off, sizeof(int32_t) * (size_t)(feat->plan_entries > 0 ? feat->plan_entries : 1)));
+    GRF_TRY(grf_buf_reserve(&K.blk_pos, sizeof(int32_t) * (2 * (size_t)nblocks + 2)));
+    int32_t* blk_pos = (int32_t*)K.blk_pos.ptr;                 // offsets [nblocks + 1], totals [nblocks], longest list
+    GRF_CUDA_TRY(cudaMemsetAsync(blk_pos + 2 * nblocks + 1, 0, sizeof(int32_t), ctx->stream));
+    {
+        grf_launch_scope scope(ctx, 8);
+        mask_node_offsets_kernel<<<nblocks, 256, 0, ctx->stream>>>(
+            (const int32_t*)feat->plan_off.ptr, (const int32_t*)feat->plan_cnt.ptr, (const int32_t*)feat->plan_col.ptr,
+            (const int32_t*)feat->psit.rowptr.ptr, (int32_t*)K.node_off.ptr, blk_pos + nblocks + 1,
+            (const int32_t*)K.cnt.ptr, blk_pos + 2 * nblocks + 1);
+    }
+    GRF_TRY(grf_exclusive_scan(ctx, blk_pos + nblocks + 1, blk_pos, nblocks, 1));
+    GRF_CUDA_TRY(cudaMemcpyAsync(ctx->pinned + 6, blk_pos + nblocks, sizeof(int32_t), cudaMemcpyDeviceToHost, ctx->stream));
+    GRF_CUDA_TRY(cudaMemcpyAsync(ctx->pinned + 7, blk_pos + 2 * nblocks + 1, sizeof(int32_t), cudaMemcpyDeviceToHost, ctx->stream));
     GRF_CUDA_TRY(cudaStreamSynchronize(ctx->stream));          // the sizes of the key lists are known only now
     const int64_t entries = ctx->pinned[5];
     if (entries < 0) return GRF_ERR_TOO_LARGE;
+    // positions are looked up once per (block, node) when they fit 16 bits, their number fits an int32 (a negative
+    // total means it did not) and both bitmaps fit shared memory; otherwise once per (row, node)
+    const int64_t total_pos = ctx->pinned[6];
+    const size_t smem_pos = (words + ((size_t)R + 31) / 32) * 8;
+    const bool by_position = total_pos >= 0 && ctx->pinned[7] <= 65535 && smem_pos <= 96 * 1024;
     const size_t val_bytes = (size_t)entries * BQ * sizeof(__nv_bfloat16);
     if (val_bytes > ((size_t)8 << 30)) return GRF_ERR_TOO_LARGE;   // no locality: the S/z route serves this object
     if (K.key.bytes < (size_t)entries * 4) GRF_TRY(grf_buf_reserve(&K.key, ((size_t)entries + (size_t)entries / 8 + 64) * 4));
@@ -633,8 +881,28 @@ extern "C" int grf_features_materialise(grf_ctx* ctx, grf_features* feat)
         grf_launch_scope scope(ctx, 8);
         mask_order_kernel<<<grf_ceil_div(nblocks, 256), 256, 0, ctx->stream>>>(nblocks, (int32_t*)K.cnt.ptr);
     }
-    GRF_CUDA_TRY(cudaFuncSetAttribute(mask_values_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_values));
-    {
+    if (by_position) {
+        GRF_TRY(grf_buf_reserve(&K.pos16, sizeof(unsigned short) * (size_t)(total_pos + total_pos / 8 + 64)));
+        GRF_TRY(grf_buf_reserve(&K.phi_pos, sizeof(int32_t) * (size_t)(feat->phi.nnz + feat->phi.nnz / 8 + 64)));
+        GRF_CUDA_TRY(cudaFuncSetAttribute(mask_positions_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_pos));
+        {
+            grf_launch_scope scope(ctx, 8);
+            mask_positions_kernel<<<nblocks, 256, smem_pos, ctx->stream>>>(
+                N, Nk, R, (const int32_t*)feat->phi.rowptr.ptr, (const int32_t*)feat->phi.col.ptr,
+                (const int32_t*)feat->plan_off.ptr, (const int32_t*)feat->plan_cnt.ptr, (const int32_t*)feat->plan_col.ptr,
+                (const int32_t*)feat->psit.rowptr.ptr, (const int32_t*)feat->psit.col.ptr, (const uint32_t*)K.bits.ptr,
+                (const int32_t*)K.node_off.ptr, blk_pos, (unsigned short*)K.pos16.ptr, (int32_t*)K.phi_pos.ptr);
+        }
+        const size_t smem_acc = (size_t)MASK_WARPS * MASK_SEG * sizeof(float);
+        GRF_CUDA_TRY(cudaFuncSetAttribute(mask_values_pos_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_acc));
+        grf_launch_scope scope(ctx, 8);
+        mask_values_pos_kernel<<<nblocks * (BQ / MASK_ROWS), MASK_WARPS * 32, smem_acc, ctx->stream>>>(
+            N, (const int32_t*)feat->phi.rowptr.ptr, (const int32_t*)feat->phi.col.ptr, (const float*)feat->phi.val.ptr,
+            (const int32_t*)K.phi_pos.ptr, (const int32_t*)feat->psit.rowptr.ptr, (const float*)feat->psit.val.ptr,
+            (const unsigned short*)K.pos16.ptr, (const int32_t*)K.off.ptr, (const int32_t*)K.cnt.ptr,
+            (__nv_bfloat16*)K.val.ptr);
+    } else {
+        GRF_CUDA_TRY(cudaFuncSetAttribute(mask_values_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_values));
         grf_launch_scope scope(ctx, 8);
         mask_values_kernel<<<nblocks * (BQ / MASK_ROWS), MASK_WARPS * 32, smem_values, ctx->stream>>>(
             N, Nk, (const int32_t*)feat->phi.rowptr.ptr, (const int32_t*)feat->phi.col.ptr, (const float*)feat->phi.val.ptr,

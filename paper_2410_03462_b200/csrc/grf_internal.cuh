@@ -100,6 +100,9 @@ struct grf_mask_dev {
     int64_t entries = 0;            // padded key entries over all blocks
     grf_buf off, cnt, key;          // cnt holds [blocks] padded counts, then [blocks] the blocks by decreasing count
     grf_buf bits;                   // per block one bit per key: the block's key set
+    // build scratch: where each node's key positions start (within its block; the blocks' offsets), the positions,
+    // and per non-zero of Phi the start of its node's positions
+    grf_buf node_off, blk_pos, pos16, phi_pos;
     grf_buf val;
 };
 

@@ -135,3 +135,40 @@ def test_mask_is_dropped_by_resampling_and_shapes_are_checked(lib):
         api.masked_attn_mhat(ctx, feat, q.cuda(), k.cuda(), v.cuda())
     B.grf_ctx_check(ctx.handle)
     feat.free()
+
+
+def test_block_with_more_keys_than_16_bit_positions_hold(lib):
+    """One node that every key reaches (a hub column of Psi) gives the first block a key list of N > 65535 entries:
+    the build then looks positions up per row instead of keeping them in 16 bits, takes many accumulator passes for
+    that block and walks a row of Psi^T far longer than its batched fetches.  Mask rows and attention against the oracle."""
+    api, B, ctx = lib
+    N, R = 66000, 66000
+    rng = np.random.default_rng(4)
+    # Phi: the diagonal plus, for the first rows, the hub node 0;  Psi: the diagonal plus the hub for every row
+    pr, pc, pv = [0], [], []
+    for i in range(N):
+        cols = [0, i] if (0 < i < 40) else [i]
+        pc += cols; pv += list(rng.uniform(0.5, 1.0, len(cols))); pr.append(len(pc))
+    sr, sc, sv = [0], [], []
+    for j in range(N):
+        cols = [0, j] if j > 0 else [0]
+        sc += cols; sv += list(rng.uniform(0.5, 1.0, len(cols))); sr.append(len(sc))
+    Phi = oracle.CSR(np.array(pr, np.int32), np.array(pc, np.int32), np.array(pv, np.float32), None, (N, R))
+    Psi = oracle.CSR(np.array(sr, np.int32), np.array(sc, np.int32), np.array(sv, np.float32), None, (N, R))
+    feat = api.features_from_csr(ctx, N, R, (Phi.rowptr, Phi.col, Phi.val), (Psi.rowptr, Psi.col, Psi.val))
+    B.grf_features_materialise(ctx.handle, feat.handle)
+    B.grf_ctx_check(ctx.handle)
+    rows = [0, 1, 17, 39, 40, 127, 128, 4095, N - 1]
+    _check_mask(_mask_rows(B, ctx, feat, rows, N), oracle.mask_rows(Phi, Psi, rows), "hub column")
+    q, k, v = tensors.qkv(1, N, 32, 64, "bf16", 5)
+    out, den = api.masked_attn_mhat(ctx, feat, q.cuda(), k.cuda(), v.cuda(), want_den=True)
+    B.grf_ctx_check(ctx.handle)
+    Mrows = oracle.mask_rows(Phi, Psi, rows)
+
+    class _Rows:          # attn_bruteforce indexes the mask by absolute row
+        def __getitem__(self, idx):
+            return np.stack([Mrows[rows.index(int(r))] for r in np.atleast_1d(idx)])
+    ref = oracle.attn_bruteforce(tensors.widen(q), tensors.widen(k), tensors.widen(v), _Rows(), rows=rows)
+    helpers.assert_attn_close(out[:, rows].float().cpu().numpy(), ref, helpers.TOL["bf16"], den[:, rows].cpu().numpy(),
+                              "hub column", same_sign=True)
+    feat.free()
