@@ -390,14 +390,43 @@ mask_positions_kernel(int32_t N, int32_t Nk, int32_t R, const int32_t* __restric
     }
     __syncthreads();
     const int32_t base = blk_pos[blk];
-    // positions of the keys of every node of the list
-    for (int32_t u = warp; u < ucnt; u += 8) {
-        const int32_t l = __ldg(ulist + u);
-        const int32_t rb = __ldg(t_rowptr + l), re = __ldg(t_rowptr + l + 1);
-        unsigned short* dst = pos16 + (size_t)base + node_off[uoff + u];
-        for (int32_t q = rb + lane; q < re; q += 32) {
-            const int32_t j = __ldg(t_col + q);
-            dst[q - rb] = (unsigned short)(kbefore[j >> 5] + __popc(kbits[j >> 5] & ((1u << (j & 31)) - 1u)));
+    // positions of the keys of every node of the list; a warp takes 32 nodes at a time (lane x holds node x's extent
+    // in Psi^T and the start of its positions) and fetches the keys of four nodes together
+    for (int32_t u0 = warp * 32; u0 < ucnt; u0 += 8 * 32) {
+        const int32_t n = min(32, ucnt - u0);
+        const int32_t my_l = lane < n ? __ldg(ulist + u0 + lane) : 0;
+        const int32_t my_beg = lane < n ? __ldg(t_rowptr + my_l) : 0;
+        const int32_t my_end = lane < n ? __ldg(t_rowptr + my_l + 1) : 0;
+        const int32_t my_dst = lane < n ? base + node_off[uoff + u0 + lane] : 0;
+        for (int32_t e0 = 0; e0 < n; e0 += 4) {
+            int32_t jj[4][4];
+            int32_t ebeg[4], eend[4], edst[4];
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                ebeg[e] = e0 + e < n ? __shfl_sync(0xffffffffu, my_beg, (e0 + e) & 31) : 0;
+                eend[e] = e0 + e < n ? __shfl_sync(0xffffffffu, my_end, (e0 + e) & 31) : 0;
+                edst[e] = __shfl_sync(0xffffffffu, my_dst, (e0 + e) & 31);
+#pragma unroll
+                for (int sl = 0; sl < 4; ++sl) {
+                    const int32_t q = ebeg[e] + sl * 32 + lane;
+                    jj[e][sl] = q < eend[e] ? __ldg(t_col + q) : -1;
+                }
+            }
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+#pragma unroll
+                for (int sl = 0; sl < 4; ++sl) {
+                    const int32_t j = jj[e][sl];
+                    if (j >= 0)
+                        pos16[(size_t)edst[e] + sl * 32 + lane] =
+                            (unsigned short)(kbefore[j >> 5] + __popc(kbits[j >> 5] & ((1u << (j & 31)) - 1u)));
+                }
+                for (int32_t q = ebeg[e] + 128 + lane; q < eend[e]; q += 32) {        // nodes with more than 128 keys
+                    const int32_t j = __ldg(t_col + q);
+                    pos16[(size_t)edst[e] + (q - ebeg[e])] =
+                        (unsigned short)(kbefore[j >> 5] + __popc(kbits[j >> 5] & ((1u << (j & 31)) - 1u)));
+                }
+            }
         }
     }
     // where the positions of its node start, for every non-zero of the block's rows of Phi (the list holds a node
