@@ -343,6 +343,8 @@ mask_node_offsets_kernel(const int32_t* __restrict__ plan_off, const int32_t* __
     }
 }
 
+constexpr int MASK_POS_PARTS = 4;
+
 __global__ void __launch_bounds__(256)
 mask_positions_kernel(int32_t N, int32_t Nk, int32_t R, const int32_t* __restrict__ phi_rowptr,
                       const int32_t* __restrict__ phi_col, const int32_t* __restrict__ plan_off,
@@ -354,7 +356,8 @@ mask_positions_kernel(int32_t N, int32_t Nk, int32_t R, const int32_t* __restric
     extern __shared__ uint32_t smem_pos[];      // key bitmap, its prefix counts, node bitmap, its prefix counts
     __shared__ int32_t warp_sums[8];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int32_t blk = blockIdx.x;
+    // MASK_POS_PARTS CTAs share a block: each takes every MASK_POS_PARTS-th batch of nodes and slice of non-zeros
+    const int32_t blk = blockIdx.x / MASK_POS_PARTS, part = blockIdx.x % MASK_POS_PARTS;
     const int32_t wk = (Nk + 31) >> 5, wr = (R + 31) >> 5;
     uint32_t* kbits = smem_pos;
     int32_t* kbefore = reinterpret_cast<int32_t*>(smem_pos + wk);
@@ -392,7 +395,7 @@ mask_positions_kernel(int32_t N, int32_t Nk, int32_t R, const int32_t* __restric
     const int32_t base = blk_pos[blk];
     // positions of the keys of every node of the list; a warp takes 32 nodes at a time (lane x holds node x's extent
     // in Psi^T and the start of its positions) and fetches the keys of four nodes together
-    for (int32_t u0 = warp * 32; u0 < ucnt; u0 += 8 * 32) {
+    for (int32_t u0 = (part * 8 + warp) * 32; u0 < ucnt; u0 += MASK_POS_PARTS * 8 * 32) {
         const int32_t n = min(32, ucnt - u0);
         const int32_t my_l = lane < n ? __ldg(ulist + u0 + lane) : 0;
         const int32_t my_beg = lane < n ? __ldg(t_rowptr + my_l) : 0;
@@ -432,7 +435,7 @@ mask_positions_kernel(int32_t N, int32_t Nk, int32_t R, const int32_t* __restric
     // where the positions of its node start, for every non-zero of the block's rows of Phi (the list holds a node
     // once, apart from the padding at its end, which repeats the last node: the first occurrence counts)
     const int32_t r0 = blk * BQ, r1 = min(N, r0 + BQ);
-    for (int32_t p = phi_rowptr[r0] + tid; p < phi_rowptr[r1]; p += 256) {
+    for (int32_t p = phi_rowptr[r0] + part * 256 + tid; p < phi_rowptr[r1]; p += MASK_POS_PARTS * 256) {
         const int32_t l = __ldg(phi_col + p);
         const int32_t u = nbefore[l >> 5] + __popc(nbits[l >> 5] & ((1u << (l & 31)) - 1u));
         phi_pos[p] = base + node_off[uoff + u];
@@ -875,7 +878,12 @@ extern "C" int grf_features_materialise(grf_ctx* ctx, grf_features* feat)
                                  cudaMemcpyDeviceToHost, ctx->stream));
     // where every node's key positions will start (per block, then over the blocks), and the longest key list
     const int32_t R = feat->psit.rows;
-    GRF_TRY(grf_buf_reserve(&K.node_off, sizeof(int32_t) * (size_t)(feat->plan_entries > 0 ? feat->plan_entries : 1)));
+    // (buffers whose size follows the sample grow with head-room: resampling changes the sizes a little every time,
+    // and a reallocation stalls the device)
+    auto reserve_with_headroom = [](grf_buf* b, size_t bytes) {
+        return b->bytes >= bytes ? GRF_OK : grf_buf_reserve(b, bytes + bytes / 8 + 256);
+    };
+    GRF_TRY(reserve_with_headroom(&K.node_off, sizeof(int32_t) * (size_t)(feat->plan_entries > 0 ? feat->plan_entries : 1)));
     GRF_TRY(grf_buf_reserve(&K.blk_pos, sizeof(int32_t) * (2 * (size_t)nblocks + 2)));
     int32_t* blk_pos = (int32_t*)K.blk_pos.ptr;                 // offsets [nblocks + 1], totals [nblocks], longest list
     GRF_CUDA_TRY(cudaMemsetAsync(blk_pos + 2 * nblocks + 1, 0, sizeof(int32_t), ctx->stream));
@@ -911,12 +919,12 @@ extern "C" int grf_features_materialise(grf_ctx* ctx, grf_features* feat)
         mask_order_kernel<<<grf_ceil_div(nblocks, 256), 256, 0, ctx->stream>>>(nblocks, (int32_t*)K.cnt.ptr);
     }
     if (by_position) {
-        GRF_TRY(grf_buf_reserve(&K.pos16, sizeof(unsigned short) * (size_t)(total_pos + total_pos / 8 + 64)));
-        GRF_TRY(grf_buf_reserve(&K.phi_pos, sizeof(int32_t) * (size_t)(feat->phi.nnz + feat->phi.nnz / 8 + 64)));
+        GRF_TRY(reserve_with_headroom(&K.pos16, sizeof(unsigned short) * (size_t)(total_pos + 1)));
+        GRF_TRY(reserve_with_headroom(&K.phi_pos, sizeof(int32_t) * (size_t)(feat->phi.nnz + 1)));
         GRF_CUDA_TRY(cudaFuncSetAttribute(mask_positions_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_pos));
         {
             grf_launch_scope scope(ctx, 8);
-            mask_positions_kernel<<<nblocks, 256, smem_pos, ctx->stream>>>(
+            mask_positions_kernel<<<nblocks * MASK_POS_PARTS, 256, smem_pos, ctx->stream>>>(
                 N, Nk, R, (const int32_t*)feat->phi.rowptr.ptr, (const int32_t*)feat->phi.col.ptr,
                 (const int32_t*)feat->plan_off.ptr, (const int32_t*)feat->plan_cnt.ptr, (const int32_t*)feat->plan_col.ptr,
                 (const int32_t*)feat->psit.rowptr.ptr, (const int32_t*)feat->psit.col.ptr, (const uint32_t*)K.bits.ptr,
