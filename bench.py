@@ -383,7 +383,8 @@ def measure(args, workload_name, route, with_cpu_baseline, with_e2e, frozen=Fals
 
     # ---- end to end through the host-buffer entry point (pinned host memory; copies inside the timing)
     e2e = None
-    if with_e2e and route == "sz" and not frozen:
+    if with_e2e and route in ("sz", "mhat") and not frozen:
+        B.grf_ctx_prefer_mask_route(ctx.handle, mhat)
         qh, kh, vh = q.pin_memory(), k.pin_memory(), v.pin_memory()
         oh = torch.empty_like(v).pin_memory()
         rp_h = torch.from_numpy(g.rowptr).pin_memory(); c_h = torch.from_numpy(g.col).pin_memory()
@@ -479,7 +480,8 @@ def measure(args, workload_name, route, with_cpu_baseline, with_e2e, frozen=Fals
             "gpu_launches": launches,
             "e2e": None if not e2e else
                    {"value": tokens_per_step / (e2e["ms"] * 1e-3), "unit": UNIT, "h2d_bytes_per_step": e2e["h2d"],
-                    "d2h_bytes_per_step": e2e["d2h"], "ms_per_step": e2e["ms"], "entry_point": "grf_step_host"},
+                    "d2h_bytes_per_step": e2e["d2h"], "ms_per_step": e2e["ms"],
+                    "entry_point": "grf_step_host" + (" after grf_ctx_prefer_mask_route" if mhat else "")},
             "roofline": {"kernel": dom, "bound": bound, "frac_of": "hbm (the metric's roofline)", "achieved": achieved,
                          "peak": pk["hbm_gbs"], "unit": "GB/s", "frac": achieved / pk["hbm_gbs"], "peak_source": pk["source"],
                          "traffic": traffic, "algorithmic_bytes": alg.get(dom, 0),
@@ -707,7 +709,7 @@ def main():
     ap.add_argument("--route", choices=["sz", "asym", "mhat"], default="sz",
                     help="sz: Alg. 1 through per-node states (the default and the headline); mhat: Eqs. 1-2 over the "
                          "materialised mask Phi Psi^T; asym: Alg. 2 (asymmetric features, Psi = I); the last two are "
-                         "variants outside the headline metric, without an end-to-end leg")
+                         "variants outside the headline metric")
     ap.add_argument("--frozen", action="store_true", help="features sampled (and prepared) once, outside the timed steps")
     ap.add_argument("--softmax", action="store_true", help="with --route asym: A_ij = exp(q_i . k_j)")
     ap.add_argument("--heads", type=int, default=0, help="override the workload's head count (profiling of a smaller case)")

@@ -260,6 +260,12 @@ int grf_ctx_check_graphs(grf_ctx* ctx, int enable);
  * stays usable.  Asynchronous. */
 int grf_debug_wait_timeout(grf_ctx* ctx, int64_t limit_cycles);
 
+/* Route of grf_step_host: 0 (default) = through the per-node states (grf_masked_linear_attn); 1 = over the materialised
+ * mask (grf_features_materialise + grf_masked_attn_mhat) whenever the shape allows it (bf16, d = 64, m in {16, 32, 64})
+ * and the mask can be built; otherwise the call falls back to the default route.  Same outputs within the stated
+ * tolerance. */
+int grf_ctx_prefer_mask_route(grf_ctx* ctx, int enable);
+
 /* Waits for the context's stream and reports whether any kernel since the previous check gave up one of its
  * bounded waits (GRF_ERR_TIMEOUT; the affected outputs are invalid), else GRF_OK. */
 int grf_ctx_check(grf_ctx* ctx);

@@ -56,6 +56,7 @@ _SIGNATURES = {
     "grf_ctx_check": (_int, [_vp]),
     "grf_debug_wait_timeout": (_int, [_vp, _i64]),
     "grf_ctx_check_graphs": (_int, [_vp, _int]),
+    "grf_ctx_prefer_mask_route": (_int, [_vp, _int]),
     "grf_ctx_use_tensor_cores": (_int, [_vp, _int]),
     "grf_ctx_enable_timing": (_int, [_vp, _int]),
     "grf_ctx_kernel_times": (_int, [_vp, _vp, _vp]),
@@ -134,6 +135,10 @@ def grf_ctx_check(ctx: int):
 
 def grf_debug_wait_timeout(ctx: int, limit_cycles: int):
     _check(lib.grf_debug_wait_timeout(ctx, limit_cycles), "grf_debug_wait_timeout")
+
+
+def grf_ctx_prefer_mask_route(ctx: int, enable: bool):
+    _check(lib.grf_ctx_prefer_mask_route(ctx, int(enable)), "grf_ctx_prefer_mask_route")
 
 
 def grf_ctx_check_graphs(ctx: int, enable: bool):

@@ -118,6 +118,13 @@ extern "C" int grf_ctx_use_tensor_cores(grf_ctx* ctx, int enable)
     return GRF_OK;
 }
 
+extern "C" int grf_ctx_prefer_mask_route(grf_ctx* ctx, int enable)
+{
+    if (!ctx) return GRF_ERR_INVALID;
+    ctx->prefer_mask_route = enable != 0;
+    return GRF_OK;
+}
+
 extern "C" int grf_ctx_check_graphs(grf_ctx* ctx, int enable)
 {
     if (!ctx) return GRF_ERR_INVALID;
@@ -401,8 +408,15 @@ extern "C" int grf_step_host(grf_ctx* ctx, int32_t N, const int32_t* rowptr, con
     }
     GRF_TRY(grf_sample(ctx, N, (const int32_t*)ctx->h_rowptr.ptr, (const int32_t*)ctx->h_col.ptr,
                        (const float*)ctx->h_w.ptr, seed, n_walks, p_halt, max_len, f_phi, f_psi, &ctx->h_feat));
+    // route: over the materialised mask when the caller prefers it and the shape and the graph allow it
+    bool by_mask = false;
+    if (ctx->prefer_mask_route && dtype == GRF_DTYPE_BF16 && d == 64 && (m == 16 || m == 32 || m == 64)) {
+        const int rc = grf_features_materialise(ctx, ctx->h_feat);
+        if (rc == GRF_OK) by_mask = true;
+        else if (rc != GRF_ERR_TOO_LARGE) return rc;          // too large = no locality: the S/z route serves it
+    }
     // workspace: one part's records if that is modest, else chunks of about 1 GiB
-    const size_t per = ws_per_problem(N, m, d, dtype);
+    const size_t per = by_mask ? 256 : ws_per_problem(N, m, d, dtype);
     size_t want = per * (size_t)gp;
     const size_t cap = (size_t)1 << 31;
     if (want > cap) want = per * (cap / per > 0 ? cap / per : 1);
@@ -412,9 +426,14 @@ extern "C" int grf_step_host(grf_ctx* ctx, int32_t N, const int32_t* rowptr, con
         if (gc <= 0) break;
         const size_t qo = (size_t)g0 * N * m * es, vo = (size_t)g0 * N * d * es;
         GRF_CUDA_TRY(cudaStreamWaitEvent(s, ctx->up_done[p], 0));
-        GRF_TRY(grf_masked_linear_attn(ctx, ctx->h_feat, gc, N, m, d, dtype, (const char*)ctx->h_q.ptr + qo,
-                                       (const char*)ctx->h_k.ptr + qo, (const char*)ctx->h_v.ptr + vo,
-                                       (char*)ctx->h_out.ptr + vo, nullptr, ctx->h_ws.ptr, ctx->h_ws.bytes));
+        if (by_mask)
+            GRF_TRY(grf_masked_attn_mhat(ctx, ctx->h_feat, gc, N, m, d, dtype, (const char*)ctx->h_q.ptr + qo,
+                                         (const char*)ctx->h_k.ptr + qo, (const char*)ctx->h_v.ptr + vo,
+                                         (char*)ctx->h_out.ptr + vo, nullptr));
+        else
+            GRF_TRY(grf_masked_linear_attn(ctx, ctx->h_feat, gc, N, m, d, dtype, (const char*)ctx->h_q.ptr + qo,
+                                           (const char*)ctx->h_k.ptr + qo, (const char*)ctx->h_v.ptr + vo,
+                                           (char*)ctx->h_out.ptr + vo, nullptr, ctx->h_ws.ptr, ctx->h_ws.bytes));
         GRF_CUDA_TRY(cudaEventRecord(ctx->part_done[p], s));
         GRF_CUDA_TRY(cudaStreamWaitEvent(ctx->down_stream, ctx->part_done[p], 0));
         GRF_CUDA_TRY(cudaMemcpyAsync((char*)out + vo, (const char*)ctx->h_out.ptr + vo, (size_t)gc * N * d * es,

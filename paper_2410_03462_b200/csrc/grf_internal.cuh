@@ -54,6 +54,7 @@ struct grf_ctx {
     int32_t* pinned = nullptr;      // small pinned host block for read-backs
     int* error_word = nullptr;      // device word set by a kernel that gave up a bounded wait
     bool use_tensor_cores = true;
+    bool prefer_mask_route = false; // grf_step_host evaluates the attention over the materialised mask where it can
     bool check_graphs = false;      // grf_sample validates the device-resident CSR first (debugging aid)
     // optional per-launch timing
     bool timing = false;

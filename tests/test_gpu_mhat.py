@@ -172,3 +172,32 @@ def test_block_with_more_keys_than_16_bit_positions_hold(lib):
     helpers.assert_attn_close(out[:, rows].float().cpu().numpy(), ref, helpers.TOL["bf16"], den[:, rows].cpu().numpy(),
                               "hub column", same_sign=True)
     feat.free()
+
+
+def test_host_buffer_path_over_the_mask_equals_device_calls(lib):
+    """grf_step_host after grf_ctx_prefer_mask_route: same bits as sampling, materialising and calling the attention
+    on device buffers; a shape the route does not cover falls back to the route through the per-node states."""
+    api, B, ctx = lib
+    w = configs.point_cloud_4096(1024)
+    g = w.graph()
+    f = B.grf_deconvolve(w.alpha).astype(np.float32)
+    q, k, v = tensors.qkv(4, g.N, w.m, w.d, w.dtype, 3)
+    out_h = torch.empty_like(v)
+    B.grf_ctx_prefer_mask_route(ctx.handle, True)
+    try:
+        B.grf_step_host(ctx.handle, g.N, g.rowptr, g.col, g.w, 9, w.n_walks, w.p_halt, w.max_len, f, None,
+                        4, w.m, w.d, B.GRF_DTYPE_BF16, q, k, v, out_h)
+        feat = api.sample(ctx, api.DeviceGraph(g), 9, w.n_walks, w.p_halt, w.max_len, f)
+        B.grf_features_materialise(ctx.handle, feat.handle)
+        out_d = api.masked_attn_mhat(ctx, feat, q.cuda(), k.cuda(), v.cuda())
+        assert torch.equal(out_h, out_d.cpu())
+        # m = 8 is not covered by the mask route: the call must still work (per-node states)
+        q8, k8, _ = tensors.qkv(4, g.N, 8, w.d, w.dtype, 3)
+        out8 = torch.empty_like(v)
+        B.grf_step_host(ctx.handle, g.N, g.rowptr, g.col, g.w, 9, w.n_walks, w.p_halt, w.max_len, f, None,
+                        4, 8, w.d, B.GRF_DTYPE_BF16, q8, k8, v, out8)
+        out8_d = api.masked_linear_attn(ctx, feat, q8.cuda(), k8.cuda(), v.cuda())
+        assert torch.equal(out8, out8_d.cpu())
+        feat.free()
+    finally:
+        B.grf_ctx_prefer_mask_route(ctx.handle, False)
