@@ -713,6 +713,7 @@ def main():
     ap.add_argument("--frozen", action="store_true", help="features sampled (and prepared) once, outside the timed steps")
     ap.add_argument("--softmax", action="store_true", help="with --route asym: A_ij = exp(q_i . k_j)")
     ap.add_argument("--heads", type=int, default=0, help="override the workload's head count (profiling of a smaller case)")
+    ap.add_argument("--no-other-routes", action="store_true", help="skip the short runs of the other routes beside the headline")
     ap.add_argument("--suite", action="store_true")
     ap.add_argument("--suite-dir", default=os.path.join(ROOT, "gpurun_out"))
     args = ap.parse_args()
@@ -734,6 +735,24 @@ def main():
             res = run_suite(args)
         else:
             res = measure(args, args.workload, args.route, not args.no_cpu_baseline, True, frozen=args.frozen)
+            # beside the headline (the route through the per-node states, features resampled every step): the same
+            # workload on the route over the materialised mask, and both routes with frozen features, in short runs
+            if res is not None and world == 1 and args.route == "sz" and not args.frozen and not args.no_other_routes:
+                w = make_workload(args.workload)
+                if w.dtype == "bf16" and w.d == 64 and w.m in (16, 32, 64):
+                    from paper_2410_03462_b200 import binding as B
+                    others = {}
+                    for name, route, frozen in (("mhat_resampled", "mhat", False), ("mhat_frozen", "mhat", True),
+                                                ("sz_frozen", "sz", True)):
+                        try:
+                            r = measure(args, args.workload, route, False, False, frozen=frozen, steps=min(args.steps, 10), warmup=3)
+                        except B.GrfError as e:
+                            others[name] = {"error": str(e)}
+                            continue
+                        others[name] = {"value": r["value"], "unit": UNIT, "ms_per_step": r["ms_per_step"],
+                                        "attn_ms": r["phases"]["attn_ms"], "step": r["config"]["step"],
+                                        "kernels_ms": {k: v["ms_per_step"] for k, v in r["kernels"].items()}}
+                    res["other_routes"] = others
         if world > 1:
             dist.destroy_process_group()
     if res is not None:
