@@ -97,7 +97,7 @@ def load_counters():
 
 
 class ClockSampler:
-    """nvidia-smi clock/throttle samples every 100 ms while the timed region runs (read-only queries)."""
+    """nvidia-smi clock/throttle samples every 10 ms while the timed region runs (read-only queries)."""
     FIELDS = ("timestamp,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
               "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
               "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
@@ -108,7 +108,7 @@ class ClockSampler:
         try:
             self.proc = subprocess.Popen(
                 ["nvidia-smi", f"--id={device_index}", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
-                 "-lms", "50"], stdout=self.tmp, stderr=subprocess.DEVNULL)
+                 "-lms", "10"], stdout=self.tmp, stderr=subprocess.DEVNULL)
         except OSError:
             self.proc = None
 

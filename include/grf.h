@@ -159,7 +159,9 @@ int grf_csr_transpose(grf_ctx* ctx, int32_t rows, int32_t cols, int64_t nnz,
  * Limits: cols <= GRF_NOALLOC_MAX_COLS and nnz <= GRF_NOALLOC_MAX_NNZ, otherwise GRF_ERR_TOO_LARGE and
  * nothing is launched.  The function calls no cudaMalloc/cudaFree and no allocating library routine.
  * The first call on a device looks up the array's device address (once per device); make that first
- * call before any stream capture begins.  All calls on one GPU share the array and it keeps the previous
+ * call before any stream capture begins, and, in a process that hands the whole device memory to its own pool,
+ * before the pool takes it: where the CUDA module is loaded lazily, the array is reserved only at that first call,
+ * which then fails with GRF_ERR_CUDA if no memory is left.  All calls on one GPU share the array and it keeps the previous
  * call's contents (the function clears what has to start at zero): two calls whose device work overlaps in
  * time, on different streams or from different threads, race on it and give wrong results — order them.
  */

@@ -57,6 +57,11 @@ def test_point_cloud_4096_all_heads_against_full_bruteforce(lib):
                                   f"{w.name} {what}", same_sign=True)
 
     _both_gather_kernels(lib, feat, q, k, v, check)
+    # the same workload over the materialised mask (Eqs. 1-2 evaluated directly)
+    B.grf_features_materialise(ctx.handle, feat.handle)
+    out, den = api.masked_attn_mhat(ctx, feat, q.cuda(), k.cuda(), v.cuda(), want_den=True)
+    B.grf_ctx_check(ctx.handle)
+    check(out, den, "materialised mask")
     feat.free()
 
 
@@ -86,6 +91,11 @@ def test_vit_grid_full_batch_of_768_problems(lib):
         assert torch.isfinite(out.float()).all()
 
     _both_gather_kernels(lib, feat, q, k, v, check)
+    # the full batch over the materialised mask as well (grid of 2 blocks x 768 problems)
+    B.grf_features_materialise(ctx.handle, feat.handle)
+    out_m, den_m = api.masked_attn_mhat(ctx, feat, q.cuda(), k.cuda(), v.cuda(), want_den=True)
+    B.grf_ctx_check(ctx.handle)
+    check(out_m, den_m, "materialised mask")
     # all problems see the same features: two problems given identical inputs must give identical outputs
     q2, k2, v2 = q.clone(), k.clone(), v.clone()
     q2[500], k2[500], v2[500] = q[3], k[3], v[3]
