@@ -570,8 +570,9 @@ mask_rows_kernel(int32_t Nk, const int32_t* __restrict__ rows, const int32_t* __
 }
 
 // ---------------------------------------------------------------------------------------------------
-// The attention kernel.  warps 0-3: row threads (one query = one tensor-memory lane each); warp 4: MMA issuer;
-// warps 5-8: producers (gathers of key-feature and value rows, a quarter of every tile each: a thread's
+// The attention kernel.  warps 0-3 and 4-7: two groups of row threads (one query = one tensor-memory lane each; the
+// first group takes the even key tiles and score buffer 0, the second the odd tiles and buffer 1, so that the
+// masking of one tile runs beside that of the next); warp 8: MMA issuer; warps 9-12: producers (gathers of key-feature and value rows, a quarter of every tile each: a thread's
 // tensor-map gathers are issued one after the other, so they are spread over sixteen threads of four warps).
 
 template <int M> struct MhShape {
@@ -588,7 +589,7 @@ template <int M> struct MhShape {
     static_assert(STAGE % 1024 == 0, "stages must keep the swizzle phase");
 };
 
-constexpr int MH_THREADS = 288;          // warps 0-3: row threads; warp 4: MMA issuer; warps 5-8: producers
+constexpr int MH_THREADS = 416;          // warps 0-3, 4-7: two groups of row threads; warp 8: MMA issuer; warps 9-12: producers
 
 template <int M>
 __global__ void __launch_bounds__(MH_THREADS)
@@ -602,9 +603,10 @@ mhat_attention_kernel(int32_t G, int32_t nblocks, int32_t N, const int32_t* __re
     constexpr int NS = Sh::NS, D = Sh::D;
     extern __shared__ unsigned char smem_dyn[];
     // kv_full, kv_empty per stage; s_full, p_full, s_free per score buffer; acc_done; drain
-    __shared__ __align__(8) unsigned long long bars[2 * NS + 6 + 2];
+    __shared__ __align__(8) unsigned long long bars[2 * NS + 6 + 3];
     __shared__ uint32_t tmem_slot;
     __shared__ int abort_flag;
+    __shared__ float den_odd[BQ];                  // row sums of the odd tiles, handed to the first group
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int32_t g = (int32_t)(blockIdx.x % (uint32_t)G);
@@ -620,16 +622,18 @@ mhat_attention_kernel(int32_t G, int32_t nblocks, int32_t N, const int32_t* __re
     auto s_free = [&](int b) { return bar_base + 8u * (uint32_t)(2 * NS + 4 + b); };
     const uint32_t acc_done = bar_base + 8u * (uint32_t)(2 * NS + 6);
     const uint32_t drain_bar = bar_base + 8u * (uint32_t)(2 * NS + 7);
+    const uint32_t den_ready = bar_base + 8u * (uint32_t)(2 * NS + 8);
 
     if (tid == 0) {
         for (int s = 0; s < NS; ++s) { mbar_init(kv_full(s), 8); mbar_init(kv_empty(s), 1); }
         for (int b = 0; b < 2; ++b) { mbar_init(s_full(b), 1); mbar_init(p_full(b), 4); mbar_init(s_free(b), 1); }
         mbar_init(acc_done, 1);
         mbar_init(drain_bar, 1);
+        mbar_init(den_ready, 4);
         abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    if (warp == 4) tmem_alloc(&tmem_slot, (uint32_t)Sh::TMEM_COLS);
+    if (warp == 8) tmem_alloc(&tmem_slot, (uint32_t)Sh::TMEM_COLS);
     // the block's queries in the K-major operand layout: 16-byte chunk c of row r at (c * 128 + r) * 16
     if (tid < BQ) {
         const int32_t row = blk * BQ + tid;
@@ -649,25 +653,27 @@ mhat_attention_kernel(int32_t G, int32_t nblocks, int32_t N, const int32_t* __re
     const int32_t off = mk_off[blk];
     const int32_t T = mk_cnt[blk] / KT;                   // key tiles of this block
 
-    if (warp < 4) {
+    if (warp < 8) {
         // ------------------------------------------------------------ row threads: P = S * Mhat, row sums, epilogue
-        const int32_t row = blk * BQ + tid;
-        const uint32_t lane_field = (uint32_t)(warp * 32) << 16;
-        const uint4* mrow = mk_val + (size_t)(off / 8) * BQ + tid;      // chunk x of this row: mrow[x * BQ]
+        const int grp = warp >> 2;                               // 0: even tiles, 1: odd tiles
+        const int rr = (warp & 3) * 32 + lane;                   // row of the block = tensor-memory lane
+        const int32_t row = blk * BQ + rr;
+        const uint32_t lane_field = (uint32_t)((warp & 3) * 32) << 16;
+        const uint4* mrow = mk_val + (size_t)(off / 8) * BQ + rr;       // chunk x of this row: mrow[x * BQ]
         float den = 0.0f;
         uint4 mk[KT / 8];
-        if (T > 0) {
+        if (grp < T) {
 #pragma unroll
-            for (int c = 0; c < KT / 8; ++c) mk[c] = __ldg(mrow + (size_t)c * BQ);
+            for (int c = 0; c < KT / 8; ++c) mk[c] = __ldg(mrow + (size_t)(grp * (KT / 8) + c) * BQ);
         }
         bool ok = true;
-        for (int32_t t = 0; t < T; ++t) {
-            const int buf = t & 1;
+        const int buf = grp;
+        const uint32_t s_addr = tmem_base + lane_field + (uint32_t)(buf * Sh::S_COLS);
+        for (int32_t t = grp; t < T; t += 2) {
             if (!mbar_wait(s_full(buf), (uint32_t)(t >> 1) & 1u, &abort_flag)) ok = false;
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
             fence_after_sync();
-            const uint32_t s_addr = tmem_base + lane_field + (uint32_t)(buf * Sh::S_COLS);
 #pragma unroll
             for (int c16 = 0; c16 < KT / 16; ++c16) {
                 uint32_t sv[16];
@@ -689,42 +695,51 @@ mhat_attention_kernel(int32_t G, int32_t nblocks, int32_t N, const int32_t* __re
                 }
                 tmem_st8(s_addr + (uint32_t)(c16 * 8), pw);
             }
-            // next tile's mask values travel while the products run
-            if (t + 1 < T) {
+            // this group's next tile: its mask values travel while the products run
+            if (t + 2 < T) {
 #pragma unroll
-                for (int c = 0; c < KT / 8; ++c) mk[c] = __ldg(mrow + (size_t)((t + 1) * (KT / 8) + c) * BQ);
+                for (int c = 0; c < KT / 8; ++c) mk[c] = __ldg(mrow + (size_t)((t + 2) * (KT / 8) + c) * BQ);
             }
             tmem_st_wait();
             fence_before_sync();
             __syncwarp();
             if (lane == 0) mbar_arrive(p_full(buf));
         }
-        if (ok && T > 0) ok = mbar_wait(acc_done, 0u, &abort_flag);
-        ok = __all_sync(0xffffffffu, ok);
-        fence_after_sync();
-        const bool live = row < N;
-        const float inv = (den != 0.0f) ? 1.0f / den : 0.0f;
-        if (live && ok && den_out) den_out[(size_t)g * N + row] = den;
-        __nv_bfloat16* orow = out + ((size_t)g * N + row) * D;
-#pragma unroll
-        for (int c0 = 0; c0 < D; c0 += 16) {
-            uint32_t r[16];
-#pragma unroll
-            for (int e = 0; e < 16; ++e) r[e] = 0u;
-            if (ok && T > 0) tmem_ld16(tmem_base + lane_field + (uint32_t)(Sh::O_COL + c0), r);
-            if (live && ok) {
-                uint32_t w[8];
-#pragma unroll
-                for (int e = 0; e < 8; ++e) {
-                    __nv_bfloat162 h = __floats2bfloat162_rn(__uint_as_float(r[2 * e]) * inv, __uint_as_float(r[2 * e + 1]) * inv);
-                    w[e] = *reinterpret_cast<uint32_t*>(&h);
+        if (grp == 1) {
+            // hand the odd tiles' row sums to the first group, which writes the block's outputs
+            den_odd[rr] = den;
+            __syncwarp();
+            if (lane == 0) mbar_arrive(den_ready);
+        } else {
+            if (ok && !mbar_wait(den_ready, 0u, &abort_flag)) ok = false;
+            den += den_odd[rr];
+            if (ok && T > 0) ok = mbar_wait(acc_done, 0u, &abort_flag);
+            ok = __all_sync(0xffffffffu, ok);
+            fence_after_sync();
+            const bool live = row < N;
+            const float inv = (den != 0.0f) ? 1.0f / den : 0.0f;
+            if (live && ok && den_out) den_out[(size_t)g * N + row] = den;
+            __nv_bfloat16* orow = out + ((size_t)g * N + row) * D;
+    #pragma unroll
+            for (int c0 = 0; c0 < D; c0 += 16) {
+                uint32_t r[16];
+    #pragma unroll
+                for (int e = 0; e < 16; ++e) r[e] = 0u;
+                if (ok && T > 0) tmem_ld16(tmem_base + lane_field + (uint32_t)(Sh::O_COL + c0), r);
+                if (live && ok) {
+                    uint32_t w[8];
+    #pragma unroll
+                    for (int e = 0; e < 8; ++e) {
+                        __nv_bfloat162 h = __floats2bfloat162_rn(__uint_as_float(r[2 * e]) * inv, __uint_as_float(r[2 * e + 1]) * inv);
+                        w[e] = *reinterpret_cast<uint32_t*>(&h);
+                    }
+                    uint4* dst = reinterpret_cast<uint4*>(orow + c0);
+                    dst[0] = make_uint4(w[0], w[1], w[2], w[3]);
+                    dst[1] = make_uint4(w[4], w[5], w[6], w[7]);
                 }
-                uint4* dst = reinterpret_cast<uint4*>(orow + c0);
-                dst[0] = make_uint4(w[0], w[1], w[2], w[3]);
-                dst[1] = make_uint4(w[4], w[5], w[6], w[7]);
             }
         }
-    } else if (warp >= 5) {
+    } else if (warp >= 9) {
         // ------------------------------------------------------------ producers: warp w takes keys 16w .. 16w+15 of every tile
         // Lanes x and x + 16 hold key x of the warp's sixteen.  Value rows: lanes 0-3 each gather four rows through
         // the tensor map (they land in the swizzled layout and complete on the stage's barrier by byte count).
@@ -732,7 +747,7 @@ mhat_attention_kernel(int32_t G, int32_t nblocks, int32_t N, const int32_t* __re
         // pieces, lanes 16-31 the odd ones.  A warp's copies of one tile form one group; it hands its part of a
         // stage over two tiles late, after that group has completed and a proxy fence.  Key indices are read one
         // tile ahead.
-        const int pw = warp - 5;
+        const int pw = warp - 9;
         const __nv_bfloat16* Kg = phiK + (size_t)g * N * M;
         const int32_t row0 = g * N;
         const int ky = pw * 16 + (lane & 15);                   // this lane's key within the tile
@@ -831,7 +846,7 @@ mhat_attention_kernel(int32_t G, int32_t nblocks, int32_t N, const int32_t* __re
 
     fence_before_sync();
     __syncthreads();
-    if (warp == 4) tmem_dealloc(tmem_base, (uint32_t)Sh::TMEM_COLS);
+    if (warp == 8) tmem_dealloc(tmem_base, (uint32_t)Sh::TMEM_COLS);
     if (tid == 0 && abort_flag) atomicExch(error_word, 1);
 }
 
