@@ -570,40 +570,47 @@ mask_rows_kernel(int32_t Nk, const int32_t* __restrict__ rows, const int32_t* __
 }
 
 // ---------------------------------------------------------------------------------------------------
-// The attention kernel.  warps 0-3 and 4-7: two groups of row threads (one query = one tensor-memory lane each; the
-// first group takes the even key tiles and score buffer 0, the second the odd tiles and buffer 1, so that the
-// masking of one tile runs beside that of the next); warp 8: MMA issuer; warps 9-12: producers (gathers of key-feature and value rows, a quarter of every tile each: a thread's
-// tensor-map gathers are issued one after the other, so they are spread over sixteen threads of four warps).
+// The attention kernel.  One CTA = 128 queries of one head; the block's keys come in tiles of 64.
+//   warps 0-3, 4-7  two groups of row threads (one query = one tensor-memory lane each): a group multiplies the
+//                   scores of every other tile by the mask, in place (fp32 scores -> bf16 pairs), and sums its rows
+//   warp 8          issues S_t = Q K_t^T into one of three score buffers
+//   warp 9          issues O += P_t V_t once the rows of tile t are masked, and frees the tile's stage and buffer
+//   warps 10-13     producers: a quarter of every tile's key-feature and value rows each, by 16-byte async copies
+// An instruction of the tensor pipe costs its issuing thread about fifty cycles, whatever its size, so the two
+// products have a thread each; three score buffers let the first product run two tiles ahead of the masking.
 
 template <int M> struct MhShape {
     static constexpr int D = 64;
     static constexpr int NS = M <= 32 ? 8 : 6;            // key/value stages in flight
-    static constexpr int V_BYTES = KT * 128;              // 64 gathered value rows, 128-byte swizzle
+    static constexpr int NB = 3;                          // score buffers
+    static constexpr int V_BYTES = KT * 128;              // 64 value rows of 128 bytes, 128-byte swizzle
     static constexpr int K_BYTES = KT * M * 2;            // [M/8][KT keys][8] bf16: K-major, unswizzled
     static constexpr int STAGE = V_BYTES + K_BYTES;
     static constexpr int Q_BYTES = BQ * M * 2;            // [M/8][128 rows][8] bf16
     static constexpr int S_COLS = KT;                     // one score buffer; P (bf16 pairs) reuses its first half
-    static constexpr int O_COL = 2 * S_COLS;
-    static constexpr int TMEM_COLS = 256;                 // 2 score buffers + the output accumulator, rounded up
+    static constexpr int O_COL = NB * S_COLS;
+    static constexpr int TMEM_COLS = 256;                 // 3 score buffers + the output accumulator
     static constexpr size_t SMEM = (size_t)NS * STAGE + Q_BYTES + 1024;
     static_assert(STAGE % 1024 == 0, "stages must keep the swizzle phase");
+    static_assert(O_COL + D <= TMEM_COLS, "tensor memory");
 };
 
-constexpr int MH_THREADS = 416;          // warps 0-3, 4-7: two groups of row threads; warp 8: MMA issuer; warps 9-12: producers
+constexpr int MH_THREADS = 448;
+constexpr int MH_ISSUER_S = 8, MH_ISSUER_O = 9, MH_PRODUCER0 = 10;
 
 template <int M>
 __global__ void __launch_bounds__(MH_THREADS)
 mhat_attention_kernel(int32_t G, int32_t nblocks, int32_t N, const int32_t* __restrict__ mk_off,
                       const int32_t* __restrict__ mk_cnt, const int32_t* __restrict__ mk_key,
                       const uint4* __restrict__ mk_val, const __nv_bfloat16* __restrict__ phiQ,
-                      const __nv_bfloat16* __restrict__ phiK, const __grid_constant__ CUtensorMap map_v,
+                      const __nv_bfloat16* __restrict__ phiK, const __nv_bfloat16* __restrict__ Vg,
                       __nv_bfloat16* __restrict__ out, float* __restrict__ den_out, int* __restrict__ error_word)
 {
     using Sh = MhShape<M>;
-    constexpr int NS = Sh::NS, D = Sh::D;
+    constexpr int NS = Sh::NS, NB = Sh::NB, D = Sh::D;
     extern __shared__ unsigned char smem_dyn[];
-    // kv_full, kv_empty per stage; s_full, p_full, s_free per score buffer; acc_done; drain
-    __shared__ __align__(8) unsigned long long bars[2 * NS + 6 + 3];
+    // kv_full, kv_empty per stage; s_full, p_full per score buffer; acc_done; den_ready; one drain barrier per issuer
+    __shared__ __align__(8) unsigned long long bars[2 * NS + 2 * NB + 4];
     __shared__ uint32_t tmem_slot;
     __shared__ int abort_flag;
     __shared__ float den_odd[BQ];                  // row sums of the odd tiles, handed to the first group
@@ -618,22 +625,22 @@ mhat_attention_kernel(int32_t G, int32_t nblocks, int32_t N, const int32_t* __re
     auto kv_full = [&](int s) { return bar_base + 8u * (uint32_t)s; };
     auto kv_empty = [&](int s) { return bar_base + 8u * (uint32_t)(NS + s); };
     auto s_full = [&](int b) { return bar_base + 8u * (uint32_t)(2 * NS + b); };
-    auto p_full = [&](int b) { return bar_base + 8u * (uint32_t)(2 * NS + 2 + b); };
-    auto s_free = [&](int b) { return bar_base + 8u * (uint32_t)(2 * NS + 4 + b); };
-    const uint32_t acc_done = bar_base + 8u * (uint32_t)(2 * NS + 6);
-    const uint32_t drain_bar = bar_base + 8u * (uint32_t)(2 * NS + 7);
-    const uint32_t den_ready = bar_base + 8u * (uint32_t)(2 * NS + 8);
+    auto p_full = [&](int b) { return bar_base + 8u * (uint32_t)(2 * NS + NB + b); };
+    const uint32_t acc_done = bar_base + 8u * (uint32_t)(2 * NS + 2 * NB);
+    const uint32_t den_ready = acc_done + 8u;
+    const uint32_t drain_s = acc_done + 16u, drain_o = acc_done + 24u;
 
     if (tid == 0) {
-        for (int s = 0; s < NS; ++s) { mbar_init(kv_full(s), 8); mbar_init(kv_empty(s), 1); }
-        for (int b = 0; b < 2; ++b) { mbar_init(s_full(b), 1); mbar_init(p_full(b), 4); mbar_init(s_free(b), 1); }
+        for (int s = 0; s < NS; ++s) { mbar_init(kv_full(s), 4); mbar_init(kv_empty(s), 1); }
+        for (int b = 0; b < NB; ++b) { mbar_init(s_full(b), 1); mbar_init(p_full(b), 4); }
         mbar_init(acc_done, 1);
-        mbar_init(drain_bar, 1);
         mbar_init(den_ready, 4);
+        mbar_init(drain_s, 1);
+        mbar_init(drain_o, 1);
         abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    if (warp == 8) tmem_alloc(&tmem_slot, (uint32_t)Sh::TMEM_COLS);
+    if (warp == MH_ISSUER_S) tmem_alloc(&tmem_slot, (uint32_t)Sh::TMEM_COLS);
     // the block's queries in the K-major operand layout: 16-byte chunk c of row r at (c * 128 + r) * 16
     if (tid < BQ) {
         const int32_t row = blk * BQ + tid;
@@ -667,13 +674,14 @@ mhat_attention_kernel(int32_t G, int32_t nblocks, int32_t N, const int32_t* __re
             for (int c = 0; c < KT / 8; ++c) mk[c] = __ldg(mrow + (size_t)(grp * (KT / 8) + c) * BQ);
         }
         bool ok = true;
-        const int buf = grp;
-        const uint32_t s_addr = tmem_base + lane_field + (uint32_t)(buf * Sh::S_COLS);
+        int buf = grp;                                           // t % NB and the parity of t / NB, kept in step
+        uint32_t par = 0u;
         for (int32_t t = grp; t < T; t += 2) {
-            if (!mbar_wait(s_full(buf), (uint32_t)(t >> 1) & 1u, &abort_flag)) ok = false;
+            if (!mbar_wait(s_full(buf), par, &abort_flag)) ok = false;
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
             fence_after_sync();
+            const uint32_t s_addr = tmem_base + lane_field + (uint32_t)(buf * Sh::S_COLS);
 #pragma unroll
             for (int c16 = 0; c16 < KT / 16; ++c16) {
                 uint32_t sv[16];
@@ -704,6 +712,8 @@ mhat_attention_kernel(int32_t G, int32_t nblocks, int32_t N, const int32_t* __re
             fence_before_sync();
             __syncwarp();
             if (lane == 0) mbar_arrive(p_full(buf));
+            buf += 2;
+            if (buf >= NB) { buf -= NB; par ^= 1u; }
         }
         if (grp == 1) {
             // hand the odd tiles' row sums to the first group, which writes the block's outputs
@@ -720,15 +730,15 @@ mhat_attention_kernel(int32_t G, int32_t nblocks, int32_t N, const int32_t* __re
             const float inv = (den != 0.0f) ? 1.0f / den : 0.0f;
             if (live && ok && den_out) den_out[(size_t)g * N + row] = den;
             __nv_bfloat16* orow = out + ((size_t)g * N + row) * D;
-    #pragma unroll
+#pragma unroll
             for (int c0 = 0; c0 < D; c0 += 16) {
                 uint32_t r[16];
-    #pragma unroll
+#pragma unroll
                 for (int e = 0; e < 16; ++e) r[e] = 0u;
                 if (ok && T > 0) tmem_ld16(tmem_base + lane_field + (uint32_t)(Sh::O_COL + c0), r);
                 if (live && ok) {
                     uint32_t w[8];
-    #pragma unroll
+#pragma unroll
                     for (int e = 0; e < 8; ++e) {
                         __nv_bfloat162 h = __floats2bfloat162_rn(__uint_as_float(r[2 * e]) * inv, __uint_as_float(r[2 * e + 1]) * inv);
                         w[e] = *reinterpret_cast<uint32_t*>(&h);
@@ -739,47 +749,51 @@ mhat_attention_kernel(int32_t G, int32_t nblocks, int32_t N, const int32_t* __re
                 }
             }
         }
-    } else if (warp >= 9) {
+    } else if (warp >= MH_PRODUCER0) {
         // ------------------------------------------------------------ producers: warp w takes keys 16w .. 16w+15 of every tile
-        // Lanes x and x + 16 hold key x of the warp's sixteen.  Value rows: lanes 0-3 each gather four rows through
-        // the tensor map (they land in the swizzled layout and complete on the stage's barrier by byte count).
-        // Key-feature rows: 16-byte pieces, piece c of key y going to (c * 64 + y) * 16; lanes 0-15 copy the even
-        // pieces, lanes 16-31 the odd ones.  A warp's copies of one tile form one group; it hands its part of a
-        // stage over two tiles late, after that group has completed and a proxy fence.  Key indices are read one
-        // tile ahead.
-        const int pw = warp - 9;
+        // Lanes x and x + 16 hold key x of the warp's sixteen.  Rows travel as 16-byte pieces.  Value rows (128
+        // bytes): eight consecutive lanes copy one row, piece c of tile row r going to r * 128 + ((c ^ (r & 7)) * 16),
+        // the 128-byte swizzle the second product's operand descriptor names.  Key-feature rows: piece c of key y
+        // goes to (c * 64 + y) * 16; lanes 0-15 copy the even pieces, lanes 16-31 the odd ones.  A warp's copies of
+        // one tile form one group; it hands its part of a stage over two tiles late, after that group has completed
+        // and a proxy fence.  Key indices are read three tiles ahead.
+        const int pw = warp - MH_PRODUCER0;
         const __nv_bfloat16* Kg = phiK + (size_t)g * N * M;
-        const int32_t row0 = g * N;
+        const __nv_bfloat16* Vh = Vg + (size_t)g * N * D;
         const int ky = pw * 16 + (lane & 15);                   // this lane's key within the tile
+        const int vc = lane & 7;                                // its piece of a value row
         bool ok = true;
-        int32_t issued = 0;
         auto hand_over = [&](int32_t t) {
             fence_async_smem();
             __syncwarp();
             if (lane == 0) mbar_arrive(kv_full(t % NS));
         };
-        int32_t kn = T > 0 ? __ldg(mk_key + off + ky) : 0;
+        const int32_t* kp = mk_key + off + ky;
+        int32_t k1 = T > 0 ? __ldg(kp) : 0, k2 = T > 1 ? __ldg(kp + KT) : 0, k3 = T > 2 ? __ldg(kp + 2 * KT) : 0;
         for (int32_t t = 0; t < T; ++t) {
             const int s = t % NS;
-            const int32_t k = kn;
-            if (t + 1 < T) kn = __ldg(mk_key + off + (t + 1) * KT + ky);
+            const int32_t k = k1;
+            k1 = k2; k2 = k3;
+            if (t + 3 < T) k3 = __ldg(kp + (size_t)(t + 3) * KT);
             if (t >= NS && !mbar_wait(kv_empty(s), (uint32_t)(t / NS - 1) & 1u, &abort_flag)) ok = false;
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
             const uint32_t v_st = stage_base + (uint32_t)s * Sh::STAGE, k_st = v_st + Sh::V_BYTES;
-            expect_tx_elected(kv_full(s), (uint32_t)Sh::V_BYTES / 4);
-            int32_t r4[4];
 #pragma unroll
-            for (int e = 0; e < 4; ++e) r4[e] = row0 + __shfl_sync(0xffffffffu, k, (4 * (lane & 3) + e) & 31);
-            if (lane < 4) tma_gather4(v_st + (uint32_t)(pw * 4 + lane) * 512u, &map_v, r4[0], r4[1], r4[2], r4[3], kv_full(s));
+            for (int i = 0; i < 4; ++i) {
+                const int y = (lane >> 3) + 4 * i;              // key of the warp's sixteen
+                const int32_t kv = __shfl_sync(0xffffffffu, k, y);
+                const int r = pw * 16 + y;
+                asm volatile("cp.async.cg.shared.global [%0], [%1], 16;"
+                             ::"r"(v_st + (uint32_t)(r * 128 + ((vc ^ (r & 7)) << 4))), "l"(Vh + (size_t)kv * D + vc * 8) : "memory");
+            }
 #pragma unroll
             for (int c2 = 0; c2 < M / 16; ++c2) {
                 const int c = 2 * c2 + (lane >> 4);
-                asm volatile("cp.async.ca.shared.global [%0], [%1], 16;"
+                asm volatile("cp.async.cg.shared.global [%0], [%1], 16;"
                              ::"r"(k_st + (uint32_t)(c * KT + ky) * 16u), "l"(Kg + (size_t)k * M + c * 8) : "memory");
             }
             asm volatile("cp.async.commit_group;" ::: "memory");
-            issued = t + 1;
             if (t >= 2) {
                 asm volatile("cp.async.wait_group 2;" ::: "memory");
                 hand_over(t - 2);
@@ -789,41 +803,18 @@ mhat_attention_kernel(int32_t G, int32_t nblocks, int32_t N, const int32_t* __re
             asm volatile("cp.async.wait_group 1;" ::: "memory");
             hand_over(T - 2);
         }
-        asm volatile("cp.async.wait_group 0;" ::: "memory");
+        asm volatile("cp.async.wait_group 0;" ::: "memory");     // also after giving up: no copy outlives the CTA
         if (ok && T > 0) hand_over(T - 1);
-        if (!ok) {
-            // gave up: the last two tiles issued never got this warp's second arrival; then let the gathers still
-            // in flight land (bounded) before the CTA's shared memory is released
-            for (int32_t t = issued > NS ? issued - NS : 0; t < issued; ++t) {
-                if (lane == 0 && t >= issued - 2) mbar_arrive(kv_full(t % NS));
-                __syncwarp();
-                mbar_drain(kv_full(t % NS), (uint32_t)(t / NS) & 1u, 20000000ll);
-            }
-        }
-    } else {
-        // ------------------------------------------------------------ MMA issuer (the whole warp runs the loop in step)
-        constexpr uint32_t idesc_s = instr_desc(KT, false, false);     // S = Q K^T: both operands K-major
-        constexpr uint32_t idesc_o = instr_desc(D, false, true);       // O += P V: V is MN-major (rows of d values)
+    } else if (warp == MH_ISSUER_S) {
+        // ------------------------------------------------------------ S_t = Q K_t^T (the whole warp runs the loop in step)
+        constexpr uint32_t idesc_s = instr_desc(KT, false, false);     // both operands K-major
         bool ok = true;
-        auto weighted_values = [&](int32_t u) {                        // O += P_u V_u
-            const int buf = u & 1, s = u % NS;
-            if (!__all_sync(0xffffffffu, mbar_wait(p_full(buf), (uint32_t)(u >> 1) & 1u, &abort_flag))) { ok = false; return; }
-            fence_after_sync();
-            const uint32_t p_op = tmem_base + (uint32_t)(buf * Sh::S_COLS);
-            const uint32_t v_st = stage_base + (uint32_t)s * Sh::STAGE;
-#pragma unroll
-            for (int ks = 0; ks < KT / 16; ++ks) {
-                const uint64_t bd = swizzled_desc(v_st + (uint32_t)ks * 2048u, 1024u, 1024u, 2);
-                mma_bf16_ts(tmem_base + (uint32_t)Sh::O_COL, p_op + (uint32_t)ks * 8u, bd, idesc_o, (u > 0 || ks > 0) ? 1u : 0u);
-            }
-            mma_commit(kv_empty(s));
-            mma_commit(s_free(buf));
-        };
-        for (int32_t t = 0; t < T && ok; ++t) {
-            const int buf = t & 1, s = t % NS;
+        int buf = 0;
+        for (int32_t t = 0; t < T; ++t) {
+            const int s = t % NS;
             if (!__all_sync(0xffffffffu, mbar_wait(kv_full(s), (uint32_t)(t / NS) & 1u, &abort_flag))) { ok = false; break; }
-            // the score buffer is free once the second product of the tile two back has read its P
-            if (t >= 2 && !__all_sync(0xffffffffu, mbar_wait(s_free(buf), (uint32_t)((t - 2) >> 1) & 1u, &abort_flag))) { ok = false; break; }
+            // the score buffer is free once the second product of the tile three back, which read its P, is complete
+            if (t >= NB && !__all_sync(0xffffffffu, mbar_wait(kv_empty((t - NB) % NS), (uint32_t)((t - NB) / NS) & 1u, &abort_flag))) { ok = false; break; }
             fence_after_sync();
             const uint32_t k_st = stage_base + (uint32_t)s * Sh::STAGE + Sh::V_BYTES;
 #pragma unroll
@@ -833,20 +824,46 @@ mhat_attention_kernel(int32_t G, int32_t nblocks, int32_t N, const int32_t* __re
                 mma_bf16_ss(tmem_base + (uint32_t)(buf * Sh::S_COLS), ad, bd, idesc_s, k > 0 ? 1u : 0u);
             }
             mma_commit(s_full(buf));
-            if (t >= 1) weighted_values(t - 1);
+            if (++buf == NB) buf = 0;
         }
-        if (ok && T > 0) weighted_values(T - 1);
-        if (T > 0) mma_commit(acc_done);
         if (!ok) {
-            mma_commit(drain_bar);
-            mbar_drain(drain_bar, 0u, 20000000ll);
+            mma_commit(drain_s);
+            mbar_drain(drain_s, 0u, 20000000ll);
+        }
+        __syncwarp();
+    } else {
+        // ------------------------------------------------------------ O += P_t V_t (the whole warp runs the loop in step)
+        constexpr uint32_t idesc_o = instr_desc(D, false, true);       // V is MN-major (rows of d values)
+        bool ok = true;
+        int buf = 0;
+        uint32_t par = 0u;
+        for (int32_t t = 0; t < T; ++t) {
+            const int s = t % NS;
+            if (!__all_sync(0xffffffffu, mbar_wait(p_full(buf), par, &abort_flag))) { ok = false; break; }
+            // (complete since the first product of this tile ran; waited on here for this thread's own view of the stage)
+            if (!__all_sync(0xffffffffu, mbar_wait(kv_full(s), (uint32_t)(t / NS) & 1u, &abort_flag))) { ok = false; break; }
+            fence_after_sync();
+            const uint32_t p_op = tmem_base + (uint32_t)(buf * Sh::S_COLS);
+            const uint32_t v_st = stage_base + (uint32_t)s * Sh::STAGE;
+#pragma unroll
+            for (int ks = 0; ks < KT / 16; ++ks) {
+                const uint64_t bd = swizzled_desc(v_st + (uint32_t)ks * 2048u, 1024u, 1024u, 2);
+                mma_bf16_ts(tmem_base + (uint32_t)Sh::O_COL, p_op + (uint32_t)ks * 8u, bd, idesc_o, (t > 0 || ks > 0) ? 1u : 0u);
+            }
+            mma_commit(kv_empty(s));                                   // frees the stage and the score buffer
+            if (++buf == NB) { buf = 0; par ^= 1u; }
+        }
+        if (ok && T > 0) mma_commit(acc_done);
+        if (!ok) {
+            mma_commit(drain_o);
+            mbar_drain(drain_o, 0u, 20000000ll);
         }
         __syncwarp();
     }
 
     fence_before_sync();
     __syncthreads();
-    if (warp == 8) tmem_dealloc(tmem_base, (uint32_t)Sh::TMEM_COLS);
+    if (warp == MH_ISSUER_S) tmem_dealloc(tmem_base, (uint32_t)Sh::TMEM_COLS);
     if (tid == 0 && abort_flag) atomicExch(error_word, 1);
 }
 
@@ -997,8 +1014,6 @@ static int launch_mhat(grf_ctx* ctx, const grf_features* feat, int32_t G, int32_
 {
     using Sh = MhShape<M>;
     const grf_mask_dev& K = feat->mask;
-    CUtensorMap map_v;
-    if (!grf_make_row_gather_map(&map_v, V, (uint64_t)G * N, 64)) return GRF_ERR_INVALID;
     // at most two CTAs per SM: each holds half of the SM's tensor memory
     const size_t smem = Sh::SMEM > 78 * 1024 ? Sh::SMEM : 78 * 1024;
     GRF_CUDA_TRY(cudaFuncSetAttribute(mhat_attention_kernel<M>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
@@ -1006,7 +1021,7 @@ static int launch_mhat(grf_ctx* ctx, const grf_features* feat, int32_t G, int32_
         grf_launch_scope scope(ctx, 9);
         mhat_attention_kernel<M><<<(unsigned)K.blocks * (unsigned)G, MH_THREADS, smem, ctx->stream>>>(
             G, K.blocks, N, (const int32_t*)K.off.ptr, (const int32_t*)K.cnt.ptr, (const int32_t*)K.key.ptr,
-            (const uint4*)K.val.ptr, (const __nv_bfloat16*)phiQ, (const __nv_bfloat16*)phiK, map_v,
+            (const uint4*)K.val.ptr, (const __nv_bfloat16*)phiQ, (const __nv_bfloat16*)phiK, (const __nv_bfloat16*)V,
             (__nv_bfloat16*)out, den_out, ctx->error_word);
     }
     return cudaGetLastError() == cudaSuccess ? GRF_OK : GRF_ERR_CUDA;
