@@ -578,6 +578,8 @@ mask_rows_kernel(int32_t Nk, const int32_t* __restrict__ rows, const int32_t* __
 //   warps 10-13     producers: a quarter of every tile's key-feature and value rows each, by 16-byte async copies
 // An instruction of the tensor pipe costs its issuing thread about fifty cycles, whatever its size, so the two
 // products have a thread each; three score buffers let the first product run two tiles ahead of the masking.
+// (A round trip to tensor memory is about 230 cycles and the hand-overs add several hundred per tile: what bounds
+// the kernel is the length of that chain, not a pipe.)
 
 template <int M> struct MhShape {
     static constexpr int D = 64;
@@ -596,10 +598,34 @@ template <int M> struct MhShape {
 };
 
 constexpr int MH_THREADS = 448;
+
+// two fp32 values in one 64-bit register: the packed multiply and add take one issue slot for both
+__device__ __forceinline__ uint64_t pack_f32x2(uint32_t lo, uint32_t hi)
+{
+    uint64_t r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "r"(lo), "r"(hi));
+    return r;
+}
+__device__ __forceinline__ void unpack_f32x2(uint64_t v, float& lo, float& hi)
+{
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ uint64_t mul_f32x2(uint64_t a, uint64_t b)
+{
+    uint64_t r;
+    asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+    return r;
+}
+__device__ __forceinline__ uint64_t add_f32x2(uint64_t a, uint64_t b)
+{
+    uint64_t r;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+    return r;
+}
 constexpr int MH_ISSUER_S = 8, MH_ISSUER_O = 9, MH_PRODUCER0 = 10;
 
 template <int M>
-__global__ void __launch_bounds__(MH_THREADS)
+__global__ void __launch_bounds__(MH_THREADS, 2)
 mhat_attention_kernel(int32_t G, int32_t nblocks, int32_t N, const int32_t* __restrict__ mk_off,
                       const int32_t* __restrict__ mk_cnt, const int32_t* __restrict__ mk_key,
                       const uint4* __restrict__ mk_val, const __nv_bfloat16* __restrict__ phiQ,
@@ -631,7 +657,7 @@ mhat_attention_kernel(int32_t G, int32_t nblocks, int32_t N, const int32_t* __re
     const uint32_t drain_s = acc_done + 16u, drain_o = acc_done + 24u;
 
     if (tid == 0) {
-        for (int s = 0; s < NS; ++s) { mbar_init(kv_full(s), 4); mbar_init(kv_empty(s), 1); }
+        for (int s = 0; s < NS; ++s) { mbar_init(kv_full(s), 128); mbar_init(kv_empty(s), 1); }
         for (int b = 0; b < NB; ++b) { mbar_init(s_full(b), 1); mbar_init(p_full(b), 4); }
         mbar_init(acc_done, 1);
         mbar_init(den_ready, 4);
@@ -667,7 +693,7 @@ mhat_attention_kernel(int32_t G, int32_t nblocks, int32_t N, const int32_t* __re
         const int32_t row = blk * BQ + rr;
         const uint32_t lane_field = (uint32_t)((warp & 3) * 32) << 16;
         const uint4* mrow = mk_val + (size_t)(off / 8) * BQ + rr;       // chunk x of this row: mrow[x * BQ]
-        float den = 0.0f;
+        uint64_t den2[2] = {0ull, 0ull};                         // row sums, four partial sums in two packed pairs
         uint4 mk[KT / 8];
         if (grp < T) {
 #pragma unroll
@@ -693,11 +719,13 @@ mhat_attention_kernel(int32_t G, int32_t nblocks, int32_t N, const int32_t* __re
                     const uint32_t mw[4] = {mm.x, mm.y, mm.z, mm.w};
 #pragma unroll
                     for (int e = 0; e < 4; ++e) {
-                        const float p0 = __uint_as_float(sv[8 * h + 2 * e]) * __uint_as_float(mw[e] << 16);
-                        const float p1 = __uint_as_float(sv[8 * h + 2 * e + 1]) * __uint_as_float(mw[e] & 0xffff0000u);
+                        // two masked scores at a time; the denominator adds them in fp32, before the rounding to bf16
+                        const uint64_t p2 = mul_f32x2(pack_f32x2(sv[8 * h + 2 * e], sv[8 * h + 2 * e + 1]),
+                                                      pack_f32x2(mw[e] << 16, mw[e] & 0xffff0000u));
+                        den2[e & 1] = add_f32x2(den2[e & 1], p2);
+                        float p0, p1;
+                        unpack_f32x2(p2, p0, p1);
                         const __nv_bfloat162 pb = __floats2bfloat162_rn(p0, p1);
-                        // the denominator adds the same rounded values the second product multiplies
-                        den += __low2float(pb) + __high2float(pb);
                         pw[4 * h + e] = *reinterpret_cast<const uint32_t*>(&pb);
                     }
                 }
@@ -714,6 +742,13 @@ mhat_attention_kernel(int32_t G, int32_t nblocks, int32_t N, const int32_t* __re
             if (lane == 0) mbar_arrive(p_full(buf));
             buf += 2;
             if (buf >= NB) { buf -= NB; par ^= 1u; }
+        }
+        float den;
+        {
+            float d0, d1, d2, d3;
+            unpack_f32x2(den2[0], d0, d1);
+            unpack_f32x2(den2[1], d2, d3);
+            den = (d0 + d1) + (d2 + d3);
         }
         if (grp == 1) {
             // hand the odd tiles' row sums to the first group, which writes the block's outputs
@@ -755,19 +790,15 @@ mhat_attention_kernel(int32_t G, int32_t nblocks, int32_t N, const int32_t* __re
         // bytes): eight consecutive lanes copy one row, piece c of tile row r going to r * 128 + ((c ^ (r & 7)) * 16),
         // the 128-byte swizzle the second product's operand descriptor names.  Key-feature rows: piece c of key y
         // goes to (c * 64 + y) * 16; lanes 0-15 copy the even pieces, lanes 16-31 the odd ones.  A warp's copies of
-        // one tile form one group; it hands its part of a stage over two tiles late, after that group has completed
-        // and a proxy fence.  Key indices are read three tiles ahead.
+        // one tile arrive on the stage's barrier by themselves as they land (the barrier counts all 128 producer
+        // threads), so a producer never waits for its own copies; the issuing threads run the proxy fence between
+        // their wait on that barrier and the product that reads the stage.  Key indices are read three tiles ahead.
         const int pw = warp - MH_PRODUCER0;
         const __nv_bfloat16* Kg = phiK + (size_t)g * N * M;
         const __nv_bfloat16* Vh = Vg + (size_t)g * N * D;
         const int ky = pw * 16 + (lane & 15);                   // this lane's key within the tile
         const int vc = lane & 7;                                // its piece of a value row
         bool ok = true;
-        auto hand_over = [&](int32_t t) {
-            fence_async_smem();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(kv_full(t % NS));
-        };
         const int32_t* kp = mk_key + off + ky;
         int32_t k1 = T > 0 ? __ldg(kp) : 0, k2 = T > 1 ? __ldg(kp + KT) : 0, k3 = T > 2 ? __ldg(kp + 2 * KT) : 0;
         for (int32_t t = 0; t < T; ++t) {
@@ -793,18 +824,10 @@ mhat_attention_kernel(int32_t G, int32_t nblocks, int32_t N, const int32_t* __re
                 asm volatile("cp.async.cg.shared.global [%0], [%1], 16;"
                              ::"r"(k_st + (uint32_t)(c * KT + ky) * 16u), "l"(Kg + (size_t)k * M + c * 8) : "memory");
             }
-            asm volatile("cp.async.commit_group;" ::: "memory");
-            if (t >= 2) {
-                asm volatile("cp.async.wait_group 2;" ::: "memory");
-                hand_over(t - 2);
-            }
+            // every thread's arrival on the stage's barrier happens when its own copies above have landed
+            asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(kv_full(s)) : "memory");
         }
-        if (ok && T >= 2) {
-            asm volatile("cp.async.wait_group 1;" ::: "memory");
-            hand_over(T - 2);
-        }
-        asm volatile("cp.async.wait_group 0;" ::: "memory");     // also after giving up: no copy outlives the CTA
-        if (ok && T > 0) hand_over(T - 1);
+        asm volatile("cp.async.wait_all;" ::: "memory");         // also after giving up: no copy outlives the CTA
     } else if (warp == MH_ISSUER_S) {
         // ------------------------------------------------------------ S_t = Q K_t^T (the whole warp runs the loop in step)
         constexpr uint32_t idesc_s = instr_desc(KT, false, false);     // both operands K-major
@@ -815,6 +838,7 @@ mhat_attention_kernel(int32_t G, int32_t nblocks, int32_t N, const int32_t* __re
             if (!__all_sync(0xffffffffu, mbar_wait(kv_full(s), (uint32_t)(t / NS) & 1u, &abort_flag))) { ok = false; break; }
             // the score buffer is free once the second product of the tile three back, which read its P, is complete
             if (t >= NB && !__all_sync(0xffffffffu, mbar_wait(kv_empty((t - NB) % NS), (uint32_t)((t - NB) / NS) & 1u, &abort_flag))) { ok = false; break; }
+            fence_async_smem();                                        // the copies wrote through the generic proxy
             fence_after_sync();
             const uint32_t k_st = stage_base + (uint32_t)s * Sh::STAGE + Sh::V_BYTES;
 #pragma unroll
@@ -842,6 +866,7 @@ mhat_attention_kernel(int32_t G, int32_t nblocks, int32_t N, const int32_t* __re
             if (!__all_sync(0xffffffffu, mbar_wait(p_full(buf), par, &abort_flag))) { ok = false; break; }
             // (complete since the first product of this tile ran; waited on here for this thread's own view of the stage)
             if (!__all_sync(0xffffffffu, mbar_wait(kv_full(s), (uint32_t)(t / NS) & 1u, &abort_flag))) { ok = false; break; }
+            fence_async_smem();
             fence_after_sync();
             const uint32_t p_op = tmem_base + (uint32_t)(buf * Sh::S_COLS);
             const uint32_t v_st = stage_base + (uint32_t)s * Sh::STAGE;
