@@ -583,7 +583,9 @@ mask_rows_kernel(int32_t Nk, const int32_t* __restrict__ rows, const int32_t* __
 
 template <int M> struct MhShape {
     static constexpr int D = 64;
-    static constexpr int NS = M <= 32 ? 8 : 6;            // key/value stages in flight
+    // key/value stages in flight: two CTAs' rings then leave the SM the larger part of its L1, which serves the mask
+    // values and the rows that neighbouring keys share (eight stages were 8 % slower at the point cloud, 25 % at the grid)
+    static constexpr int NS = M <= 32 ? 5 : 3;
     static constexpr int NB = 3;                          // score buffers
     static constexpr int V_BYTES = KT * 128;              // 64 value rows of 128 bytes, 128-byte swizzle
     static constexpr int K_BYTES = KT * M * 2;            // [M/8][KT keys][8] bf16: K-major, unswizzled
