@@ -514,10 +514,31 @@ __global__ void __launch_bounds__(256) block_order_kernel(int32_t nblocks, int32
 
 }  // namespace
 
-int grf_build_block_plan(grf_ctx* ctx, grf_features* feat)
+// The coefficient table of the tensor-core gather (Phi's values per union entry and row), for a plan that is ready.
+static int build_plan_coefficients(grf_ctx* ctx, grf_features* feat)
+{
+    grf_csr_dev& phi = feat->phi;
+    const int32_t N = phi.rows, R = phi.cols;
+    const size_t words = (size_t)(R + 31) / 32;
+    const size_t table_bytes = (size_t)feat->plan_entries * BQ * sizeof(__nv_bfloat16);
+    if (feat->plan_coef.bytes < table_bytes) GRF_TRY(grf_buf_reserve(&feat->plan_coef, table_bytes + table_bytes / 8));
+    GRF_CUDA_TRY(cudaFuncSetAttribute(block_coef_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(words * 8)));
+    {
+        grf_launch_scope scope(ctx, 7);
+        block_coef_kernel<<<feat->plan_blocks, 256, words * 8, ctx->stream>>>(
+            N, R, (const int32_t*)phi.rowptr.ptr, (const int32_t*)phi.col.ptr, (const float*)phi.val.ptr,
+            (const int32_t*)feat->plan_off.ptr, (const int32_t*)feat->plan_cnt.ptr, (__nv_bfloat16*)feat->plan_coef.ptr);
+    }
+    GRF_CUDA_TRY(cudaGetLastError());
+    feat->plan_coef_ready = true;
+    return GRF_OK;
+}
+
+int grf_build_block_plan(grf_ctx* ctx, grf_features* feat, bool with_coef)
 {
     grf_csr_dev& phi = feat->phi;
     feat->plan_ready = false;
+    feat->plan_coef_ready = false;
     const int32_t N = phi.rows, R = phi.cols;
     const size_t words = (size_t)(R + 31) / 32;
     if (words * 8 > 200 * 1024 || phi.nnz <= 0) return GRF_OK;   // no plan: the ALU kernel serves this object
@@ -545,19 +566,10 @@ int grf_build_block_plan(grf_ctx* ctx, grf_features* feat)
     const size_t entries = (size_t)ctx->pinned[4];
     const size_t table_bytes = entries * BQ * sizeof(__nv_bfloat16);
     if (table_bytes > ((size_t)2 << 30)) return GRF_OK;           // too little sharing between neighbouring rows
-    if (feat->plan_coef.bytes < table_bytes) GRF_TRY(grf_buf_reserve(&feat->plan_coef, table_bytes + table_bytes / 8));
-    GRF_CUDA_TRY(cudaFuncSetAttribute(block_coef_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(words * 8)));
-    {
-        grf_launch_scope scope(ctx, 7);
-        block_coef_kernel<<<nblocks, 256, words * 8, ctx->stream>>>(
-            N, R, (const int32_t*)phi.rowptr.ptr, (const int32_t*)phi.col.ptr, (const float*)phi.val.ptr,
-            (const int32_t*)feat->plan_off.ptr, (const int32_t*)feat->plan_cnt.ptr, (__nv_bfloat16*)feat->plan_coef.ptr);
-    }
-    GRF_CUDA_TRY(cudaGetLastError());
     feat->plan_blocks = nblocks;
     feat->plan_entries = (int64_t)entries;
     feat->plan_ready = true;
-    return GRF_OK;
+    return with_coef ? build_plan_coefficients(ctx, feat) : GRF_OK;
 }
 
 extern "C" int grf_debug_wait_timeout(grf_ctx* ctx, int64_t limit_cycles)
@@ -612,13 +624,18 @@ static int launch_tc(grf_ctx* ctx, const grf_features* feat, int32_t G, int32_t 
     return cudaGetLastError() == cudaSuccess ? GRF_OK : GRF_ERR_CUDA;
 }
 
-// The plan is a cache inside the feature object, built on first use (the asymmetric route never needs it).
-int grf_ensure_block_plan(grf_ctx* ctx, const grf_features* feat)
+// The plan is a cache inside the feature object, built on first use (the asymmetric route never needs it); the
+// route over the materialised mask uses its node lists but not the coefficient table, which is then left out until
+// the gather kernel asks for it.
+int grf_ensure_block_plan(grf_ctx* ctx, const grf_features* feat, bool with_coef)
 {
-    if (!feat->plan_stale) return GRF_OK;
     grf_features* f = const_cast<grf_features*>(feat);
-    GRF_TRY(grf_build_block_plan(ctx, f));
-    f->plan_stale = false;
+    if (feat->plan_stale) {
+        GRF_TRY(grf_build_block_plan(ctx, f, with_coef));
+        f->plan_stale = false;
+        return GRF_OK;
+    }
+    if (with_coef && feat->plan_ready && !feat->plan_coef_ready) return build_plan_coefficients(ctx, f);
     return GRF_OK;
 }
 

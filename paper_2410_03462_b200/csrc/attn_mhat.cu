@@ -917,7 +917,7 @@ extern "C" int grf_features_materialise(grf_ctx* ctx, grf_features* feat)
     // the values kernel keeps the key bitmap, its prefix counts and the accumulators in shared memory
     const size_t smem_values = ((words + 1) & ~(size_t)1) * 8 + (size_t)MASK_WARPS * MASK_SEG * sizeof(float);
     if (smem_values > 200 * 1024) return GRF_ERR_TOO_LARGE;
-    GRF_TRY(grf_ensure_block_plan(ctx, feat));
+    GRF_TRY(grf_ensure_block_plan(ctx, feat, false));         // the node lists only
     if (!feat->plan_ready) return GRF_ERR_TOO_LARGE;          // rows of a block share too little
     const int32_t nblocks = feat->plan_blocks;
     GRF_TRY(grf_buf_reserve(&K.cnt, sizeof(int32_t) * 2 * (size_t)nblocks));

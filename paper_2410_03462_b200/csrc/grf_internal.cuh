@@ -118,6 +118,7 @@ struct grf_features {
     int32_t plan_blocks = 0;
     int64_t plan_entries = 0;       // node-list entries over all blocks (padded to multiples of 4)
     bool plan_ready = false;
+    bool plan_coef_ready = false;   // the gather kernel's coefficient table exists for the present plan
     bool plan_stale = true;         // Phi changed since the plan was built: the gather kernel's launcher rebuilds it
 };
 
@@ -160,8 +161,8 @@ int grf_gather_contract_alu(grf_ctx* ctx, const grf_csr_dev& phi, int32_t G, int
 void grf_mask_invalidate(grf_features* feat);
 void grf_mask_release(grf_features* feat);
 // attn_gather_tc.cu
-int grf_build_block_plan(grf_ctx* ctx, grf_features* feat);
-int grf_ensure_block_plan(grf_ctx* ctx, const grf_features* feat);   // builds it if Phi changed since the last build
+int grf_build_block_plan(grf_ctx* ctx, grf_features* feat, bool with_coef = true);
+int grf_ensure_block_plan(grf_ctx* ctx, const grf_features* feat, bool with_coef = true);   // builds it if Phi changed since the last build
 int grf_gather_contract_tc(grf_ctx* ctx, const grf_features* feat, int32_t G, int32_t N, int32_t m, int32_t d,
                            const void* phiQ, const void* records, void* out, float* den_out);
 
