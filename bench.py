@@ -262,7 +262,10 @@ DTYPE_NOTE = {
 }
 
 
-def measure(args, workload_name, route, with_cpu_baseline, with_e2e, frozen=False, steps=None, warmup=None):
+def measure(args, workload_name, route, with_cpu_baseline, with_e2e, frozen=False, steps=None, warmup=None,
+            remodulate=False):
+    """remodulate: the walks are sampled once and kept; every step gives them new coefficients (Alg. 1 with learnable
+    f: grf_remodulate), prepares the feature object again and runs the attention."""
     import torch
     import torch.distributed as dist
 
@@ -306,6 +309,11 @@ def measure(args, workload_name, route, with_cpu_baseline, with_e2e, frozen=Fals
     feat = api.Features(ctx, None)
 
     def sample(seed):
+        if remodulate and feat.handle is not None:
+            # same walks, new coefficients (a small change of every f_t that differs from step to step)
+            fi = (f * np.float32(1.0 - 0.001 * (seed % 7))).astype(np.float32)
+            B.grf_remodulate(ctx.handle, feat.handle, w.max_len, fi, None if f_psi is None else f_psi)
+            return
         feat.handle = B.grf_sample(ctx.handle, N, dg.rowptr, dg.col, dg.w, seed, w.n_walks, w.p_halt, w.max_len, f, f_psi,
                                    feat.handle)
 
@@ -330,6 +338,11 @@ def measure(args, workload_name, route, with_cpu_baseline, with_e2e, frozen=Fals
 
     sampler = ClockSampler(local) if rank == 0 else None
     B.grf_ctx_enable_timing(ctx.handle, True)      # per-kernel events exist before the timed region starts
+    if remodulate:                                  # the walks themselves are kept with the features
+        B.grf_ctx_keep_walks(ctx.handle, True)
+        sample(configs.WALK_SEED)
+        B.grf_ctx_keep_walks(ctx.handle, False)
+        prepare()
     if frozen:                                      # walks "pre-computed and frozen" (Sec. 4): outside the step
         sample(configs.WALK_SEED)
         prepare()
@@ -383,7 +396,7 @@ def measure(args, workload_name, route, with_cpu_baseline, with_e2e, frozen=Fals
 
     # ---- end to end through the host-buffer entry point (pinned host memory; copies inside the timing)
     e2e = None
-    if with_e2e and route in ("sz", "mhat") and not frozen:
+    if with_e2e and route in ("sz", "mhat") and not frozen and not remodulate:
         B.grf_ctx_prefer_mask_route(ctx.handle, mhat)
         qh, kh, vh = q.pin_memory(), k.pin_memory(), v.pin_memory()
         oh = torch.empty_like(v).pin_memory()
@@ -473,9 +486,12 @@ def measure(args, workload_name, route, with_cpu_baseline, with_e2e, frozen=Fals
                        "nnz_phi": nnz_phi, "nnz_psi": nnz_psi,
                        "node_order": "as given" if "unsorted" in w.name else
                                      ("Morton order of the points" if "pointcloud" in w.name else "generator's order"),
-                       "features": "frozen: sampled once before the timed region" if frozen else "resampled every step",
+                       "features": "frozen: sampled once before the timed region" if frozen else
+                                   ("walks sampled once and kept; new coefficients every step (grf_remodulate)" if remodulate
+                                    else "resampled every step"),
                        "l2": "256 MiB flush write between steps, outside the per-step events",
-                       "step": step_text + (", attention only (features frozen)" if frozen else ", features resampled every step")},
+                       "step": step_text.replace("grf_sample (both ensembles)", "grf_remodulate") + ", walks kept" if remodulate else
+                               step_text + (", attention only (features frozen)" if frozen else ", features resampled every step")},
             "clocks": clocks,
             "gpu_launches": launches,
             "e2e": None if not e2e else
@@ -492,7 +508,7 @@ def measure(args, workload_name, route, with_cpu_baseline, with_e2e, frozen=Fals
             "phases": {"sample_ms": statistics.mean(sample_ms), "attn_ms": statistics.mean(attn_ms),
                        "sample_ms_min_med_max": [min(sample_ms), statistics.median(sample_ms), max(sample_ms)],
                        "attn_ms_min_med_max": [min(attn_ms), statistics.median(attn_ms), max(attn_ms)],
-                       "walks_per_s": None if frozen else 2 * N * w.n_walks / (statistics.mean(sample_ms) * 1e-3),
+                       "walks_per_s": None if (frozen or remodulate) else 2 * N * w.n_walks / (statistics.mean(sample_ms) * 1e-3),
                        "attn_tokens_per_s": w.batch * N / (statistics.mean(attn_ms) * 1e-3),
                        "attn_hbm_frac": (2 * w.G * N * w.m * w.d * es + w.G * N * (2 * w.m + 2 * w.d) * es) / 1e9 /
                                         (statistics.mean(attn_ms) * 1e-3) / pk["hbm_gbs"] if route == "sz" else None,
@@ -623,17 +639,18 @@ def loglog_slope(xs, ys):
 
 
 def run_suite(args):
-    """All workloads on both symmetric routes, the unsorted point cloud, frozen features, the sweep 2^10..2^20 (sz
+    """All workloads on both symmetric routes, the unsorted point cloud, frozen and re-modulated features, the sweep 2^10..2^20 (sz
     route) with the fitted slopes, and the operation counts; writes <dir>/bench_suite.jsonl and <dir>/bench_suite.md."""
     os.makedirs(args.suite_dir, exist_ok=True)
     lines, md = [], []
 
-    def run(name, route, frozen=False, steps=10):
+    def run(name, route, frozen=False, steps=10, remodulate=False):
         from paper_2410_03462_b200 import binding as B
-        case = f"{name}/{route}" + ("/frozen" if frozen else "")
+        case = f"{name}/{route}" + ("/frozen" if frozen else "") + ("/remodulated" if remodulate else "")
         try:
-            r = measure(args, name, route, False, route == "sz" and not frozen and name in ("pc32768", "vit", "pc4096"),
-                        frozen=frozen, steps=steps, warmup=3)
+            r = measure(args, name, route, False,
+                        route == "sz" and not frozen and not remodulate and name in ("pc32768", "vit", "pc4096"),
+                        frozen=frozen, steps=steps, warmup=3, remodulate=remodulate)
         except B.GrfError as e:          # e.g. the materialised mask of a graph without locality exceeds its limit
             lines.append({"suite_case": case, "error": str(e)})
             md.append(f"| {case} | not run: {e} |")
@@ -661,6 +678,9 @@ def run_suite(args):
             row(run(name, "sz", frozen=True))
             row(run(name, "mhat"))
             row(run(name, "mhat", frozen=True))
+            if name in ("vit", "pc32768"):
+                row(run(name, "sz", remodulate=True))
+                row(run(name, "mhat", remodulate=True))
     sweep = []
     for k in range(10, 21):
         r = run(f"sweep{k}", "sz", steps=10 if k < 18 else 4)
@@ -711,6 +731,8 @@ def main():
                          "materialised mask Phi Psi^T; asym: Alg. 2 (asymmetric features, Psi = I); the last two are "
                          "variants outside the headline metric")
     ap.add_argument("--frozen", action="store_true", help="features sampled (and prepared) once, outside the timed steps")
+    ap.add_argument("--remodulate", action="store_true",
+                    help="walks sampled once and kept; every timed step re-modulates them with new coefficients")
     ap.add_argument("--softmax", action="store_true", help="with --route asym: A_ij = exp(q_i . k_j)")
     ap.add_argument("--heads", type=int, default=0, help="override the workload's head count (profiling of a smaller case)")
     ap.add_argument("--no-other-routes", action="store_true", help="skip the short runs of the other routes beside the headline")
@@ -734,18 +756,21 @@ def main():
         if args.suite:
             res = run_suite(args)
         else:
-            res = measure(args, args.workload, args.route, not args.no_cpu_baseline, True, frozen=args.frozen)
+            res = measure(args, args.workload, args.route, not args.no_cpu_baseline, True, frozen=args.frozen,
+                          remodulate=args.remodulate)
             # beside the headline (the route through the per-node states, features resampled every step): the same
             # workload on the route over the materialised mask, and both routes with frozen features, in short runs
-            if res is not None and world == 1 and args.route == "sz" and not args.frozen and not args.no_other_routes:
+            if res is not None and world == 1 and args.route == "sz" and not args.frozen and not args.remodulate and not args.no_other_routes:
                 w = make_workload(args.workload)
                 if w.dtype == "bf16" and w.d == 64 and w.m in (16, 32, 64):
                     from paper_2410_03462_b200 import binding as B
                     others = {}
                     for name, route, frozen in (("mhat_resampled", "mhat", False), ("mhat_frozen", "mhat", True),
-                                                ("sz_frozen", "sz", True)):
+                                                ("sz_frozen", "sz", True), ("mhat_remodulated", "mhat", "remod"),
+                                                ("sz_remodulated", "sz", "remod")):
                         try:
-                            r = measure(args, args.workload, route, False, False, frozen=frozen, steps=min(args.steps, 10), warmup=3)
+                            r = measure(args, args.workload, route, False, False, frozen=(frozen is True),
+                                        remodulate=(frozen == "remod"), steps=min(args.steps, 10), warmup=3)
                         except B.GrfError as e:
                             others[name] = {"error": str(e)}
                             continue

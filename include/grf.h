@@ -94,8 +94,10 @@ int grf_sample(grf_ctx* ctx, int32_t N, const int32_t* rowptr, const int32_t* co
  * grf_remodulate: gives a feature object sampled in that mode new coefficients (HOST arrays of max_len + 1
  * values, max_len as sampled; f_psi == NULL means f_phi).  Values become sum (f_t * load) * (1 / n_walks) over the
  * entry's deposits, same operations and order as the sampler's: the result is bit-identical to sampling again
- * with the same seed and the new coefficients, without any walk being taken.  Psi^T is regrouped.  Asynchronous.
- * GRF_ERR_INVALID if the object holds no deposits or max_len differs.
+ * with the same seed and the new coefficients, without any walk being taken.  Psi^T receives the new values through
+ * the entry order recorded at the first call.  The index structure is unchanged, so what was derived from it stays:
+ * the next attention call rebuilds only the coefficient table of its block plan, the next grf_features_materialise
+ * only the mask's values.  Asynchronous.  GRF_ERR_INVALID if the object holds no deposits or max_len differs.
  */
 int grf_ctx_keep_walks(grf_ctx* ctx, int enable);
 int grf_remodulate(grf_ctx* ctx, grf_features* feat, int32_t max_len, const float* f_phi, const float* f_psi);
@@ -218,8 +220,10 @@ int grf_masked_attn_asym(grf_ctx* ctx, const grf_features* feat, int32_t G, int3
  *
  * grf_features_materialise: forms Mhat once for a feature object (N x N; Phi and Psi may be N x R) as dense bf16
  * blocks, one per 128 consecutive rows, over the sorted list of keys the block reaches (sums in fp32, fixed order).
- * Needs the block plan of Phi (built here if absent).  Waits for the stream twice.  The mask is dropped when the
- * object is resampled or re-modulated.  GRF_ERR_TOO_LARGE when N > 294912 or the blocks would exceed 8 GiB (no
+ * Needs the node lists of Phi's block plan (built here if absent).  Waits for the stream twice.  The mask is dropped
+ * when the object is resampled; after grf_remodulate its values are stale (grf_mask_stats, grf_mask_rows and
+ * grf_masked_attn_mhat return GRF_ERR_INVALID) until this call forms them again, which then takes one kernel over
+ * the key lists already in place and does not wait for the stream.  GRF_ERR_TOO_LARGE when N > 294912 or the blocks would exceed 8 GiB (no
  * locality: use grf_masked_linear_attn).
  * grf_mask_stats: HOST outputs (any may be NULL): number of blocks, key entries summed over the blocks (padded
  * to multiples of 64), device bytes held.  GRF_ERR_INVALID when the object holds no mask.
@@ -227,8 +231,8 @@ int grf_masked_attn_asym(grf_ctx* ctx, const grf_features* feat, int32_t G, int3
  * rows: DEVICE int32 [n].  Asynchronous.
  * grf_masked_attn_mhat: out_i = sum_j Mhat_ij (phi(q_i).phi(k_j)) v_j / sum_j Mhat_ij (phi(q_i).phi(k_j)) for G
  * problems; arguments as grf_masked_linear_attn, no workspace.  dtype GRF_DTYPE_BF16, d = 64, m in {16, 32, 64}
- * (other shapes: GRF_ERR_INVALID); scores are fp32, the masked scores are rounded to bf16 before they multiply V and
- * before they are added into the denominator.  Summation order is fixed.  Asynchronous.
+ * (other shapes: GRF_ERR_INVALID); scores are fp32, the masked scores are added into the denominator in fp32 and
+ * rounded to bf16 before they multiply V.  Summation order is fixed.  Asynchronous.
  */
 int grf_features_materialise(grf_ctx* ctx, grf_features* feat);
 int grf_mask_stats(const grf_features* feat, int32_t* blocks, int64_t* key_entries, int64_t* bytes);

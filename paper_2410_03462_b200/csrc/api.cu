@@ -212,6 +212,7 @@ extern "C" int grf_features_free(grf_features* feat)
     for (int e = 0; e < 2; ++e) {
         grf_buf_release(&feat->kept.dep_ptr[e]); grf_buf_release(&feat->kept.dep_t[e]); grf_buf_release(&feat->kept.dep_load[e]);
     }
+    grf_buf_release(&feat->kept.psit_perm);
     delete feat;
     return GRF_OK;
 }

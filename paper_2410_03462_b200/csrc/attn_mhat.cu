@@ -896,7 +896,38 @@ mhat_attention_kernel(int32_t G, int32_t nblocks, int32_t N, const int32_t* __re
 
 }  // namespace
 
-void grf_mask_invalidate(grf_features* feat) { feat->mask.ready = false; }
+void grf_mask_invalidate(grf_features* feat) { feat->mask.ready = false; feat->mask.structure_ready = false; }
+// Phi's and Psi's values changed, their structure did not (re-modulation): key lists and positions stay
+void grf_mask_values_stale(grf_features* feat) { feat->mask.ready = false; }
+
+namespace {
+// The values of the mask from the present values of Phi and Psi^T, over key lists (and positions) that are in place.
+int launch_mask_values(grf_ctx* ctx, grf_features* feat, bool by_position)
+{
+    grf_mask_dev& K = feat->mask;
+    const int32_t N = feat->phi.rows, Nk = feat->psi.rows, nblocks = feat->plan_blocks;
+    const size_t words = ((size_t)Nk + 31) / 32;
+    if (by_position) {
+        const size_t smem_acc = (size_t)MASK_WARPS * MASK_SEG * sizeof(float);
+        GRF_CUDA_TRY(cudaFuncSetAttribute(mask_values_pos_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_acc));
+        grf_launch_scope scope(ctx, 8);
+        mask_values_pos_kernel<<<nblocks * (BQ / MASK_ROWS), MASK_WARPS * 32, smem_acc, ctx->stream>>>(
+            N, (const int32_t*)feat->phi.rowptr.ptr, (const int32_t*)feat->phi.col.ptr, (const float*)feat->phi.val.ptr,
+            (const int32_t*)K.phi_pos.ptr, (const int32_t*)feat->psit.rowptr.ptr, (const float*)feat->psit.val.ptr,
+            (const unsigned short*)K.pos16.ptr, (const int32_t*)K.off.ptr, (const int32_t*)K.cnt.ptr,
+            (__nv_bfloat16*)K.val.ptr);
+    } else {
+        const size_t smem_values = ((words + 1) & ~(size_t)1) * 8 + (size_t)MASK_WARPS * MASK_SEG * sizeof(float);
+        GRF_CUDA_TRY(cudaFuncSetAttribute(mask_values_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_values));
+        grf_launch_scope scope(ctx, 8);
+        mask_values_kernel<<<nblocks * (BQ / MASK_ROWS), MASK_WARPS * 32, smem_values, ctx->stream>>>(
+            N, Nk, (const int32_t*)feat->phi.rowptr.ptr, (const int32_t*)feat->phi.col.ptr, (const float*)feat->phi.val.ptr,
+            (const int32_t*)feat->psit.rowptr.ptr, (const int32_t*)feat->psit.col.ptr, (const float*)feat->psit.val.ptr,
+            (const int32_t*)K.off.ptr, (const int32_t*)K.cnt.ptr, (const uint32_t*)K.bits.ptr, (__nv_bfloat16*)K.val.ptr);
+    }
+    return cudaGetLastError() == cudaSuccess ? GRF_OK : GRF_ERR_CUDA;
+}
+}  // namespace
 
 void grf_mask_release(grf_features* feat)
 {
@@ -904,6 +935,7 @@ void grf_mask_release(grf_features* feat)
     grf_buf_release(&K.off); grf_buf_release(&K.cnt); grf_buf_release(&K.key); grf_buf_release(&K.bits); grf_buf_release(&K.val); grf_buf_release(&K.node_off);
     grf_buf_release(&K.blk_pos); grf_buf_release(&K.pos16); grf_buf_release(&K.phi_pos);
     K.ready = false;
+    K.structure_ready = false;
 }
 
 extern "C" int grf_features_materialise(grf_ctx* ctx, grf_features* feat)
@@ -912,6 +944,13 @@ extern "C" int grf_features_materialise(grf_ctx* ctx, grf_features* feat)
     GRF_CUDA_TRY(cudaSetDevice(ctx->device));
     grf_mask_dev& K = feat->mask;
     K.ready = false;
+    if (K.structure_ready && feat->plan_ready && !feat->plan_stale) {
+        // same walks, new coefficients: the key lists and positions still hold
+        GRF_TRY(launch_mask_values(ctx, feat, K.by_position));
+        K.ready = true;
+        return GRF_OK;
+    }
+    K.structure_ready = false;
     const int32_t N = feat->phi.rows, Nk = feat->psi.rows;
     const size_t words = ((size_t)Nk + 31) / 32;
     // the values kernel keeps the key bitmap, its prefix counts and the accumulators in shared memory
@@ -989,25 +1028,13 @@ extern "C" int grf_features_materialise(grf_ctx* ctx, grf_features* feat)
                 (const int32_t*)feat->psit.rowptr.ptr, (const int32_t*)feat->psit.col.ptr, (const uint32_t*)K.bits.ptr,
                 (const int32_t*)K.node_off.ptr, blk_pos, (unsigned short*)K.pos16.ptr, (int32_t*)K.phi_pos.ptr);
         }
-        const size_t smem_acc = (size_t)MASK_WARPS * MASK_SEG * sizeof(float);
-        GRF_CUDA_TRY(cudaFuncSetAttribute(mask_values_pos_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_acc));
-        grf_launch_scope scope(ctx, 8);
-        mask_values_pos_kernel<<<nblocks * (BQ / MASK_ROWS), MASK_WARPS * 32, smem_acc, ctx->stream>>>(
-            N, (const int32_t*)feat->phi.rowptr.ptr, (const int32_t*)feat->phi.col.ptr, (const float*)feat->phi.val.ptr,
-            (const int32_t*)K.phi_pos.ptr, (const int32_t*)feat->psit.rowptr.ptr, (const float*)feat->psit.val.ptr,
-            (const unsigned short*)K.pos16.ptr, (const int32_t*)K.off.ptr, (const int32_t*)K.cnt.ptr,
-            (__nv_bfloat16*)K.val.ptr);
-    } else {
-        GRF_CUDA_TRY(cudaFuncSetAttribute(mask_values_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_values));
-        grf_launch_scope scope(ctx, 8);
-        mask_values_kernel<<<nblocks * (BQ / MASK_ROWS), MASK_WARPS * 32, smem_values, ctx->stream>>>(
-            N, Nk, (const int32_t*)feat->phi.rowptr.ptr, (const int32_t*)feat->phi.col.ptr, (const float*)feat->phi.val.ptr,
-            (const int32_t*)feat->psit.rowptr.ptr, (const int32_t*)feat->psit.col.ptr, (const float*)feat->psit.val.ptr,
-            (const int32_t*)K.off.ptr, (const int32_t*)K.cnt.ptr, (const uint32_t*)K.bits.ptr, (__nv_bfloat16*)K.val.ptr);
     }
+    GRF_TRY(launch_mask_values(ctx, feat, by_position));
     GRF_CUDA_TRY(cudaGetLastError());
     K.blocks = nblocks;
     K.entries = entries;
+    K.by_position = by_position;
+    K.structure_ready = true;
     K.ready = true;
     return GRF_OK;
 }

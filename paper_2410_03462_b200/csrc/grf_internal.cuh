@@ -89,6 +89,8 @@ struct grf_kept_walks {
     int32_t n_walks = 0, max_len = 0;
     int64_t deposits[2] = {0, 0};
     grf_buf dep_ptr[2], dep_t[2], dep_load[2];
+    bool perm_valid = false;        // psit_perm[x] = the entry of Psi that entry x of Psi^T copies (built by the first re-modulation)
+    grf_buf psit_perm;
 };
 
 // The mask estimate Mhat = Phi Psi^T held as dense blocks: for every block of GRF_PLAN_BLOCK consecutive rows the
@@ -97,6 +99,8 @@ struct grf_kept_walks {
 #define GRF_MASK_TILE 64
 struct grf_mask_dev {
     bool ready = false;
+    bool structure_ready = false;   // key lists (and positions) match the features' structure; values may be stale
+    bool by_position = false;       // which of the two value kernels the structure serves
     int32_t blocks = 0;
     int64_t entries = 0;            // padded key entries over all blocks
     grf_buf off, cnt, key;          // cnt holds [blocks] padded counts, then [blocks] the blocks by decreasing count
@@ -159,6 +163,7 @@ int grf_gather_contract_alu(grf_ctx* ctx, const grf_csr_dev& phi, int32_t G, int
                             int dtype, const void* phiQ, const void* records, void* out, float* den_out);
 // attn_mhat.cu
 void grf_mask_invalidate(grf_features* feat);
+void grf_mask_values_stale(grf_features* feat);
 void grf_mask_release(grf_features* feat);
 // attn_gather_tc.cu
 int grf_build_block_plan(grf_ctx* ctx, grf_features* feat, bool with_coef = true);

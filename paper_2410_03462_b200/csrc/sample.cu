@@ -253,6 +253,26 @@ compact_deposits_kernel(int32_t N, int32_t stage_stride, int32_t cap,
 // Re-modulation (Alg. 1 step 2 with new "learnable mask parameters (f_i)"): every entry's value is rebuilt from its
 // kept deposits as sum (f_t * load) * (1/n), the products and the sum taken in the sampler's operations and order.
 struct grf_remod_params { float f[2][GRF_MAX_WALK_LEN + 1]; float inv_n; };
+__global__ void index_as_float_kernel(int32_t n, float* __restrict__ out)
+{
+    const int32_t i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < n) out[i] = (float)i;
+}
+
+__global__ void float_to_index_kernel(int32_t n, const float* __restrict__ in, int32_t* __restrict__ out)
+{
+    const int32_t i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < n) out[i] = (int32_t)in[i];
+}
+
+// out[x] = src[perm[x]]: Psi^T's values from Psi's
+__global__ void gather_values_kernel(int32_t n, const int32_t* __restrict__ perm, const float* __restrict__ src,
+                                     float* __restrict__ out)
+{
+    const int32_t i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < n) out[i] = src[perm[i]];
+}
+
 __global__ void __launch_bounds__(256)
 remodulate_kernel(const __grid_constant__ grf_remod_params P, int32_t e, int64_t nnz, const int32_t* __restrict__ dep_ptr,
                   const unsigned char* __restrict__ dep_t, const float* __restrict__ dep_load, float* __restrict__ val)
@@ -388,6 +408,7 @@ static int sample_into(grf_ctx* ctx, grf_features* feat, const grf_walk_params& 
 
     const bool keep = ctx->keep_walks;
     feat->kept.valid = false;
+    feat->kept.perm_valid = false;
     if (keep) {
         GRF_TRY(grf_buf_reserve(&ctx->stage_dep_start, rows2 * stride * sizeof(int32_t)));
         GRF_TRY(grf_buf_reserve(&ctx->stage_dep_t, rows2 * (size_t)P.cap));
@@ -478,6 +499,7 @@ static int sample_into(grf_ctx* ctx, grf_features* feat, const grf_walk_params& 
         }
         GRF_CUDA_TRY(cudaGetLastError());
         K.n_walks = P.n_walks; K.max_len = P.max_len; K.valid = true;
+        K.perm_valid = false;
     }
 
     GRF_TRY(grf_transpose_launch(ctx, N, N, nnz_psi, (const int32_t*)feat->psi.rowptr.ptr,
@@ -570,13 +592,42 @@ extern "C" int grf_remodulate(grf_ctx* ctx, grf_features* feat, int32_t max_len,
             (const float*)K.dep_load[e].ptr, (float*)mats[e]->val.ptr);
     }
     GRF_CUDA_TRY(cudaGetLastError());
-    // Psi^T carries copies of Psi's values: regroup again (same structure, new values)
-    GRF_TRY(grf_transpose_launch(ctx, feat->psi.rows, feat->psi.cols, feat->psi.nnz, (const int32_t*)feat->psi.rowptr.ptr,
-                                 (const int32_t*)feat->psi.col.ptr, (const float*)feat->psi.val.ptr,
-                                 (int32_t*)feat->psit.rowptr.ptr, (int32_t*)feat->psit.col.ptr,
-                                 (float*)feat->psit.val.ptr));
-    feat->plan_stale = true;       // the coefficient table of the tensor-core gather holds Phi's old values
-    feat->plan_ready = false;
-    grf_mask_invalidate(feat);
+    // Psi^T carries copies of Psi's values in another order, which does not change with the coefficients: the first
+    // re-modulation regroups the entries' own indices (exact in fp32 below 2^24 entries) and keeps the result; from then
+    // on the new values are fetched through it
+    const int64_t nnz_psi = feat->psi.nnz;
+    if (nnz_psi > 0 && nnz_psi < (1ll << 24)) {
+        const int blocks = grf_ceil_div(nnz_psi, 256);
+        if (!K.perm_valid) {
+            if (K.psit_perm.bytes < (size_t)nnz_psi * 4) GRF_TRY(grf_buf_reserve(&K.psit_perm, ((size_t)nnz_psi + (size_t)nnz_psi / 8 + 64) * 4));
+            {
+                grf_launch_scope scope(ctx, 2);
+                index_as_float_kernel<<<blocks, 256, 0, ctx->stream>>>((int32_t)nnz_psi, (float*)K.psit_perm.ptr);
+            }
+            GRF_TRY(grf_transpose_launch(ctx, feat->psi.rows, feat->psi.cols, nnz_psi, (const int32_t*)feat->psi.rowptr.ptr,
+                                         (const int32_t*)feat->psi.col.ptr, (const float*)K.psit_perm.ptr,
+                                         (int32_t*)feat->psit.rowptr.ptr, (int32_t*)feat->psit.col.ptr,
+                                         (float*)feat->psit.val.ptr));
+            {
+                grf_launch_scope scope(ctx, 2);
+                float_to_index_kernel<<<blocks, 256, 0, ctx->stream>>>((int32_t)nnz_psi, (const float*)feat->psit.val.ptr,
+                                                                       (int32_t*)K.psit_perm.ptr);
+            }
+            K.perm_valid = true;
+        }
+        grf_launch_scope scope(ctx, 2);
+        gather_values_kernel<<<blocks, 256, 0, ctx->stream>>>((int32_t)nnz_psi, (const int32_t*)K.psit_perm.ptr,
+                                                              (const float*)feat->psi.val.ptr, (float*)feat->psit.val.ptr);
+    } else {
+        GRF_TRY(grf_transpose_launch(ctx, feat->psi.rows, feat->psi.cols, feat->psi.nnz, (const int32_t*)feat->psi.rowptr.ptr,
+                                     (const int32_t*)feat->psi.col.ptr, (const float*)feat->psi.val.ptr,
+                                     (int32_t*)feat->psit.rowptr.ptr, (int32_t*)feat->psit.col.ptr,
+                                     (float*)feat->psit.val.ptr));
+    }
+    GRF_CUDA_TRY(cudaGetLastError());
+    // the structure is the same: the block plan's node lists and the mask's key lists stay; the gather kernel's
+    // coefficient table and the mask's values hold the old values
+    feat->plan_coef_ready = false;
+    grf_mask_values_stale(feat);
     return GRF_OK;
 }

@@ -115,6 +115,65 @@ def test_attention_after_remodulation_matches_oracle(lib):
     feat.free()
 
 
+def test_mask_after_remodulation_rebuilds_values_only_and_matches_a_full_build(lib):
+    """The materialised mask after new coefficients: its key lists and positions are kept (same walks, same
+    structure), only the values are formed again; they must equal, bit for bit, those of a mask built from scratch
+    on a fresh object with the same coefficients, and the oracle's rows of Phi Psi^T within the bf16 bound."""
+    api, B, ctx = lib
+    w = configs.point_cloud_4096(1000)                       # ragged last block
+    g = w.graph()
+    N = g.N
+    dg = api.DeviceGraph(g)
+    f0 = oracle.deconvolve(w.alpha).astype(np.float32)
+    f1 = (f0 * np.linspace(1.0, -0.3, w.max_len + 1)).astype(np.float32)      # mixed signs
+    f1[2] = 0.0
+    B.grf_ctx_keep_walks(ctx.handle, True)
+    feat = api.sample(ctx, dg, configs.WALK_SEED, w.n_walks, w.p_halt, w.max_len, f0)
+    fresh = api.sample(ctx, dg, configs.WALK_SEED, w.n_walks, w.p_halt, w.max_len, f1)
+    B.grf_ctx_keep_walks(ctx.handle, False)
+    B.grf_features_materialise(ctx.handle, feat.handle)      # structure and values for f0
+    stats0 = B.grf_mask_stats(feat.handle)
+    launches0 = ctx.launches
+    B.grf_features_materialise(ctx.handle, fresh.handle)
+    full_build = ctx.launches - launches0
+    B.grf_remodulate(ctx.handle, feat.handle, w.max_len, f1, None)
+    with pytest.raises(B.GrfError):                           # the old values are not served
+        B.grf_mask_stats(feat.handle)
+    launches0 = ctx.launches
+    B.grf_features_materialise(ctx.handle, feat.handle)
+    assert ctx.launches - launches0 == 1 < full_build         # the values kernel alone
+    assert B.grf_mask_stats(feat.handle) == stats0 == B.grf_mask_stats(fresh.handle)
+    rows = torch.arange(N, dtype=torch.int32, device="cuda")
+    a = torch.empty((N, N), dtype=torch.float32, device="cuda")
+    b = torch.empty_like(a)
+    B.grf_mask_rows(ctx.handle, feat.handle, N, rows, a)
+    B.grf_mask_rows(ctx.handle, fresh.handle, N, rows, b)
+    torch.cuda.synchronize()
+    assert torch.equal(a, b)
+    traj, load = oracle.walks(g.rowptr, g.col, g.w, configs.WALK_SEED, w.n_walks, w.p_halt, w.max_len)
+    Phi = oracle.features_from_walks(traj, load, 0, f1, keep_zero=True)
+    Psi = oracle.features_from_walks(traj, load, 1, f1, keep_zero=True)
+    sel = sorted(set([0, 1, N // 2, N - 1] + list(range(0, N, 29))))
+    want = oracle.mask_rows(Phi, Psi, sel)
+    got = a[sel].cpu().numpy().astype(np.float64)
+    assert (np.abs(got - want) <= 2.0 ** -8 * np.abs(want) + 1e-37).all()
+    # and the attention over it
+    q, k, v = tensors.qkv(2, N, w.m, 64, "bf16", configs.QKV_SEED)
+    out1 = api.masked_attn_mhat(ctx, feat, q.cuda(), k.cuda(), v.cuda())
+    out2 = api.masked_attn_mhat(ctx, fresh, q.cuda(), k.cuda(), v.cuda())
+    torch.cuda.synchronize()
+    B.grf_ctx_check(ctx.handle)
+    assert torch.equal(out1, out2)
+    # resampling drops the structure as well
+    feat.handle = B.grf_sample(ctx.handle, N, dg.rowptr, dg.col, dg.w, configs.WALK_SEED + 1, w.n_walks, w.p_halt, w.max_len,
+                               f1, None, feat.handle)
+    launches0 = ctx.launches
+    B.grf_features_materialise(ctx.handle, feat.handle)
+    assert ctx.launches - launches0 > 1
+    feat.free()
+    fresh.free()
+
+
 def test_remodulate_rejects_objects_without_deposits(lib):
     api, B, ctx = lib
     w = configs.tiny()
