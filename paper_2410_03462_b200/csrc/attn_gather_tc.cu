@@ -383,7 +383,10 @@ __global__ void __launch_bounds__(32) wait_timeout_probe_kernel(long long limit_
 // ---------------------------------------------------------------------------------------------------
 // Block plan: for every block of BQ consecutive rows of Phi, the sorted list of distinct columns.
 
-__global__ void __launch_bounds__(256)
+constexpr int PLAN_THREADS = 1024;   // one CTA per block: the passes over the block's non-zeros use all of them,
+                                     // the ordered parts (one contiguous range of bitmap words per thread) the first 256
+
+__global__ void __launch_bounds__(PLAN_THREADS)
 block_plan_kernel(int32_t N, int32_t R, const int32_t* __restrict__ rowptr, const int32_t* __restrict__ col,
                   int32_t* __restrict__ plan_off, int32_t* __restrict__ plan_cnt, int32_t* __restrict__ plan_col,
                   int32_t* __restrict__ plan_total)
@@ -394,17 +397,17 @@ block_plan_kernel(int32_t N, int32_t R, const int32_t* __restrict__ rowptr, cons
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int32_t blk = blockIdx.x;
     const int32_t words = (R + 31) >> 5;
-    for (int32_t x = tid; x < words; x += 256) bitmap[x] = 0u;
+    for (int32_t x = tid; x < words; x += PLAN_THREADS) bitmap[x] = 0u;
     __syncthreads();
     const int32_t r0 = blk * BQ, r1 = min(N, r0 + BQ);
-    for (int32_t p = rowptr[r0] + tid; p < rowptr[r1]; p += 256) {
+    for (int32_t p = rowptr[r0] + tid; p < rowptr[r1]; p += PLAN_THREADS) {
         const int32_t c = col[p];
         atomicOr(&bitmap[c >> 5], 1u << (c & 31));
     }
     __syncthreads();
-    // each thread owns a contiguous range of words so that the output stays sorted
+    // each of the first 256 threads owns a contiguous range of words so that the output stays sorted
     const int32_t per = (words + 255) / 256;
-    const int32_t w0 = min(words, tid * per), w1 = min(words, w0 + per);
+    const int32_t w0 = min(words, min(tid, 256) * per), w1 = tid < 256 ? min(words, w0 + per) : w0;
     int32_t mine = 0;
     for (int32_t x = w0; x < w1; ++x) mine += __popc(bitmap[x]);
     int32_t inc = mine;
@@ -413,10 +416,10 @@ block_plan_kernel(int32_t N, int32_t R, const int32_t* __restrict__ rowptr, cons
         const int32_t y = __shfl_up_sync(0xffffffffu, inc, o);
         if (lane >= o) inc += y;
     }
-    if (lane == 31) warp_sums[warp] = inc;
+    if (lane == 31 && warp < 8) warp_sums[warp] = inc;
     __syncthreads();
     int32_t before = inc - mine;
-    for (int w = 0; w < warp; ++w) before += warp_sums[w];
+    for (int w = 0; w < min(warp, 8); ++w) before += warp_sums[w];
     if (tid == 255) {
         // lists are padded to a multiple of four entries (the last column repeated, with zero coefficients)
         const int32_t total = before + mine, padded = (total + 3) & ~3;
@@ -426,6 +429,7 @@ block_plan_kernel(int32_t N, int32_t R, const int32_t* __restrict__ rowptr, cons
         plan_cnt[blk] = padded;
     }
     __syncthreads();
+    if (tid >= 256) return;
     int32_t o = base_off + before;
     for (int32_t x = w0; x < w1; ++x) {
         uint32_t bits = bitmap[x];
@@ -449,7 +453,7 @@ block_plan_kernel(int32_t N, int32_t R, const int32_t* __restrict__ rowptr, cons
 // Second pass of the plan: the block's coefficients as a dense table, four union entries (bf16) per 8-byte
 // word, [quad][row][4], so that a row thread of the gather kernel reads its coefficients with one coalesced
 // load per four union entries.
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(PLAN_THREADS)
 block_coef_kernel(int32_t N, int32_t R, const int32_t* __restrict__ rowptr, const int32_t* __restrict__ col,
                   const float* __restrict__ val, const int32_t* __restrict__ plan_off,
                   const int32_t* __restrict__ plan_cnt, __nv_bfloat16* __restrict__ plan_coef)
@@ -461,20 +465,20 @@ block_coef_kernel(int32_t N, int32_t R, const int32_t* __restrict__ rowptr, cons
     const int32_t words = (R + 31) >> 5;
     uint32_t* bitmap = smem_plan;
     int32_t* before_word = reinterpret_cast<int32_t*>(smem_plan + words);
-    for (int32_t x = tid; x < words; x += 256) bitmap[x] = 0u;
+    for (int32_t x = tid; x < words; x += PLAN_THREADS) bitmap[x] = 0u;
     __syncthreads();
     const int32_t r0 = blk * BQ, r1 = min(N, r0 + BQ);
-    for (int32_t p = rowptr[r0] + tid; p < rowptr[r1]; p += 256) {
+    for (int32_t p = rowptr[r0] + tid; p < rowptr[r1]; p += PLAN_THREADS) {
         const int32_t c = col[p];
         atomicOr(&bitmap[c >> 5], 1u << (c & 31));
     }
     // zero this block's part of the table meanwhile
     const int32_t off = plan_off[blk], cnt = plan_cnt[blk];
     uint4* tab4 = reinterpret_cast<uint4*>(plan_coef + (size_t)off * BQ);
-    for (int32_t x = tid; x < cnt * (BQ * 2 / 16); x += 256) tab4[x] = make_uint4(0u, 0u, 0u, 0u);
+    for (int32_t x = tid; x < cnt * (BQ * 2 / 16); x += PLAN_THREADS) tab4[x] = make_uint4(0u, 0u, 0u, 0u);
     __syncthreads();
     const int32_t per = (words + 255) / 256;
-    const int32_t w0 = min(words, tid * per), w1 = min(words, w0 + per);
+    const int32_t w0 = min(words, min(tid, 256) * per), w1 = tid < 256 ? min(words, w0 + per) : w0;
     int32_t mine = 0;
     for (int32_t x = w0; x < w1; ++x) mine += __popc(bitmap[x]);
     int32_t inc = mine;
@@ -483,14 +487,14 @@ block_coef_kernel(int32_t N, int32_t R, const int32_t* __restrict__ rowptr, cons
         const int32_t y = __shfl_up_sync(0xffffffffu, inc, o);
         if (lane >= o) inc += y;
     }
-    if (lane == 31) warp_sums[warp] = inc;
+    if (lane == 31 && warp < 8) warp_sums[warp] = inc;
     __syncthreads();
     int32_t run = inc - mine;
-    for (int w = 0; w < warp; ++w) run += warp_sums[w];
+    for (int w = 0; w < min(warp, 8); ++w) run += warp_sums[w];
     for (int32_t x = w0; x < w1; ++x) { before_word[x] = run; run += __popc(bitmap[x]); }
     __syncthreads();
     __nv_bfloat16* tab = plan_coef + (size_t)off * BQ;
-    for (int32_t r = r0 + warp; r < r1; r += 8)
+    for (int32_t r = r0 + warp; r < r1; r += PLAN_THREADS / 32)
         for (int32_t p = rowptr[r] + lane; p < rowptr[r + 1]; p += 32) {
             const int32_t c = col[p];
             const int32_t u = before_word[c >> 5] + __popc(bitmap[c >> 5] & ((1u << (c & 31)) - 1u));
@@ -525,7 +529,7 @@ static int build_plan_coefficients(grf_ctx* ctx, grf_features* feat)
     GRF_CUDA_TRY(cudaFuncSetAttribute(block_coef_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(words * 8)));
     {
         grf_launch_scope scope(ctx, 7);
-        block_coef_kernel<<<feat->plan_blocks, 256, words * 8, ctx->stream>>>(
+        block_coef_kernel<<<feat->plan_blocks, PLAN_THREADS, words * 8, ctx->stream>>>(
             N, R, (const int32_t*)phi.rowptr.ptr, (const int32_t*)phi.col.ptr, (const float*)phi.val.ptr,
             (const int32_t*)feat->plan_off.ptr, (const int32_t*)feat->plan_cnt.ptr, (__nv_bfloat16*)feat->plan_coef.ptr);
     }
@@ -551,7 +555,7 @@ int grf_build_block_plan(grf_ctx* ctx, grf_features* feat, bool with_coef)
     GRF_CUDA_TRY(cudaFuncSetAttribute(block_plan_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(words * 4)));
     {
         grf_launch_scope scope(ctx, 7);
-        block_plan_kernel<<<nblocks, 256, words * 4, ctx->stream>>>(
+        block_plan_kernel<<<nblocks, PLAN_THREADS, words * 4, ctx->stream>>>(
             N, R, (const int32_t*)phi.rowptr.ptr, (const int32_t*)phi.col.ptr, (int32_t*)feat->plan_off.ptr,
             (int32_t*)feat->plan_cnt.ptr, (int32_t*)feat->plan_col.ptr, (int32_t*)feat->plan_total.ptr);
     }

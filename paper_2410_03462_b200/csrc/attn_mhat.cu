@@ -31,7 +31,9 @@ constexpr int KT = GRF_MASK_TILE;       // keys per tile
 // A warp takes 32 nodes at a time (lane x holds node x's extent in Psi^T) and fetches the keys of four nodes
 // together, so that several loads are in flight.  The bitmap and the count (padded to whole tiles) are kept.
 
-__global__ void __launch_bounds__(256)
+constexpr int MASK_BITMAP_THREADS = 1024;     // one CTA per block: many warps, each with a few batches of 32 nodes
+
+__global__ void __launch_bounds__(MASK_BITMAP_THREADS)
 mask_bitmap_kernel(int32_t Nk, const int32_t* __restrict__ plan_off, const int32_t* __restrict__ plan_cnt,
                    const int32_t* __restrict__ plan_col, const int32_t* __restrict__ t_rowptr,
                    const int32_t* __restrict__ t_col, uint32_t* __restrict__ bits, int32_t* __restrict__ mk_cnt)
@@ -41,11 +43,11 @@ mask_bitmap_kernel(int32_t Nk, const int32_t* __restrict__ plan_off, const int32
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int32_t blk = blockIdx.x;
     const int32_t words = (Nk + 31) >> 5;
-    for (int32_t x = tid; x < words; x += 256) bitmap[x] = 0u;
+    for (int32_t x = tid; x < words; x += MASK_BITMAP_THREADS) bitmap[x] = 0u;
     __syncthreads();
     const int32_t* ulist = plan_col + plan_off[blk];
     const int32_t ucnt = plan_cnt[blk];
-    for (int32_t u0 = warp * 32; u0 < ucnt; u0 += 8 * 32) {
+    for (int32_t u0 = warp * 32; u0 < ucnt; u0 += MASK_BITMAP_THREADS) {
         const int32_t n = min(32, ucnt - u0);
         const int32_t my_l = lane < n ? __ldg(ulist + u0 + lane) : 0;
         const int32_t my_beg = lane < n ? __ldg(t_rowptr + my_l) : 0;
@@ -76,9 +78,9 @@ mask_bitmap_kernel(int32_t Nk, const int32_t* __restrict__ plan_off, const int32
         }
     }
     __syncthreads();
-    // the bitmap, and behind it the number of set bits before each of its words
+    // the bitmap, and behind it the number of set bits before each of its words (the first 256 threads)
     const int32_t per = (words + 255) / 256;
-    const int32_t w0 = min(words, tid * per), w1 = min(words, w0 + per);
+    const int32_t w0 = min(words, min(tid, 256) * per), w1 = tid < 256 ? min(words, w0 + per) : w0;
     int32_t mine = 0;
     for (int32_t x = w0; x < w1; ++x) mine += __popc(bitmap[x]);
     int32_t inc = mine;
@@ -87,8 +89,9 @@ mask_bitmap_kernel(int32_t Nk, const int32_t* __restrict__ plan_off, const int32
         const int32_t y = __shfl_up_sync(0xffffffffu, inc, o);
         if (lane >= o) inc += y;
     }
-    if (lane == 31) warp_sums[warp] = inc;
+    if (lane == 31 && warp < 8) warp_sums[warp] = inc;
     __syncthreads();
+    if (tid >= 256) return;
     int32_t run = inc - mine;
     for (int w = 0; w < warp; ++w) run += warp_sums[w];
     uint32_t* dst = bits + (size_t)blk * 2 * words;
@@ -965,7 +968,7 @@ extern "C" int grf_features_materialise(grf_ctx* ctx, grf_features* feat)
     GRF_CUDA_TRY(cudaFuncSetAttribute(mask_bitmap_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(words * 4)));
     {
         grf_launch_scope scope(ctx, 8);
-        mask_bitmap_kernel<<<nblocks, 256, words * 4, ctx->stream>>>(
+        mask_bitmap_kernel<<<nblocks, MASK_BITMAP_THREADS, words * 4, ctx->stream>>>(
             Nk, (const int32_t*)feat->plan_off.ptr, (const int32_t*)feat->plan_cnt.ptr, (const int32_t*)feat->plan_col.ptr,
             (const int32_t*)feat->psit.rowptr.ptr, (const int32_t*)feat->psit.col.ptr, (uint32_t*)K.bits.ptr,
             (int32_t*)K.cnt.ptr);
