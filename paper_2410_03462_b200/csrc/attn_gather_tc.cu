@@ -292,10 +292,23 @@ gather_contract_tc_kernel(int32_t G, int32_t nblocks, int32_t N, int32_t R, cons
 
 // ---------------------------------------------------------------------------------------------------
 // Denominators of Eq. 12 for the tensor-core path: den_i = phi(q_i) . (sum_l Phi_il z_l), one warp per
-// (problem, query); m/2 lanes take one node's z_l (its bf16 copy in the record, two components per lane), so a
-// warp handles 64/m nodes side by side.
+// (problem, query); m/4 lanes take one node's z_l (its bf16 copy in the record, four components = 8 bytes per lane),
+// so a warp handles 128/m nodes side by side; the sums run on packed pairs of fp32.
 
 constexpr int DEN_GH = 4;   // problems per warp of the denominators kernel: they share the row's indices and coefficients
+
+__device__ __forceinline__ uint64_t den_pack2(uint32_t lo, uint32_t hi)
+{
+    uint64_t r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "r"(lo), "r"(hi));
+    return r;
+}
+__device__ __forceinline__ uint64_t den_fma2(uint64_t a, uint64_t b, uint64_t c)
+{
+    uint64_t r;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c));
+    return r;
+}
 
 template <int M, int D>
 __global__ void __launch_bounds__(256)
@@ -303,22 +316,20 @@ row_denominators_kernel(int32_t G, int32_t N, int32_t R, const int32_t* __restri
                         const float* __restrict__ val, const __nv_bfloat16* __restrict__ phiQ,
                         const unsigned char* __restrict__ records, float* __restrict__ den)
 {
-    constexpr int LPL = M / 2 < 32 ? M / 2 : 32;            // lanes per node: each takes pairs of components (bf16 x 2)
+    constexpr int LPL = M / 4;                              // lanes per node: each takes four components (bf16 x 4)
     constexpr int LPW = 32 / LPL;                           // nodes handled side by side in a warp
-    constexpr int NT = (M / 2) / LPL;                       // pairs per lane
     constexpr size_t REC = (size_t)M * D * 2 + (size_t)M * 4 + (size_t)M * 2;
+    static_assert(LPL >= 1 && LPL <= 32 && REC % 8 == 0, "layout");
     const int lane = threadIdx.x & 31;
     const int sub = lane / LPL, pl = lane % LPL;
     const int32_t i = blockIdx.x * 8 + (threadIdx.x >> 5);
     const int32_t g0 = blockIdx.y * DEN_GH;
     if (i >= N) return;
     const size_t gstride = (size_t)R * REC;                 // from one problem's records to the next one's
-    const unsigned char* zbase = records + (size_t)g0 * gstride + (size_t)M * D * 2 + (size_t)M * 4;   // the bf16 copy of z
-    float z0[DEN_GH][NT], z1[DEN_GH][NT];
+    const unsigned char* zbase = records + (size_t)g0 * gstride + (size_t)M * D * 2 + (size_t)M * 4 + (size_t)pl * 8;   // the bf16 copy of z
+    uint64_t z01[DEN_GH], z23[DEN_GH];                      // components 0,1 and 2,3 of this lane's four
 #pragma unroll
-    for (int h = 0; h < DEN_GH; ++h)
-#pragma unroll
-        for (int t = 0; t < NT; ++t) { z0[h][t] = 0.0f; z1[h][t] = 0.0f; }
+    for (int h = 0; h < DEN_GH; ++h) { z01[h] = 0ull; z23[h] = 0ull; }
     const int32_t beg = rowptr[i], end = rowptr[i + 1];
     for (int32_t p0 = beg; p0 < end; p0 += 32) {
         const int32_t n = min(32, end - p0);
@@ -329,34 +340,31 @@ row_denominators_kernel(int32_t G, int32_t N, int32_t R, const int32_t* __restri
             const int32_t l = __shfl_sync(0xffffffffu, c_mine, jj & 31);
             const float phi = __shfl_sync(0xffffffffu, v_mine, jj & 31);
             if (jj < n) {
-                const uint32_t* zl = reinterpret_cast<const uint32_t*>(zbase + (size_t)l * REC) + pl;
-                uint32_t w[DEN_GH][NT];
+                const unsigned char* zl = zbase + (size_t)l * REC;
+                uint2 w[DEN_GH];
 #pragma unroll
                 for (int h = 0; h < DEN_GH; ++h)
+                    w[h] = g0 + h < G ? __ldg(reinterpret_cast<const uint2*>(zl + (size_t)h * gstride)) : make_uint2(0u, 0u);
+                const uint64_t phi2 = den_pack2(__float_as_uint(phi), __float_as_uint(phi));
 #pragma unroll
-                    for (int t = 0; t < NT; ++t)
-                        w[h][t] = g0 + h < G ? __ldg(reinterpret_cast<const uint32_t*>(reinterpret_cast<const unsigned char*>(zl) + (size_t)h * gstride) + LPL * t) : 0u;
-#pragma unroll
-                for (int h = 0; h < DEN_GH; ++h)
-#pragma unroll
-                    for (int t = 0; t < NT; ++t) {
-                        z0[h][t] = fmaf(phi, __uint_as_float(w[h][t] << 16), z0[h][t]);
-                        z1[h][t] = fmaf(phi, __uint_as_float(w[h][t] & 0xffff0000u), z1[h][t]);
-                    }
+                for (int h = 0; h < DEN_GH; ++h) {
+                    z01[h] = den_fma2(phi2, den_pack2(w[h].x << 16, w[h].x & 0xffff0000u), z01[h]);
+                    z23[h] = den_fma2(phi2, den_pack2(w[h].y << 16, w[h].y & 0xffff0000u), z23[h]);
+                }
             }
         }
     }
 #pragma unroll
     for (int h = 0; h < DEN_GH; ++h) {
         if (g0 + h >= G) break;
-        const uint32_t* q = reinterpret_cast<const uint32_t*>(phiQ + ((size_t)(g0 + h) * N + i) * M);
-        float d = 0.0f;
-#pragma unroll
-        for (int t = 0; t < NT; ++t) {
-            const uint32_t w = __ldg(q + pl + LPL * t);
-            d = fmaf(__uint_as_float(w << 16), z0[h][t], d);
-            d = fmaf(__uint_as_float(w & 0xffff0000u), z1[h][t], d);
-        }
+        const uint2 q = __ldg(reinterpret_cast<const uint2*>(phiQ + ((size_t)(g0 + h) * N + i) * M) + pl);
+        float a0, a1, a2, a3;
+        asm("mov.b64 {%0, %1}, %2;" : "=f"(a0), "=f"(a1) : "l"(z01[h]));
+        asm("mov.b64 {%0, %1}, %2;" : "=f"(a2), "=f"(a3) : "l"(z23[h]));
+        float d = __uint_as_float(q.x << 16) * a0;
+        d = fmaf(__uint_as_float(q.x & 0xffff0000u), a1, d);
+        d = fmaf(__uint_as_float(q.y << 16), a2, d);
+        d = fmaf(__uint_as_float(q.y & 0xffff0000u), a3, d);
 #pragma unroll
         for (int off = 1; off < 32; off <<= 1) d += __shfl_xor_sync(0xffffffffu, d, off);
         if (lane == 0) den[(size_t)(g0 + h) * N + i] = d;
