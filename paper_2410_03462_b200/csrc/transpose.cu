@@ -31,33 +31,87 @@ bucket_scatter_kernel(int32_t rows, const int32_t* __restrict__ rowptr, const in
 }
 
 constexpr int BUCKET_SMEM = 1024;  // entries of one bucket staged per warp
+constexpr int BUCKET_RANKED = 192; // up to this length ranking (len^2 / 32 comparisons per lane) beats the sorting network
 
-// One warp per bucket: each element's final position is the number of bucket entries with a smaller
-// source row (rows are distinct).  Buckets longer than the staging area are ranked from global memory.
+// A warp sorts n (row, value) pairs by row, ascending, in place (shared or global memory): a bitonic network whose
+// comparators all point the same way (every merge starts by comparing i with its mirror image in the block), so
+// that a length that is no power of two needs no padding: a comparator whose upper end lies beyond n is skipped.
+__device__ __forceinline__ void warp_sort_pairs(int32_t* rows, float* vals, int32_t n, int lane)
+{
+    int32_t P = 1;
+    while (P < n) P <<= 1;
+    auto exchange = [&](int32_t a, int32_t b) {
+        if (b < n) {
+            const int32_t ra = rows[a], rb = rows[b];
+            if (rb < ra) {
+                rows[a] = rb; rows[b] = ra;
+                const float va = vals[a]; vals[a] = vals[b]; vals[b] = va;
+            }
+        }
+    };
+    for (int32_t k = 2; k <= P; k <<= 1) {
+        const int32_t h = k >> 1;
+        for (int32_t i = lane; i < (P >> 1); i += 32) {
+            const int32_t blk = i / h, off = i - blk * h;
+            exchange(blk * k + off, blk * k + (k - 1 - off));
+        }
+        __syncwarp();
+        for (int32_t j = h >> 1; j >= 1; j >>= 1) {
+            for (int32_t i = lane; i < (P >> 1); i += 32) {
+                const int32_t a = (i / j) * 2 * j + (i % j);
+                exchange(a, a + j);
+            }
+            __syncwarp();
+        }
+    }
+}
+
+// One warp per bucket: its entries are ordered by source row (rows are distinct, so the result is unique).  This
+// kernel takes the buckets of up to BUCKET_RANKED entries: each element's place is the number of smaller rows.
 __global__ void __launch_bounds__(128)
 bucket_order_kernel(int32_t cols, const int32_t* __restrict__ t_rowptr,
                     const int32_t* __restrict__ tmp_row, const float* __restrict__ tmp_val,
                     int32_t* __restrict__ t_col, float* __restrict__ t_val)
 {
-    __shared__ int32_t staged[4][BUCKET_SMEM];
+    __shared__ int32_t staged[4][BUCKET_RANKED];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int32_t c = blockIdx.x * 4 + warp;
     if (c >= cols) return;
     const int32_t beg = t_rowptr[c], len = t_rowptr[c + 1] - beg;
-    const bool in_smem = len <= BUCKET_SMEM;
-    if (in_smem)
-        for (int32_t x = lane; x < len; x += 32) staged[warp][x] = tmp_row[beg + x];
+    if (len > BUCKET_RANKED) return;
+    for (int32_t x = lane; x < len; x += 32) staged[warp][x] = tmp_row[beg + x];
     __syncwarp();
     for (int32_t x = lane; x < len; x += 32) {
-        const int32_t mine = in_smem ? staged[warp][x] : tmp_row[beg + x];
+        const int32_t mine = staged[warp][x];
         int32_t rank = 0;
-        if (in_smem) {
-            for (int32_t y = 0; y < len; ++y) rank += staged[warp][y] < mine;
-        } else {
-            for (int32_t y = 0; y < len; ++y) rank += tmp_row[beg + y] < mine;
-        }
+        for (int32_t y = 0; y < len; ++y) rank += staged[warp][y] < mine;
         t_col[beg + rank] = mine;
         t_val[beg + rank] = tmp_val[beg + x];
+    }
+}
+
+// The longer buckets (hub columns): sorted by the network above, in shared memory when they fit, else in place in
+// the scratch arrays.
+__global__ void __launch_bounds__(128)
+bucket_sort_long_kernel(int32_t cols, const int32_t* __restrict__ t_rowptr,
+                        int32_t* __restrict__ tmp_row, float* __restrict__ tmp_val,
+                        int32_t* __restrict__ t_col, float* __restrict__ t_val)
+{
+    __shared__ int32_t staged[4][BUCKET_SMEM];
+    __shared__ float staged_val[4][BUCKET_SMEM];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int32_t c = blockIdx.x * 4 + warp;
+    if (c >= cols) return;
+    const int32_t beg = t_rowptr[c], len = t_rowptr[c + 1] - beg;
+    if (len <= BUCKET_RANKED) return;
+    if (len <= BUCKET_SMEM) {
+        for (int32_t x = lane; x < len; x += 32) { staged[warp][x] = tmp_row[beg + x]; staged_val[warp][x] = tmp_val[beg + x]; }
+        __syncwarp();
+        warp_sort_pairs(staged[warp], staged_val[warp], len, lane);
+        for (int32_t x = lane; x < len; x += 32) { t_col[beg + x] = staged[warp][x]; t_val[beg + x] = staged_val[warp][x]; }
+    } else {
+        warp_sort_pairs(tmp_row + beg, tmp_val + beg, len, lane);
+        for (int32_t x = lane; x < len; x += 32) { t_col[beg + x] = tmp_row[beg + x]; t_val[beg + x] = tmp_val[beg + x]; }
     }
 }
 
@@ -97,11 +151,13 @@ int grf_transpose_launch(grf_ctx* ctx, int32_t rows, int32_t cols, int64_t nnz,
         copy_i32_kernel<<<grf_ceil_div(cols, 256), 256, 0, ctx->stream>>>(t_rowptr, cursor, cols);
     }
     if (nnz > 0) {
-        grf_launch_scope scope(ctx, 3, 2);
+        grf_launch_scope scope(ctx, 3, 3);
         bucket_scatter_kernel<<<grf_ceil_div(rows, 8), 256, 0, ctx->stream>>>(
             rows, rowptr, col, val, cursor, (int32_t*)ctx->t_tmp_col.ptr, (float*)ctx->t_tmp_val.ptr);
         bucket_order_kernel<<<grf_ceil_div(cols, 4), 128, 0, ctx->stream>>>(
             cols, t_rowptr, (const int32_t*)ctx->t_tmp_col.ptr, (const float*)ctx->t_tmp_val.ptr, t_col, t_val);
+        bucket_sort_long_kernel<<<grf_ceil_div(cols, 4), 128, 0, ctx->stream>>>(
+            cols, t_rowptr, (int32_t*)ctx->t_tmp_col.ptr, (float*)ctx->t_tmp_val.ptr, t_col, t_val);
     }
     GRF_CUDA_TRY(cudaGetLastError());
     return GRF_OK;
@@ -170,6 +226,7 @@ extern "C" int grf_csr_transpose_noalloc(int device, void* cuda_stream, int32_t 
     if (nnz > 0) {
         bucket_scatter_kernel<<<grf_ceil_div(rows, 8), 256, 0, stream>>>(rows, rowptr, col, val, cursor, tmp_row, tmp_val);
         bucket_order_kernel<<<grf_ceil_div(cols, 4), 128, 0, stream>>>(cols, t_rowptr, tmp_row, tmp_val, t_col, t_val);
+        bucket_sort_long_kernel<<<grf_ceil_div(cols, 4), 128, 0, stream>>>(cols, t_rowptr, tmp_row, tmp_val, t_col, t_val);
     }
     GRF_CUDA_TRY(cudaGetLastError());
     return GRF_OK;
