@@ -360,6 +360,33 @@ def test_transpose_standalone(lib):
     helpers.assert_csr_equal((t_rp.cpu().numpy(), t_c.cpu().numpy(), t_v.cpu().numpy()), want, "transpose", val_rtol=0)
 
 
+def test_transpose_columns_of_every_length_class(lib):
+    """Columns with 0, a few, a few hundred (sorted in shared memory) and several thousand entries (sorted in place),
+    rectangular, rows in arbitrary arrival order: the regrouped matrix must equal the oracle's, bit for bit."""
+    api, B, ctx = lib
+    rng = np.random.default_rng(11)
+    rows, cols = 6000, 40
+    want_len = [0, 1, 5, 31, 32, 33, 64, 100, 191, 192, 193, 200, 255, 256, 257, 500, 1000, 1023, 1024, 1025, 1500, 3000, 5999, 6000]
+    want_len += [int(x) for x in rng.integers(0, 400, cols - len(want_len))]
+    member = np.zeros((rows, cols), dtype=bool)
+    for c, n in enumerate(want_len):
+        member[rng.choice(rows, size=n, replace=False), c] = True
+    rp = np.zeros(rows + 1, dtype=np.int32)
+    rp[1:] = np.cumsum(member.sum(axis=1))
+    ci = np.nonzero(member)[1].astype(np.int32)           # row-major order: columns ascending inside a row
+    vals = rng.standard_normal(ci.size).astype(np.float32)
+    nnz = int(ci.size)
+    want = oracle.transpose(oracle.CSR(rp, ci, vals, None, (rows, cols)))
+    d = lambda a: torch.from_numpy(a).cuda()
+    t_rp = torch.empty(cols + 1, dtype=torch.int32, device="cuda")
+    t_c = torch.empty(nnz, dtype=torch.int32, device="cuda")
+    t_v = torch.empty(nnz, dtype=torch.float32, device="cuda")
+    B.grf_csr_transpose(ctx.handle, rows, cols, nnz, d(rp), d(ci), d(vals), t_rp, t_c, t_v)
+    torch.cuda.synchronize()
+    helpers.assert_csr_equal((t_rp.cpu().numpy(), t_c.cpu().numpy(), t_v.cpu().numpy()), want, "transpose, all length classes",
+                             val_rtol=0)
+
+
 def test_step_host_matches_device_path(lib):
     api, B, ctx = lib
     w = configs.point_cloud_4096(512)
