@@ -395,7 +395,12 @@ extern "C" int grf_step_host(grf_ctx* ctx, int32_t N, const int32_t* rowptr, con
         }
         GRF_CUDA_TRY(cudaEventCreateWithFlags(&ctx->down_done, cudaEventDisableTiming));
     }
-    const int parts = G >= 2 * grf_ctx::HOST_PARTS ? grf_ctx::HOST_PARTS : (G >= 2 ? 2 : 1);
+    // Two parts on the route through the per-node states, whose kernels lose more on small batches than the finer
+    // overlap returns (four parts were measured slower there); four on the route over the mask, whose attention is
+    // short, so that most of the outputs leave while later parts are computed.
+    const bool mask_shape = ctx->prefer_mask_route && dtype == GRF_DTYPE_BF16 && d == 64 && (m == 16 || m == 32 || m == 64);
+    const int want_parts = mask_shape ? grf_ctx::HOST_PARTS : 2;
+    const int parts = G >= 2 * want_parts ? want_parts : (G >= 2 ? 2 : 1);
     const int32_t gp = (G + parts - 1) / parts;           // problems per part
     for (int p = 0; p < parts; ++p) {
         const int32_t g0 = p * gp, gc = g0 + gp <= G ? gp : G - g0;

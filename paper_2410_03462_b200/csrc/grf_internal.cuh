@@ -48,7 +48,7 @@ struct grf_ctx {
     grf_features* h_feat = nullptr;
     // host-buffer path: phi(Q), phi(K), V are uploaded on one stream and the outputs downloaded on another, in
     // parts of a few problems each, beside the sampler and the attention of the other parts
-    static constexpr int HOST_PARTS = 2;
+    static constexpr int HOST_PARTS = 4;     // most parts grf_step_host splits a batch into
     cudaStream_t copy_stream = nullptr, down_stream = nullptr;
     cudaEvent_t up_done[HOST_PARTS] = {}, part_done[HOST_PARTS] = {}, down_done = nullptr;
     int32_t* pinned = nullptr;      // small pinned host block for read-backs
