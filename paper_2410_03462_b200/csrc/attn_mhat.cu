@@ -10,9 +10,9 @@
 //     S = phi(Q_blk) phi(K_tile)^T   (tcgen05, accumulator in tensor memory)
 //     P = S * Mhat_tile              (row threads: tensor memory -> registers -> tensor memory, bf16)
 //     O += P V_tile                  (tcgen05, P read from tensor memory)
-// and the row sums of P give the denominators.  Key and value rows are gathered by key index: value rows by the
-// tensor-map copy engine (tile::gather4) into the 128-byte-swizzled operand layout, key-feature rows by 16-byte
-// asynchronous copies into the unswizzled K-major layout.
+// and the row sums of P (taken in fp32, before its rounding) give the denominators.  Key and value rows are gathered
+// by key index with 16-byte asynchronous copies: value rows into the 128-byte-swizzled MN-major operand layout,
+// key-feature rows into the unswizzled K-major layout.
 //
 // Building the mask (once per feature object): the key list of a block is the union of the rows of Psi^T over the
 // block's node list (the block plan of Phi); the values are accumulated row by row, one warp per row, in ascending
